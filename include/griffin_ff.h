@@ -1,0 +1,184 @@
+/*
+ * griffin_ff.h -- C ABI of libgriffin_ff.so
+ *
+ * GRIFFIN (arXiv 2404.01365) for one gated feed-forward (FF) block of a decoder layer,
+ * as hand-written CUDA kernels for NVIDIA B200 (sm_100a).  Four steps:
+ *
+ *   griffin_ff_prefill_score   prompt phase: full FF over the S prompt tokens and the
+ *                              selection statistic s                       (Eqs. 1, 3, 6)
+ *   griffin_select_topk        expert set E = top-k of s                  (Section 4.2)
+ *   griffin_compact_experts    slice W_g, W_1 by rows and W_2 by columns  (Section 4.2)
+ *   griffin_ff_decode          generation phase: pruned FF on every new token (Eqs. 4, 5)
+ *
+ * Notation (Section 3 of the paper): d = D, d_ff = D_FF, w_gate = W_g [d_ff, d],
+ * w_up = W_1 [d_ff, d], w_down = W_2 [d, d_ff], b_gate/b_up/b_down = b_g/b_1/b_2,
+ * X [S, d] prompt hidden states, Z = FF_1(X) [S, d_ff], s [d_ff], E (k indices).
+ *
+ * General rules
+ *   - Every pointer is a DEVICE pointer unless its comment says "host".  All matrices are
+ *     dense row-major; base pointers must be 16-byte aligned; d and d_ff must be multiples
+ *     of 8.  `dtype` is the storage type of X, the weights, the biases and Y; scores are
+ *     always fp32 and indices int32.  Accumulation is always fp32.
+ *   - The library allocates no device memory and frees none: the caller owns every
+ *     buffer, including the workspace (size it with griffin_workspace_bytes and clear it
+ *     once with griffin_workspace_init).
+ *   - Every call validates its arguments on the host first; on a validation error nothing
+ *     is enqueued.  Work is enqueued on `stream` (a cudaStream_t passed as void*, NULL =
+ *     the default stream) and the call returns without synchronising.  The only call that
+ *     synchronises is griffin_check_device_status.
+ *   - Calls that share a workspace must be ordered on one stream (they may not overlap on
+ *     the GPU).
+ *   - No exceptions cross this boundary; every call returns a griffin_status.
+ */
+#ifndef GRIFFIN_FF_H
+#define GRIFFIN_FF_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define GRIFFIN_FF_VERSION 1
+#define GRIFFIN_MAX_BATCH 32      /* sequences per griffin_ff_decode call              */
+#define GRIFFIN_MAX_D 8192        /* largest model width the decode kernels accept     */
+#define GRIFFIN_MAX_COMBINE 256   /* samples per griffin_combine_scores call           */
+
+typedef enum {
+    GRIFFIN_OK = 0,
+    GRIFFIN_ERR_INVALID_ARG = 1,  /* null pointer, size out of range, k not in [1,d_ff] */
+    GRIFFIN_ERR_UNSUPPORTED = 2,  /* shape / dtype / activation this build cannot run   */
+    GRIFFIN_ERR_ALIGNMENT = 3,    /* a pointer or leading dimension is not 16-byte aligned */
+    GRIFFIN_ERR_WORKSPACE = 4,    /* workspace missing or smaller than griffin_workspace_bytes */
+    GRIFFIN_ERR_CUDA = 5,         /* a CUDA runtime call or a kernel launch failed      */
+    GRIFFIN_ERR_TIMEOUT = 6       /* a bounded device-side wait gave up (see griffin_check_device_status) */
+} griffin_status;
+
+/* Gate non-linearity sigma of Eq. 3 (the paper names the GLU variants in Section 1). */
+typedef enum {
+    GRIFFIN_ACT_SWIGLU = 0,       /* sigma(t) = t / (1 + exp(-t))                                   */
+    GRIFFIN_ACT_GEGLU_TANH = 1,   /* sigma(t) = t/2 (1 + tanh(sqrt(2/pi) (t + 0.044715 t^3)))       */
+    GRIFFIN_ACT_REGLU = 2         /* sigma(t) = max(t, 0)                                           */
+} griffin_act;
+
+typedef enum { GRIFFIN_DT_F32 = 0, GRIFFIN_DT_BF16 = 1 } griffin_dtype;
+
+/* Shape and types of one FF block (Section 3). */
+typedef struct {
+    int32_t d;                    /* model width D                                      */
+    int32_t d_ff;                 /* FF width D_FF                                      */
+    int32_t act;                  /* griffin_act                                        */
+    int32_t dtype;                /* griffin_dtype                                      */
+} griffin_ff_desc;
+
+/* Full weights of one FF block (Eqs. 1 and 3).  Biases may be NULL (= absent). */
+typedef struct {
+    const void *w_gate;           /* [d_ff, d]  W_g                                     */
+    const void *w_up;             /* [d_ff, d]  W_1                                     */
+    const void *w_down;           /* [d, d_ff]  W_2                                     */
+    const void *b_gate;           /* [d_ff] or NULL                                     */
+    const void *b_up;             /* [d_ff] or NULL                                     */
+    const void *b_down;           /* [d]    or NULL                                     */
+} griffin_ff_weights;
+
+/* Compact weights of one sequence's expert set (Section 3: W_g_hat, W_1_hat in R^{k x D},
+ * W_2_hat in R^{D x k}).  Rows of w_down_c are padded to ldk elements, ldk = k rounded up
+ * to a multiple of 8 (griffin_compact_ldk); the padding holds zeros.  With E = all neurons
+ * the full weights themselves are a valid compact set (k = ldk = d_ff), which is how the
+ * unpruned FF is run through the same decode kernels. */
+typedef struct {
+    void *w_gate_c;               /* [k, d]                                             */
+    void *w_up_c;                 /* [k, d]                                             */
+    void *w_down_c;               /* [d, ldk]                                           */
+    void *b_gate_c;               /* [k] or NULL                                        */
+    void *b_up_c;                 /* [k] or NULL                                        */
+    int32_t k;                    /* number of expert neurons                           */
+    int32_t ldk;                  /* leading dimension of w_down_c, >= k, multiple of 8 */
+} griffin_ff_compact;
+
+/* Flags of griffin_ff_decode. */
+#define GRIFFIN_DECODE_DEFAULT 0u
+/* Launch the decode kernels with programmatic dependent launch: each kernel may begin
+ * streaming its (read-only) weights into shared memory while the previous kernel on the
+ * stream is still finishing; it reads x and writes y / the workspace only after that
+ * kernel has completed.  The caller promises that no earlier work still running on the
+ * stream WRITES the compact weights this call reads (do not set it on the first decode
+ * call after griffin_compact_experts). */
+#define GRIFFIN_DECODE_OVERLAP_WEIGHT_PREFETCH 1u
+
+/* Status text for a code (static string, never NULL). */
+const char *griffin_status_string(griffin_status st);
+
+/* Library ABI version (GRIFFIN_FF_VERSION at build time). */
+int32_t griffin_version(void);
+
+/* k for a keep ratio (= 1 - the paper's "FF sparsity", Section 5): floor(keep*d_ff + 0.5)
+ * clamped to [1, d_ff].  Host-only arithmetic. */
+int32_t griffin_k_from_keep_ratio(int32_t d_ff, double keep);
+
+/* ldk for k experts: k rounded up to a multiple of 8. */
+int32_t griffin_compact_ldk(int32_t k);
+
+/* Bytes of workspace that any call on this FF shape needs, for prompts of at most S_max
+ * tokens and at most n_seq_max sequences per decode call.  Returns 0 if desc is NULL or
+ * invalid. */
+size_t griffin_workspace_bytes(const griffin_ff_desc *desc, int32_t S_max, int32_t n_seq_max);
+
+/* Clears the workspace header (device status word).  Enqueue once before first use. */
+griffin_status griffin_workspace_init(void *workspace, size_t ws_bytes, void *stream);
+
+/* Prompt phase (Section 4.2, "Prompt Phase Expert Neuron Selection").
+ *   y[S, d]      = FF(X) = (sigma(X W_g^T + b_g) * (X W_1^T + b_1)) W_2^T + b_2   (Eqs. 1, 3)
+ *                  -- the full block, never pruned, independent of k;
+ *   score[d_ff]  = s, s_j = || column j of Zbar ||_2, Zbar_i = Z_i / ||Z_i||_2   (Eq. 6);
+ *                  a token whose activation row is all zero contributes nothing.
+ * x [S, d] in, y [S, d] out (dtype of desc), score fp32 out.  1 <= S.  Z is held in the
+ * workspace in the storage dtype.  y may be NULL to skip the down projection. */
+griffin_status griffin_ff_prefill_score(const griffin_ff_desc *desc, const griffin_ff_weights *w,
+                                        const void *x, int32_t S, void *y, float *score,
+                                        void *workspace, size_t ws_bytes, void *stream);
+
+/* Expert selection (Section 4.2): for each of n_seq score vectors, the indices of its k
+ * largest entries, written in ascending index order; equal scores go to the lower index.
+ * score [n_seq, d_ff] fp32 in, idx [n_seq, k] int32 out.  Scores must not be NaN. */
+griffin_status griffin_select_topk(const float *score, int32_t n_seq, int32_t d_ff, int32_t k,
+                                   int32_t *idx, void *stream);
+
+/* Batch statistic s_bar = sum_i s_i / sqrt(S_i) (Eq. 7) for sharing one expert set among
+ * n_seq <= GRIFFIN_MAX_COMBINE samples.  score [n_seq, d_ff] fp32 in, prompt_len: HOST
+ * array of n_seq lengths (each >= 1), out [d_ff] fp32. */
+griffin_status griffin_combine_scores(const float *score, const int32_t *prompt_len /*host*/,
+                                      int32_t n_seq, int32_t d_ff, float *out, void *stream);
+
+/* Expert compaction (Section 4.2): out.w_gate_c = W_g[E, :], out.w_up_c = W_1[E, :],
+ * out.w_down_c[:, 0:k] = W_2[:, E] (padding columns k..ldk zeroed), and the matching bias
+ * entries when both the source bias and the destination are non-NULL.  Bit copies.
+ * idx [k] int32, every entry in [0, d_ff); an out-of-range entry is not dereferenced: its
+ * row / column is filled with zeros and, when `workspace` is not NULL, the device status
+ * word is raised.  out->k and out->ldk must be set by the caller (ldk from
+ * griffin_compact_ldk).  Source and destination buffers must not overlap. */
+griffin_status griffin_compact_experts(const griffin_ff_desc *desc, const griffin_ff_weights *w,
+                                       const int32_t *idx, const griffin_ff_compact *out,
+                                       void *workspace /*may be NULL*/, void *stream);
+
+/* Generation phase (Eqs. 4, 5): for each of B sequences, with its own compact set,
+ *   y[b] = W_2_hat (sigma(W_g_hat x[b] + b_g_hat) * (W_1_hat x[b] + b_1_hat)) + b_2.
+ * sets: HOST array of B structs (entries may repeat to share a set); every set must have
+ * the same k and ldk.  b_down [d] or NULL is shared by all sequences.  x [B, d] in,
+ * y [B, d] out.  1 <= B <= GRIFFIN_MAX_BATCH, d <= GRIFFIN_MAX_D.  flags: GRIFFIN_DECODE_*.
+ * The activations z_hat [B, ldk] live in the workspace as fp32 between the two kernels. */
+griffin_status griffin_ff_decode(const griffin_ff_desc *desc, int32_t B,
+                                 const griffin_ff_compact *sets /*host*/, const void *b_down,
+                                 const void *x, void *y, void *workspace, size_t ws_bytes,
+                                 uint32_t flags, void *stream);
+
+/* Synchronises `stream`, then reads the workspace's device status word.  GRIFFIN_OK,
+ * GRIFFIN_ERR_TIMEOUT (a bounded wait inside a kernel gave up), GRIFFIN_ERR_INVALID_ARG
+ * (a kernel met an out-of-range expert index) or GRIFFIN_ERR_CUDA. */
+griffin_status griffin_check_device_status(const void *workspace, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GRIFFIN_FF_H */
