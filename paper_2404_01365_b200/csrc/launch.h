@@ -1,0 +1,41 @@
+// Host-side launchers behind the C ABI (one per kernel family).  Arguments are already
+// validated by the caller in api.cu.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "griffin_ff.h"
+
+namespace griffin {
+
+// Number of SMs of the current device (cached per device); <= 0 on error.
+int device_sm_count();
+
+// Raises the opt-in dynamic shared memory limit of `fn` on the current device when needed.
+cudaError_t ensure_dynamic_smem(const void *fn, size_t bytes);
+
+griffin_status launch_decode(const griffin_ff_desc *desc, int B, const griffin_ff_compact *sets, const void *b_down,
+                             const void *x, void *y, float *z, void *ws, uint32_t flags, cudaStream_t stream);
+
+griffin_status launch_select_topk(const float *score, int n_seq, int d_ff, int k, int32_t *idx, cudaStream_t stream);
+
+griffin_status launch_combine_scores(const float *score, const int32_t *prompt_len_host, int n_seq, int d_ff,
+                                     float *out, cudaStream_t stream);
+
+griffin_status launch_compact(const griffin_ff_desc *desc, const griffin_ff_weights *w, const int32_t *idx,
+                              const griffin_ff_compact *out, void *ws, cudaStream_t stream);
+
+// Carve-up of the workspace behind its header for the prompt-phase path.
+struct PrefillScratch {
+    size_t z_off, rowsq_off, inv_off, colpart_off, total;  // byte offsets from the scratch base
+    int n_col_tiles;                                        // partial row sums kept per token
+    int n_row_chunks;                                       // partial column sums kept per neuron
+};
+PrefillScratch prefill_scratch(const griffin_ff_desc *desc, int S);
+
+griffin_status launch_prefill_score(const griffin_ff_desc *desc, const griffin_ff_weights *w, const void *x, int S,
+                                    void *y, float *score, uint8_t *scratch, void *ws, cudaStream_t stream);
+
+}  // namespace griffin
