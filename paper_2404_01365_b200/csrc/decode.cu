@@ -1,0 +1,486 @@
+// Generation-phase pruned FF (Eqs. 4 and 5 of the GRIFFIN paper):
+//   z_hat = sigma(W_g_hat x + b_g_hat) * (W_1_hat x + b_1_hat)        kernel "gate_up"
+//   y_hat = W_2_hat z_hat + b_2                                        kernel "down"
+//
+// At batch 1..8 both products are matrix-vector products whose cost is the single pass
+// over the compact weights, so both kernels are built around keeping HBM busy:
+//   * one CTA per SM, persistent over its share of the work items;
+//   * a producer warp streams weight rows into a ring of shared-memory stages with 1-D
+//     bulk copies (TMA, no multicast) tracked by mbarriers; 8 consumer warps read the
+//     stages, keep the vector operand (x, or a tile of z) in registers and reduce with
+//     warp shuffles;
+//   * with programmatic dependent launch the producer starts streaming weights before
+//     the previous kernel on the stream has finished; everything that depends on that
+//     kernel (x, z, y) is touched only after griddepcontrol.wait.
+// Results are deterministic: every sum has a fixed order.
+#include "common.cuh"
+#include "launch.h"
+
+namespace griffin {
+
+constexpr int DEC_CONSUMER_WARPS = 8;
+constexpr int DEC_CONSUMERS = DEC_CONSUMER_WARPS * 32;
+constexpr int DEC_THREADS = DEC_CONSUMERS + 32;  // + producer warp
+constexpr int DEC_MAX_ROWS = 64;                 // rows per work item (neurons / output rows)
+constexpr int DEC_DOWN_ITER = 2;                 // 16-byte vectors per consumer thread per row segment
+constexpr int DEC_PART_FLOATS = DEC_MAX_ROWS * DEC_CONSUMER_WARPS * 2;  // one parity buffer
+
+struct DecodeSeq {
+    const void *w_gate, *w_up, *w_down, *b_gate, *b_up;
+};
+struct DecodeParams {
+    DecodeSeq seq[GRIFFIN_MAX_BATCH];
+    const void *b_down;
+    const void *x;  // [B, d]
+    void *y;        // [B, d]
+    float *z;       // [B, ldk] fp32 scratch
+    void *ws;       // workspace header (status word), may be null
+    int d, k, ldk, B;
+    int n_slices;  // work items per sequence
+    int n_stages;
+    int kt_len;    // down kernel: elements per k-tile (multiple of 8)
+    int n_ktiles;
+};
+
+struct DecSmem {
+    uint8_t *stages;
+    uint64_t *full, *empty;
+    float *part;
+    volatile int *abort;
+};
+
+__device__ __forceinline__ DecSmem carve(uint8_t *smem, int n_stages, int stage_bytes) {
+    DecSmem s;
+    s.stages = smem;
+    s.full = reinterpret_cast<uint64_t *>(smem + (size_t)n_stages * stage_bytes);
+    s.empty = s.full + n_stages;
+    s.part = reinterpret_cast<float *>(s.empty + n_stages);
+    s.abort = reinterpret_cast<volatile int *>(s.part + 2 * DEC_PART_FLOATS);
+    return s;
+}
+static size_t dec_smem_bytes(int n_stages, int stage_bytes) {
+    return (size_t)n_stages * stage_bytes + 2 * n_stages * sizeof(uint64_t) + 2 * DEC_PART_FLOATS * sizeof(float) + 16;
+}
+
+// Barrier wait that gives up after WAIT_LIMIT_NS, or as soon as another thread of the CTA
+// has given up.  On a give-up the status word is raised and false is returned.
+__device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort, void *ws,
+                                              int where) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 128; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort) return false;
+        if (global_timer_ns() - t0 > WAIT_LIMIT_NS) {
+            *abort = 1;
+            raise_status(ws, DEV_STATUS_TIMEOUT, where);
+            return false;
+        }
+    }
+}
+
+__device__ __forceinline__ void consumer_barrier() {
+    asm volatile("bar.sync 1, %0;" ::"n"(DEC_CONSUMERS) : "memory");
+}
+
+// After its last issue the producer stays until every copy it started has landed, so the
+// CTA's shared memory is never released under a copy in flight.  (Only matters after a
+// give-up: normally the consumers have already waited for every stage.)
+__device__ __forceinline__ void producer_drain(const DecSmem &s, int n_stages, uint32_t issued) {
+    const uint32_t first = issued > (uint32_t)n_stages ? issued - n_stages : 0;
+    for (uint32_t it = first; it < issued; ++it) {
+        const int stage = it % n_stages;
+        const uint32_t parity = (it / n_stages) & 1;
+        const unsigned long long t0 = global_timer_ns();
+        while (!mbar_try_wait(&s.full[stage], parity))
+            if (global_timer_ns() - t0 > WAIT_LIMIT_NS) break;
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Kernel gate_up:
+//   z[b, j] = sigma(w_gate_c[j,:] . x[b] + b_gate_c[j]) * (w_up_c[j,:] . x[b] + b_up_c[j])
+// Work item = (sequence b, slice of neurons).  Stage = gate row j followed by up row j.
+// ---------------------------------------------------------------------------------------
+template <typename T, int ITER>
+__global__ void __launch_bounds__(DEC_THREADS) decode_gate_up_kernel(const __grid_constant__ DecodeParams p, int act) {
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    constexpr int VEC = Elem<T>::VEC;
+    const int row_bytes = p.d * (int)sizeof(T);
+    const int stage_bytes = 2 * row_bytes;
+    const DecSmem s = carve(smem_raw, p.n_stages, stage_bytes);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    if (tid == 0) {
+        for (int i = 0; i < p.n_stages; ++i) {
+            mbar_init(&s.full[i], 1);
+            mbar_init(&s.empty[i], DEC_CONSUMER_WARPS);
+        }
+        *s.abort = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+    pdl_launch_dependents();
+
+    const int n_items = p.B * p.n_slices;
+    if (warp == DEC_CONSUMER_WARPS) {
+        // ---- producer: touches weights only, so it never waits for the previous grid
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+                const int b = item / p.n_slices, sl = item - b * p.n_slices;
+                const int j0 = (int)((long long)sl * p.k / p.n_slices);
+                const int j1 = (int)((long long)(sl + 1) * p.k / p.n_slices);
+                const uint8_t *g = static_cast<const uint8_t *>(p.seq[b].w_gate);
+                const uint8_t *u = static_cast<const uint8_t *>(p.seq[b].w_up);
+                for (int j = j0; j < j1; ++j, ++it) {
+                    const int stage = it % p.n_stages;
+                    const uint32_t use = it / p.n_stages;
+                    if (use > 0 && !wait_or_abort(&s.empty[stage], (use - 1) & 1, s.abort, p.ws, 1)) {
+                        ok = false;
+                        break;
+                    }
+                    uint8_t *dst = s.stages + (size_t)stage * stage_bytes;
+                    mbar_arrive_expect_tx(&s.full[stage], stage_bytes);
+                    bulk_g2s(dst, g + (size_t)j * row_bytes, row_bytes, &s.full[stage]);
+                    bulk_g2s(dst + row_bytes, u + (size_t)j * row_bytes, row_bytes, &s.full[stage]);
+                }
+            }
+            producer_drain(s, p.n_stages, it);
+        }
+        return;
+    }
+
+    // ---- consumers
+    pdl_wait_prior_grids();  // x and the z scratch belong to earlier work on the stream
+    uint32_t it = 0;
+    int item_parity = 0;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, item_parity ^= 1) {
+        const int b = item / p.n_slices, sl = item - b * p.n_slices;
+        const int j0 = (int)((long long)sl * p.k / p.n_slices);
+        const int j1 = (int)((long long)(sl + 1) * p.k / p.n_slices);
+        float2 *part = reinterpret_cast<float2 *>(s.part + item_parity * DEC_PART_FLOATS);
+
+        float xr[ITER][VEC];
+#pragma unroll
+        for (int i = 0; i < ITER; ++i) {
+            const int col = (tid + i * DEC_CONSUMERS) * VEC;
+            if (col < p.d) {
+                const uint4 v = *reinterpret_cast<const uint4 *>(static_cast<const T *>(p.x) + (size_t)b * p.d + col);
+                Elem<T>::unpack(v, xr[i]);
+            } else {
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) xr[i][e] = 0.f;
+            }
+        }
+
+        bool ok = true;
+        for (int j = j0; j < j1; ++j, ++it) {
+            const int stage = it % p.n_stages;
+            if (!wait_or_abort(&s.full[stage], (it / p.n_stages) & 1, s.abort, p.ws, 2)) {
+                ok = false;
+                break;
+            }
+            const uint8_t *src = s.stages + (size_t)stage * stage_bytes;
+            float ga = 0.f, ua = 0.f;
+#pragma unroll
+            for (int i = 0; i < ITER; ++i) {
+                const int col = (tid + i * DEC_CONSUMERS) * VEC;
+                if (col < p.d) {
+                    float gf[VEC], uf[VEC];
+                    Elem<T>::unpack(*reinterpret_cast<const uint4 *>(src + (size_t)col * sizeof(T)), gf);
+                    Elem<T>::unpack(*reinterpret_cast<const uint4 *>(src + row_bytes + (size_t)col * sizeof(T)), uf);
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) {
+                        ga = fmaf(gf[e], xr[i][e], ga);
+                        ua = fmaf(uf[e], xr[i][e], ua);
+                    }
+                }
+            }
+            ga = warp_sum(ga);
+            ua = warp_sum(ua);
+            if (lane == 0) {
+                // every lane's shared-memory reads fed the shuffles above, so they are done
+                mbar_arrive(&s.empty[stage]);
+                part[(j - j0) * DEC_CONSUMER_WARPS + warp] = make_float2(ga, ua);
+            }
+        }
+        consumer_barrier();
+        if (!ok || *s.abort) break;
+        if (tid < j1 - j0) {
+            float ga = 0.f, ua = 0.f;
+#pragma unroll
+            for (int w = 0; w < DEC_CONSUMER_WARPS; ++w) {
+                const float2 v = part[tid * DEC_CONSUMER_WARPS + w];
+                ga += v.x;
+                ua += v.y;
+            }
+            const int j = j0 + tid;
+            if (p.seq[b].b_gate) ga += Elem<T>::to_float(static_cast<const T *>(p.seq[b].b_gate)[j]);
+            if (p.seq[b].b_up) ua += Elem<T>::to_float(static_cast<const T *>(p.seq[b].b_up)[j]);
+            p.z[(size_t)b * p.ldk + j] = sigma_rt(act, ga) * ua;
+        }
+        // the last slice also clears the padding of z (at most 7 entries)
+        const int pad = tid - (DEC_CONSUMERS - 8);
+        if (sl == p.n_slices - 1 && pad >= 0 && p.k + pad < p.ldk) p.z[(size_t)b * p.ldk + p.k + pad] = 0.f;
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Kernel down:  y[b, c] = w_down_c[c, 0:k] . z[b, 0:k] + b_down[c]
+// Work item = (sequence b, chunk of output rows).  Rows are cut into k-tiles so that the
+// matching tile of z sits in registers; stage = the same k-tile of two consecutive rows.
+// ---------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(DEC_THREADS) decode_down_kernel(const __grid_constant__ DecodeParams p) {
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    constexpr int VEC = Elem<T>::VEC;
+    constexpr int ITER = DEC_DOWN_ITER;
+    const int seg_bytes_max = p.kt_len * (int)sizeof(T);
+    const int stage_bytes = 2 * seg_bytes_max;
+    const DecSmem s = carve(smem_raw, p.n_stages, stage_bytes);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    if (tid == 0) {
+        for (int i = 0; i < p.n_stages; ++i) {
+            mbar_init(&s.full[i], 1);
+            mbar_init(&s.empty[i], DEC_CONSUMER_WARPS);
+        }
+        *s.abort = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+    pdl_launch_dependents();
+
+    const int n_items = p.B * p.n_slices;
+    if (warp == DEC_CONSUMER_WARPS) {
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+                const int b = item / p.n_slices, sl = item - b * p.n_slices;
+                const int c0 = (int)((long long)sl * p.d / p.n_slices);
+                const int c1 = (int)((long long)(sl + 1) * p.d / p.n_slices);
+                const uint8_t *w = static_cast<const uint8_t *>(p.seq[b].w_down);
+                for (int kt = 0; ok && kt < p.n_ktiles; ++kt) {
+                    const int e0 = kt * p.kt_len;
+                    const int len = min(p.kt_len, p.ldk - e0);
+                    const uint32_t seg_bytes = (uint32_t)len * sizeof(T);
+                    for (int c = c0; c < c1; c += 2, ++it) {
+                        const int stage = it % p.n_stages;
+                        const uint32_t use = it / p.n_stages;
+                        if (use > 0 && !wait_or_abort(&s.empty[stage], (use - 1) & 1, s.abort, p.ws, 3)) {
+                            ok = false;
+                            break;
+                        }
+                        uint8_t *dst = s.stages + (size_t)stage * stage_bytes;
+                        const bool two = c + 1 < c1;
+                        mbar_arrive_expect_tx(&s.full[stage], two ? 2 * seg_bytes : seg_bytes);
+                        bulk_g2s(dst, w + ((size_t)c * p.ldk + e0) * sizeof(T), seg_bytes, &s.full[stage]);
+                        if (two)
+                            bulk_g2s(dst + seg_bytes_max, w + ((size_t)(c + 1) * p.ldk + e0) * sizeof(T), seg_bytes,
+                                     &s.full[stage]);
+                    }
+                }
+            }
+            producer_drain(s, p.n_stages, it);
+        }
+        return;
+    }
+
+    pdl_wait_prior_grids();  // z comes from the gate_up kernel
+    uint32_t it = 0;
+    int item_parity = 0;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, item_parity ^= 1) {
+        const int b = item / p.n_slices, sl = item - b * p.n_slices;
+        const int c0 = (int)((long long)sl * p.d / p.n_slices);
+        const int c1 = (int)((long long)(sl + 1) * p.d / p.n_slices);
+        float *part = s.part + item_parity * DEC_PART_FLOATS;
+        bool ok = true;
+        for (int kt = 0; ok && kt < p.n_ktiles; ++kt) {
+            const int e0 = kt * p.kt_len;
+            const int len = min(p.kt_len, p.ldk - e0);
+            float zr[ITER][VEC];
+#pragma unroll
+            for (int i = 0; i < ITER; ++i) {
+                const int col = (tid + i * DEC_CONSUMERS) * VEC;
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) zr[i][e] = 0.f;
+                if (col < len) {
+                    const float4 *zp = reinterpret_cast<const float4 *>(p.z + (size_t)b * p.ldk + e0 + col);
+#pragma unroll
+                    for (int q = 0; q < VEC / 4; ++q) {
+                        const float4 v = zp[q];
+                        zr[i][4 * q + 0] = v.x; zr[i][4 * q + 1] = v.y;
+                        zr[i][4 * q + 2] = v.z; zr[i][4 * q + 3] = v.w;
+                    }
+                }
+            }
+            for (int c = c0; c < c1; c += 2, ++it) {
+                const int stage = it % p.n_stages;
+                if (!wait_or_abort(&s.full[stage], (it / p.n_stages) & 1, s.abort, p.ws, 4)) {
+                    ok = false;
+                    break;
+                }
+                const uint8_t *src = s.stages + (size_t)stage * stage_bytes;
+                const bool two = c + 1 < c1;
+                float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+                for (int i = 0; i < ITER; ++i) {
+                    const int col = (tid + i * DEC_CONSUMERS) * VEC;
+                    if (col < len) {
+                        float w0[VEC];
+                        Elem<T>::unpack(*reinterpret_cast<const uint4 *>(src + (size_t)col * sizeof(T)), w0);
+#pragma unroll
+                        for (int e = 0; e < VEC; ++e) a0 = fmaf(w0[e], zr[i][e], a0);
+                        if (two) {
+                            float w1[VEC];
+                            Elem<T>::unpack(
+                                *reinterpret_cast<const uint4 *>(src + seg_bytes_max + (size_t)col * sizeof(T)), w1);
+#pragma unroll
+                            for (int e = 0; e < VEC; ++e) a1 = fmaf(w1[e], zr[i][e], a1);
+                        }
+                    }
+                }
+                a0 = warp_sum(a0);
+                a1 = warp_sum(a1);
+                if (lane == 0) {
+                    mbar_arrive(&s.empty[stage]);
+                    float *q = part + (c - c0) * DEC_CONSUMER_WARPS + warp;  // rows c and c+1
+                    if (kt == 0) {
+                        q[0] = a0;
+                        q[DEC_CONSUMER_WARPS] = a1;
+                    } else {
+                        q[0] += a0;
+                        q[DEC_CONSUMER_WARPS] += a1;
+                    }
+                }
+            }
+        }
+        consumer_barrier();
+        if (!ok || *s.abort) break;
+        if (tid < c1 - c0) {
+            float acc = 0.f;
+#pragma unroll
+            for (int w = 0; w < DEC_CONSUMER_WARPS; ++w) acc += part[tid * DEC_CONSUMER_WARPS + w];
+            const int c = c0 + tid;
+            if (p.b_down) acc += Elem<T>::to_float(static_cast<const T *>(p.b_down)[c]);
+            static_cast<T *>(p.y)[(size_t)b * p.d + c] = Elem<T>::from_float(acc);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------------------
+static cudaError_t launch_maybe_overlapped(const void *func, dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                           bool overlap, void **args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = overlap ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelExC(&cfg, func, args);
+}
+
+static int pick_stages(int stage_bytes) {
+    // about 96 KB of stages: deep enough to cover HBM latency, small enough that the next
+    // kernel's CTA fits beside this one on the SM and can prefetch its own weights
+    int n = (96 * 1024) / stage_bytes;
+    if (n < 2) n = 2;
+    if (n > 12) n = 12;
+    return n;
+}
+
+static int slices_for(int rows, int grid) {
+    // a multiple of the grid, fine enough that one item has at most DEC_MAX_ROWS rows
+    int per = (rows + grid * DEC_MAX_ROWS - 1) / (grid * DEC_MAX_ROWS);
+    if (per < 1) per = 1;
+    return grid * per;
+}
+
+template <typename T>
+static griffin_status decode_typed(const griffin_ff_desc *desc, int B, const griffin_ff_compact *sets,
+                                   const void *b_down, const void *x, void *y, float *z, void *ws, uint32_t flags,
+                                   cudaStream_t stream) {
+    constexpr int VEC = Elem<T>::VEC;
+    DecodeParams p = {};
+    for (int b = 0; b < B; ++b) {
+        p.seq[b].w_gate = sets[b].w_gate_c;
+        p.seq[b].w_up = sets[b].w_up_c;
+        p.seq[b].w_down = sets[b].w_down_c;
+        p.seq[b].b_gate = sets[b].b_gate_c;
+        p.seq[b].b_up = sets[b].b_up_c;
+    }
+    p.b_down = b_down;
+    p.x = x;
+    p.y = y;
+    p.z = z;
+    p.ws = ws;
+    p.d = desc->d;
+    p.k = sets[0].k;
+    p.ldk = sets[0].ldk;
+    p.B = B;
+
+    const int sms = device_sm_count();
+    if (sms <= 0) return GRIFFIN_ERR_CUDA;
+    const bool overlap = (flags & GRIFFIN_DECODE_OVERLAP_WEIGHT_PREFETCH) != 0;
+
+    {  // gate_up
+        const int stage_bytes = 2 * p.d * (int)sizeof(T);
+        p.n_stages = pick_stages(stage_bytes);
+        p.n_slices = slices_for(p.k, sms);
+        const int grid = min(sms, B * p.n_slices);
+        const size_t smem = dec_smem_bytes(p.n_stages, stage_bytes);
+        const int iter = (p.d + DEC_CONSUMERS * VEC - 1) / (DEC_CONSUMERS * VEC);
+        const void *fn = nullptr;
+        switch (iter) {
+            case 1: fn = (const void *)decode_gate_up_kernel<T, 1>; break;
+            case 2: fn = (const void *)decode_gate_up_kernel<T, 2>; break;
+            case 3: fn = (const void *)decode_gate_up_kernel<T, 3>; break;
+            case 4: fn = (const void *)decode_gate_up_kernel<T, 4>; break;
+            case 5: case 6: fn = (const void *)decode_gate_up_kernel<T, 6>; break;
+            case 7: case 8: fn = (const void *)decode_gate_up_kernel<T, 8>; break;
+            default: return GRIFFIN_ERR_UNSUPPORTED;
+        }
+        if (ensure_dynamic_smem(fn, smem) != cudaSuccess) return GRIFFIN_ERR_CUDA;
+        int act = desc->act;
+        void *args[] = {&p, &act};
+        if (launch_maybe_overlapped(fn, dim3(grid), dim3(DEC_THREADS), smem, stream, overlap, args) != cudaSuccess)
+            return GRIFFIN_ERR_CUDA;
+    }
+    {  // down: may always start early, since gate_up never writes weights
+        const int kt_max = DEC_CONSUMERS * VEC * DEC_DOWN_ITER;
+        p.n_ktiles = (p.ldk + kt_max - 1) / kt_max;
+        const int kt_len = (p.ldk + p.n_ktiles - 1) / p.n_ktiles;
+        p.kt_len = (kt_len + 7) / 8 * 8;
+        const int stage_bytes = 2 * p.kt_len * (int)sizeof(T);
+        p.n_stages = pick_stages(stage_bytes);
+        p.n_slices = slices_for(p.d, sms);
+        const int grid = min(sms, B * p.n_slices);
+        const size_t smem = dec_smem_bytes(p.n_stages, stage_bytes);
+        const void *fn = (const void *)decode_down_kernel<T>;
+        if (ensure_dynamic_smem(fn, smem) != cudaSuccess) return GRIFFIN_ERR_CUDA;
+        void *args[] = {&p};
+        if (launch_maybe_overlapped(fn, dim3(grid), dim3(DEC_THREADS), smem, stream, true, args) != cudaSuccess)
+            return GRIFFIN_ERR_CUDA;
+    }
+    return GRIFFIN_OK;
+}
+
+griffin_status launch_decode(const griffin_ff_desc *desc, int B, const griffin_ff_compact *sets, const void *b_down,
+                             const void *x, void *y, float *z, void *ws, uint32_t flags, cudaStream_t stream) {
+    if (desc->dtype == GRIFFIN_DT_F32)
+        return decode_typed<float>(desc, B, sets, b_down, x, y, z, ws, flags, stream);
+    return decode_typed<__nv_bfloat16>(desc, B, sets, b_down, x, y, z, ws, flags, stream);
+}
+
+}  // namespace griffin
