@@ -1,0 +1,150 @@
+// Expert compaction (Section 4.2 of the GRIFFIN paper): W_g_hat = W_g[E, :],
+// W_1_hat = W_1[E, :], W_2_hat = W_2[:, E], plus the matching bias entries.  Bit copies, so
+// elements are moved as raw 16- or 32-bit words.
+//
+//   rows kernel     16-byte vector copy of the selected rows of W_g and W_1; consecutive
+//                   threads move consecutive vectors of one row (coalesced both ways).
+//   columns kernel  W_2 is [d, d_ff] row-major, so selecting columns is a gather inside
+//                   each row.  One CTA takes four rows; a thread reads 16 bytes' worth of
+//                   output columns of E once, picks those elements from each of the four
+//                   rows (E is ascending and dense, so neighbouring threads hit
+//                   neighbouring sectors) and writes one 16-byte vector per row.  Padding
+//                   columns k..ldk are written as zeros.
+#include "common.cuh"
+#include "launch.h"
+
+namespace griffin {
+
+constexpr int CP_THREADS = 256;
+constexpr int CP_ROWS_PER_CTA = 4;
+
+__device__ __forceinline__ uint4 ld_stream(const uint4 *p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void st_stream(uint4 *p, const uint4 &v) {
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+
+// dst_g[jj, :] = src_g[idx[jj], :], dst_u likewise; nv = 16-byte vectors per row.
+__global__ void __launch_bounds__(CP_THREADS) compact_rows_kernel(const uint4 *__restrict__ src_g,
+                                                                  const uint4 *__restrict__ src_u,
+                                                                  uint4 *__restrict__ dst_g, uint4 *__restrict__ dst_u,
+                                                                  const int32_t *__restrict__ idx, int k, int d_ff,
+                                                                  int nv, void *ws) {
+    const long long total = 2ll * k * nv;
+    const long long stride = (long long)gridDim.x * CP_THREADS;
+    constexpr int U = 4;
+    for (long long v0 = (long long)blockIdx.x * CP_THREADS + threadIdx.x; v0 < total; v0 += stride * U) {
+        uint4 val[U];
+        uint4 *dst[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const long long v = v0 + u * stride;
+            dst[u] = nullptr;
+            val[u] = make_uint4(0, 0, 0, 0);
+            if (v < total) {
+                const int row = (int)(v / nv);
+                const int col = (int)(v - (long long)row * nv);
+                const int m = row >= k;
+                const int jj = m ? row - k : row;
+                const int e = idx[jj];
+                dst[u] = (m ? dst_u : dst_g) + (size_t)jj * nv + col;
+                if (e >= 0 && e < d_ff)
+                    val[u] = ld_stream((m ? src_u : src_g) + (size_t)e * nv + col);
+                else
+                    raise_status(ws, DEV_STATUS_BAD_INDEX, 10);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (dst[u]) st_stream(dst[u], val[u]);
+    }
+}
+
+template <typename U>
+__global__ void compact_bias_kernel(const U *__restrict__ src_g, const U *__restrict__ src_u, U *__restrict__ dst_g,
+                                    U *__restrict__ dst_u, const int32_t *__restrict__ idx, int k, int d_ff) {
+    const int jj = blockIdx.x * blockDim.x + threadIdx.x;
+    if (jj >= k) return;
+    const int e = idx[jj];
+    const bool ok = e >= 0 && e < d_ff;
+    if (src_g && dst_g) dst_g[jj] = ok ? src_g[e] : (U)0;
+    if (src_u && dst_u) dst_u[jj] = ok ? src_u[e] : (U)0;
+}
+
+// dst[c, jj] = src[c, idx[jj]] for jj < k, 0 for k <= jj < ldk.
+template <typename U>
+__global__ void __launch_bounds__(CP_THREADS) compact_cols_kernel(const U *__restrict__ src, U *__restrict__ dst,
+                                                                  const int32_t *__restrict__ idx, int d, int d_ff,
+                                                                  int k, int ldk, void *ws) {
+    constexpr int VEC = 16 / (int)sizeof(U);
+    const int c0 = blockIdx.x * CP_ROWS_PER_CTA;
+    const int nvec = ldk / VEC;
+    for (int v = threadIdx.x; v < nvec; v += CP_THREADS) {
+        int e[VEC];
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) {
+            const int jj = v * VEC + i;
+            e[i] = jj < k ? idx[jj] : -1;
+            if (jj < k && (e[i] < 0 || e[i] >= d_ff)) {
+                e[i] = -1;
+                raise_status(ws, DEV_STATUS_BAD_INDEX, 11);
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < CP_ROWS_PER_CTA; ++r) {
+            const int c = c0 + r;
+            if (c < d) {
+                const U *row = src + (size_t)c * d_ff;
+                union {
+                    uint4 u;
+                    U t[VEC];
+                } pack;
+                pack.u = make_uint4(0, 0, 0, 0);
+#pragma unroll
+                for (int i = 0; i < VEC; ++i)
+                    if (e[i] >= 0) pack.t[i] = row[e[i]];
+                st_stream(reinterpret_cast<uint4 *>(dst + (size_t)c * ldk) + v, pack.u);
+            }
+        }
+    }
+}
+
+template <typename U>
+static griffin_status compact_typed(const griffin_ff_desc *desc, const griffin_ff_weights *w, const int32_t *idx,
+                                    const griffin_ff_compact *out, void *ws, cudaStream_t stream) {
+    const int d = desc->d, d_ff = desc->d_ff, k = out->k, ldk = out->ldk;
+    const int nv = d * (int)sizeof(U) / 16;
+    const int sms = device_sm_count();
+    if (sms <= 0) return GRIFFIN_ERR_CUDA;
+    const long long want = (2ll * k * nv + CP_THREADS * 4 - 1) / (CP_THREADS * 4);
+    int grid = (int)(want < (long long)sms * 8 ? want : (long long)sms * 8);
+    if (grid < 1) grid = 1;
+    compact_rows_kernel<<<grid, CP_THREADS, 0, stream>>>(
+        static_cast<const uint4 *>(w->w_gate), static_cast<const uint4 *>(w->w_up),
+        static_cast<uint4 *>(out->w_gate_c), static_cast<uint4 *>(out->w_up_c), idx, k, d_ff, nv, ws);
+    if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
+    compact_cols_kernel<U><<<(d + CP_ROWS_PER_CTA - 1) / CP_ROWS_PER_CTA, CP_THREADS, 0, stream>>>(
+        static_cast<const U *>(w->w_down), static_cast<U *>(out->w_down_c), idx, d, d_ff, k, ldk, ws);
+    if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
+    if ((w->b_gate && out->b_gate_c) || (w->b_up && out->b_up_c)) {
+        compact_bias_kernel<U><<<(k + 255) / 256, 256, 0, stream>>>(
+            static_cast<const U *>(w->b_gate), static_cast<const U *>(w->b_up), static_cast<U *>(out->b_gate_c),
+            static_cast<U *>(out->b_up_c), idx, k, d_ff);
+        if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
+    }
+    return GRIFFIN_OK;
+}
+
+griffin_status launch_compact(const griffin_ff_desc *desc, const griffin_ff_weights *w, const int32_t *idx,
+                              const griffin_ff_compact *out, void *ws, cudaStream_t stream) {
+    if (desc->dtype == GRIFFIN_DT_F32) return compact_typed<uint32_t>(desc, w, idx, out, ws, stream);
+    return compact_typed<uint16_t>(desc, w, idx, out, ws, stream);
+}
+
+}  // namespace griffin
