@@ -1,0 +1,269 @@
+// Prompt-phase FF and selection statistic (Section 4.2, Eqs. 1, 3 and 6 of the GRIFFIN paper).
+//
+//   1. Z = sigma(X W_g^T + b_g) * (X W_1^T + b_1)          [S, d_ff]  (Eq. 3), stored in the
+//      storage dtype; the same kernel leaves, per token and per column tile, the partial
+//      sum of squares of the stored row                                 (for ||Z_i||^2)
+//   2. Y = Z W_2^T + b_2                                    [S, d]     (Eq. 1)
+//   3. inv_i = 1 / ||Z_i||_2^2  (0 for an all-zero row)
+//   4. colpart[chunk, j] = sum over the chunk's tokens of Z_ij^2 * inv_i
+//   5. s_j = sqrt(sum over chunks of colpart[chunk, j])                 (Eq. 6)
+//
+// The row normaliser spans every column tile, so the column sums cannot finish inside
+// step 1: steps 3-5 re-read Z (which mostly still sits in L2).  All partial sums are kept
+// and added in a fixed order, so s is deterministic.
+//
+// This file holds the fp32-FMA (SIMT) matrix kernels, which serve the fp32 storage type
+// and any shape the tensor-core path does not take, plus steps 3-5 and the dispatcher.
+#include <type_traits>
+
+#include "common.cuh"
+#include "launch.h"
+#include "prefill_tc.h"
+
+namespace griffin {
+
+constexpr int PF_BM = 64, PF_BN = 64, PF_BK = 16, PF_THREADS = 256, PF_PAD = 4;
+constexpr int PF_ROW_CHUNK = 64;  // tokens per partial column sum
+
+static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+PrefillScratch prefill_scratch(const griffin_ff_desc *desc, int S) {
+    PrefillScratch ps;
+    const size_t esz = desc->dtype == GRIFFIN_DT_F32 ? 4 : 2;
+    ps.n_col_tiles = (desc->d_ff + PF_BN - 1) / PF_BN;  // the narrowest column tile any path uses
+    ps.n_row_chunks = (S + PF_ROW_CHUNK - 1) / PF_ROW_CHUNK;
+    size_t off = 0;
+    ps.z_off = off;
+    off = align_up(off + (size_t)S * desc->d_ff * esz, 256);
+    ps.rowsq_off = off;
+    off = align_up(off + (size_t)S * ps.n_col_tiles * sizeof(float), 256);
+    ps.inv_off = off;
+    off = align_up(off + (size_t)S * sizeof(float), 256);
+    ps.colpart_off = off;
+    off = align_up(off + (size_t)ps.n_row_chunks * desc->d_ff * sizeof(float), 256);
+    ps.total = off;
+    return ps;
+}
+
+// Loads a [64 x 16] tile of a row-major [rows, K] matrix (K contiguous) into shared memory
+// as fp32, transposed to [k][row].  256 threads; rows/K beyond the matrix read as zero.
+template <typename T>
+__device__ __forceinline__ void load_tile_t(const T *__restrict__ src, int ld, int rows, int K, int r0, int k0,
+                                            float (*dst)[PF_BM + PF_PAD], int tid) {
+    constexpr int VEC = Elem<T>::VEC;
+    constexpr int VPR = PF_BK / VEC;  // vectors per tile row
+    if (tid < PF_BM * VPR) {
+        const int r = tid / VPR, kv = tid - r * VPR;
+        const int row = r0 + r, kk = k0 + kv * VEC;
+        float f[VEC];
+        if (row < rows && kk < K) {
+            Elem<T>::unpack(*reinterpret_cast<const uint4 *>(src + (size_t)row * ld + kk), f);
+        } else {
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) f[e] = 0.f;
+        }
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) dst[kv * VEC + e][r] = f[e];
+    }
+}
+
+// Step 1 (SIMT): one CTA = 64 tokens x 64 neurons.
+template <typename T>
+__global__ void __launch_bounds__(PF_THREADS) ff1_simt_kernel(const T *__restrict__ x, const T *__restrict__ w_gate,
+                                                              const T *__restrict__ w_up, const T *__restrict__ b_gate,
+                                                              const T *__restrict__ b_up, T *__restrict__ z,
+                                                              float *__restrict__ rowsq, int S, int d, int d_ff,
+                                                              int n_col_tiles, int act) {
+    __shared__ float xs[PF_BK][PF_BM + PF_PAD], gs[PF_BK][PF_BN + PF_PAD], us[PF_BK][PF_BN + PF_PAD];
+    __shared__ float red[PF_BM][17];
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    const int m0 = blockIdx.y * PF_BM, n0 = blockIdx.x * PF_BN;
+    float ga[4][4] = {}, ua[4][4] = {};
+    for (int k0 = 0; k0 < d; k0 += PF_BK) {
+        load_tile_t<T>(x, d, S, d, m0, k0, xs, tid);
+        load_tile_t<T>(w_gate, d, d_ff, d, n0, k0, gs, tid);
+        load_tile_t<T>(w_up, d, d_ff, d, n0, k0, us, tid);
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < PF_BK; ++kk) {
+            const float4 a = *reinterpret_cast<const float4 *>(&xs[kk][ty * 4]);
+            const float4 g = *reinterpret_cast<const float4 *>(&gs[kk][tx * 4]);
+            const float4 u = *reinterpret_cast<const float4 *>(&us[kk][tx * 4]);
+            const float av[4] = {a.x, a.y, a.z, a.w}, gv[4] = {g.x, g.y, g.z, g.w}, uv[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    ga[i][j] = fmaf(av[i], gv[j], ga[i][j]);
+                    ua[i][j] = fmaf(av[i], uv[j], ua[i][j]);
+                }
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int row = m0 + ty * 4 + i;
+        float sq = 0.f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int col = n0 + tx * 4 + j;
+            if (row < S && col < d_ff) {
+                float g = ga[i][j], u = ua[i][j];
+                if (b_gate) g += Elem<T>::to_float(b_gate[col]);
+                if (b_up) u += Elem<T>::to_float(b_up[col]);
+                const T zt = Elem<T>::from_float(sigma_rt(act, g) * u);
+                z[(size_t)row * d_ff + col] = zt;
+                const float zf = Elem<T>::to_float(zt);  // the norm is that of the stored row
+                sq = fmaf(zf, zf, sq);
+            }
+        }
+        red[ty * 4 + i][tx] = sq;
+    }
+    __syncthreads();
+    if (tid < PF_BM && m0 + tid < S) {
+        float sq = 0.f;
+#pragma unroll
+        for (int t = 0; t < 16; ++t) sq += red[tid][t];
+        rowsq[(size_t)(m0 + tid) * n_col_tiles + blockIdx.x] = sq;
+    }
+}
+
+// Step 2 (SIMT): Y = Z W_2^T + b_2, one CTA = 64 tokens x 64 outputs.
+template <typename T>
+__global__ void __launch_bounds__(PF_THREADS) ff2_simt_kernel(const T *__restrict__ z, const T *__restrict__ w_down,
+                                                              const T *__restrict__ b_down, T *__restrict__ y, int S,
+                                                              int d, int d_ff) {
+    __shared__ float zs[PF_BK][PF_BM + PF_PAD], ws[PF_BK][PF_BN + PF_PAD];
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    const int m0 = blockIdx.y * PF_BM, n0 = blockIdx.x * PF_BN;
+    float acc[4][4] = {};
+    for (int k0 = 0; k0 < d_ff; k0 += PF_BK) {
+        load_tile_t<T>(z, d_ff, S, d_ff, m0, k0, zs, tid);
+        load_tile_t<T>(w_down, d_ff, d, d_ff, n0, k0, ws, tid);
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < PF_BK; ++kk) {
+            const float4 a = *reinterpret_cast<const float4 *>(&zs[kk][ty * 4]);
+            const float4 b = *reinterpret_cast<const float4 *>(&ws[kk][tx * 4]);
+            const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int row = m0 + ty * 4 + i;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int col = n0 + tx * 4 + j;
+            if (row < S && col < d) {
+                float v = acc[i][j];
+                if (b_down) v += Elem<T>::to_float(b_down[col]);
+                y[(size_t)row * d + col] = Elem<T>::from_float(v);
+            }
+        }
+    }
+}
+
+// Step 3: one warp per token.
+__global__ void row_inv_kernel(const float *__restrict__ rowsq, int S, int n_col_tiles, float *__restrict__ inv) {
+    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (row >= S) return;
+    float sq = 0.f;
+    for (int t = lane; t < n_col_tiles; t += 32) sq += rowsq[(size_t)row * n_col_tiles + t];
+    sq = warp_sum(sq);
+    if (lane == 0) inv[row] = sq > 0.f ? 1.0f / sq : 0.f;
+}
+
+// Step 4: a thread owns 16 bytes' worth of neighbouring columns over one chunk of tokens.
+template <typename T>
+__global__ void __launch_bounds__(128) col_partial_kernel(const T *__restrict__ z, const float *__restrict__ inv, int S,
+                                                          int d_ff, float *__restrict__ colpart) {
+    constexpr int VEC = Elem<T>::VEC;
+    const int col = (blockIdx.x * 128 + threadIdx.x) * VEC;
+    if (col >= d_ff) return;
+    const int r0 = blockIdx.y * PF_ROW_CHUNK, r1 = min(S, r0 + PF_ROW_CHUNK);
+    float acc[VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
+#pragma unroll 4
+    for (int r = r0; r < r1; ++r) {
+        float f[VEC];
+        Elem<T>::unpack(*reinterpret_cast<const uint4 *>(z + (size_t)r * d_ff + col), f);
+        const float w = __ldg(inv + r);
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) acc[e] = fmaf(f[e] * f[e], w, acc[e]);
+    }
+    float *dst = colpart + (size_t)blockIdx.y * d_ff + col;
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) dst[e] = acc[e];
+}
+
+// Step 5.
+__global__ void score_finish_kernel(const float *__restrict__ colpart, int n_row_chunks, int d_ff,
+                                    float *__restrict__ score) {
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= d_ff) return;
+    float acc = 0.f;
+    for (int c = 0; c < n_row_chunks; ++c) acc += colpart[(size_t)c * d_ff + j];
+    score[j] = sqrtf(acc);
+}
+
+template <typename T>
+static griffin_status prefill_typed(const griffin_ff_desc *desc, const griffin_ff_weights *w, const void *x, int S,
+                                    void *y, float *score, uint8_t *scratch, void *ws, cudaStream_t stream) {
+    const int d = desc->d, d_ff = desc->d_ff;
+    const PrefillScratch ps = prefill_scratch(desc, S);
+    T *z = reinterpret_cast<T *>(scratch + ps.z_off);
+    float *rowsq = reinterpret_cast<float *>(scratch + ps.rowsq_off);
+    float *inv = reinterpret_cast<float *>(scratch + ps.inv_off);
+    float *colpart = reinterpret_cast<float *>(scratch + ps.colpart_off);
+
+    int n_col_tiles = 0;
+    bool ff2_done = false;
+    bool use_tc = false;
+    if constexpr (std::is_same<T, __nv_bfloat16>::value) use_tc = prefill_tc_supported(desc, S);
+    if (use_tc) {
+        if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+            griffin_status st = launch_prefill_tc(desc, w, x, S, y, z, rowsq, &n_col_tiles, ws, stream);
+            if (st != GRIFFIN_OK) return st;
+        }
+        ff2_done = true;
+    } else {
+        n_col_tiles = (d_ff + PF_BN - 1) / PF_BN;
+        const dim3 g1(n_col_tiles, (S + PF_BM - 1) / PF_BM);
+        ff1_simt_kernel<T><<<g1, PF_THREADS, 0, stream>>>(
+            static_cast<const T *>(x), static_cast<const T *>(w->w_gate), static_cast<const T *>(w->w_up),
+            static_cast<const T *>(w->b_gate), static_cast<const T *>(w->b_up), z, rowsq, S, d, d_ff, n_col_tiles,
+            desc->act);
+        if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
+    }
+    if (!ff2_done && y != nullptr) {
+        const dim3 g2((d + PF_BN - 1) / PF_BN, (S + PF_BM - 1) / PF_BM);
+        ff2_simt_kernel<T><<<g2, PF_THREADS, 0, stream>>>(z, static_cast<const T *>(w->w_down),
+                                                          static_cast<const T *>(w->b_down), static_cast<T *>(y), S, d,
+                                                          d_ff);
+        if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
+    }
+    row_inv_kernel<<<(S + 7) / 8, 256, 0, stream>>>(rowsq, S, n_col_tiles, inv);
+    if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
+    constexpr int VEC = Elem<T>::VEC;
+    const dim3 g4((d_ff + 128 * VEC - 1) / (128 * VEC), ps.n_row_chunks);
+    col_partial_kernel<T><<<g4, 128, 0, stream>>>(z, inv, S, d_ff, colpart);
+    if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
+    score_finish_kernel<<<(d_ff + 255) / 256, 256, 0, stream>>>(colpart, ps.n_row_chunks, d_ff, score);
+    if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
+    return GRIFFIN_OK;
+}
+
+griffin_status launch_prefill_score(const griffin_ff_desc *desc, const griffin_ff_weights *w, const void *x, int S,
+                                    void *y, float *score, uint8_t *scratch, void *ws, cudaStream_t stream) {
+    if (desc->dtype == GRIFFIN_DT_F32)
+        return prefill_typed<float>(desc, w, x, S, y, score, scratch, ws, stream);
+    return prefill_typed<__nv_bfloat16>(desc, w, x, S, y, score, scratch, ws, stream);
+}
+
+}  // namespace griffin
