@@ -1,0 +1,206 @@
+"""Per-kernel parity of the CUDA path (through the C ABI) against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import griffin_oracle as O
+from paper_2404_01365_b200 import binding as G
+from gpu_util import (GpuLayer, TOL_OUT, TOL_SCORE, check_expert_set, dev, np64, rand, rel_l2)
+
+pytestmark = pytest.mark.gpu
+
+TD = {"f32": torch.float32, "bf16": torch.bfloat16}
+
+
+def make_layer(d, d_ff, dtype, act="swiglu", bias=False, seed=0, S_max=0, n_seq=1):
+    td = TD[dtype]
+    wg, wu = rand((d_ff, d), td, seed + 1, d ** -0.5), rand((d_ff, d), td, seed + 2, d ** -0.5)
+    wd = rand((d, d_ff), td, seed + 3, d_ff ** -0.5)
+    bg = rand((d_ff,), td, seed + 4, 0.3) if bias else None
+    bu = rand((d_ff,), td, seed + 5, 0.3) if bias else None
+    bd = rand((d,), td, seed + 6, 0.3) if bias else None
+    host = dict(wg=wg, wu=wu, wd=wd, bg=bg, bu=bu, bd=bd)
+    return GpuLayer(d, d_ff, act, dtype, wg, wu, wd, bg, bu, bd, S_max=S_max, n_seq=n_seq), host
+
+
+def h64(host, name):
+    return None if host[name] is None else np64(host[name])
+
+
+# ------------------------------------------------------------------ top-k ---
+
+@pytest.mark.parametrize("d_ff,k", [(8, 1), (8, 8), (688, 344), (1000, 999), (11008, 5504), (24576, 12288),
+                                    (24576, 1), (4099, 2000)])
+def test_topk_exact(d_ff, k):
+    g = torch.Generator().manual_seed(d_ff + k)
+    s = torch.rand((3, d_ff), generator=g)
+    s[1] = torch.round(s[1] * 8) / 8          # many exact ties
+    s[2] = 0.5                                 # all equal -> lowest indices
+    s[2, -1] = 0.0
+    e = torch.empty((3, k), device=dev(), dtype=torch.int32)
+    G.griffin_select_topk(s.to(dev()), k, e)
+    e = e.cpu().numpy()
+    for i in range(3):
+        assert np.array_equal(e[i], O.select_topk(s[i].double().numpy(), k)), i
+
+
+def test_topk_negative_and_zero_scores():
+    s = torch.tensor([[-1.0, 0.0, -0.0, 2.0, -3.0, 0.0, 1e-30, -1e-30]])
+    for k in range(1, 9):
+        e = torch.empty((1, k), device=dev(), dtype=torch.int32)
+        G.griffin_select_topk(s.to(dev()), k, e)
+        assert np.array_equal(e.cpu().numpy()[0], O.select_topk(s[0].double().numpy(), k)), k
+
+
+def test_combine_scores():
+    g = torch.Generator().manual_seed(5)
+    s = torch.rand((5, 1000), generator=g)
+    lens = [3, 64, 512, 7, 1]
+    out = torch.empty((1000,), device=dev())
+    G.griffin_combine_scores(s.to(dev()), lens, out)
+    ref = O.combine_scores([r for r in s.double().numpy()], lens)
+    assert np.max(np.abs(np64(out) - ref) / ref) < 1e-6
+
+
+# ------------------------------------------------------------- compaction ---
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("d,d_ff,k", [(64, 96, 37), (256, 688, 344), (1024, 2816, 1408), (520, 1032, 1032),
+                                      (72, 200, 1)])
+def test_compact_exact(dtype, d, d_ff, k):
+    L, host = make_layer(d, d_ff, dtype, bias=True, seed=d + k)
+    rs = np.random.default_rng(k)
+    e_np = np.sort(rs.choice(d_ff, size=k, replace=False)).astype(np.int32)
+    e = torch.from_numpy(e_np).to(dev())
+    cs = L.compact(e)
+    assert L.status() == G.OK
+    g, u, dn, bg, bu = cs._keep
+    ref = O.compact_experts(e_np, host["wg"].numpy() if dtype == "f32" else host["wg"].view(torch.int16).numpy(),
+                            host["wu"].numpy() if dtype == "f32" else host["wu"].view(torch.int16).numpy(),
+                            host["wd"].numpy() if dtype == "f32" else host["wd"].view(torch.int16).numpy(),
+                            host["bg"].numpy() if dtype == "f32" else host["bg"].view(torch.int16).numpy(),
+                            host["bu"].numpy() if dtype == "f32" else host["bu"].view(torch.int16).numpy())
+    bits = (lambda t: t.cpu().numpy()) if dtype == "f32" else (lambda t: t.cpu().view(torch.int16).numpy())
+    assert np.array_equal(bits(g), ref["w_gate"])
+    assert np.array_equal(bits(u), ref["w_up"])
+    assert np.array_equal(bits(dn)[:, :k], ref["w_down"])
+    assert np.all(bits(dn)[:, k:] == 0)                       # padding columns are zero
+    assert np.array_equal(bits(bg), ref["b_gate"]) and np.array_equal(bits(bu), ref["b_up"])
+
+
+def test_compact_out_of_range_index_is_reported_not_read():
+    L, host = make_layer(64, 96, "bf16")
+    e = torch.tensor([0, 5, 96, 7], dtype=torch.int32, device=dev())   # 96 is out of range
+    cs = L.compact(e)
+    assert L.status() == G.ERR_INVALID_ARG
+    g = cs._keep[0].cpu()
+    assert torch.all(g[2] == 0) and torch.equal(g[1], host["wg"][5])
+    G.griffin_workspace_init(L.ws)
+    assert L.status() == G.OK
+
+
+# ----------------------------------------------------------------- decode ---
+
+DECODE_SHAPES = [
+    # d, d_ff, k, B
+    (256, 688, 344, 1),      # the tiny workload
+    (64, 96, 37, 3),         # odd k -> padded ldk, several sequences
+    (1000, 1504, 751, 2),    # d not a multiple of the vector tiling
+    (2048, 5632, 2816, 1),
+    (3072, 4096, 4096, 1),   # k = d_ff
+    (4096, 11008, 5504, 1),  # Llama-2-7B shape
+    (5120, 2048, 1024, 8),   # widest d of the workloads, batch 8
+    (8192, 1024, 512, 1),    # largest supported d
+]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("d,d_ff,k,B", DECODE_SHAPES)
+def test_decode_matches_oracle(dtype, d, d_ff, k, B):
+    act = "geglu_tanh" if d == 3072 else "swiglu"
+    L, host = make_layer(d, d_ff, dtype, act=act, bias=(d_ff < 2000), seed=d + k, n_seq=B)
+    rs = np.random.default_rng(d + k)
+    x = rand((B, d), TD[dtype], 99)
+    sets, refs = [], []
+    for b in range(B):
+        e_np = np.sort(rs.choice(d_ff, size=k, replace=False)).astype(np.int32)
+        sets.append(L.compact(torch.from_numpy(e_np).to(dev())))
+        c = O.compact_experts(e_np, h64(host, "wg"), h64(host, "wu"), h64(host, "wd"), h64(host, "bg"), h64(host, "bu"))
+        refs.append(O.ff_pruned(np64(x[b]), c, act, h64(host, "bd")))
+    y = L.decode(sets, x)
+    y2 = L.decode(sets, x, G.DECODE_OVERLAP_WEIGHT_PREFETCH)
+    y3 = L.decode(sets, x, G.DECODE_OVERLAP_WEIGHT_PREFETCH)
+    assert L.status() == G.OK
+    for b in range(B):
+        assert rel_l2(np64(y[b]), refs[b]) < TOL_OUT[dtype], b
+    assert torch.equal(y, y2) and torch.equal(y, y3)   # deterministic, launch mode does not matter
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_decode_with_all_neurons_is_the_dense_ff(dtype):
+    d, d_ff = 512, 1536
+    L, host = make_layer(d, d_ff, dtype, act="geglu_tanh", bias=True)
+    x = rand((2, d), TD[dtype], 3)
+    y = L.decode([L.dense_set(), L.dense_set()], x)
+    ref, _ = O.ff_dense(np64(x), h64(host, "wg"), h64(host, "wu"), h64(host, "wd"), "geglu_tanh",
+                        h64(host, "bg"), h64(host, "bu"), h64(host, "bd"))
+    assert rel_l2(np64(y), ref) < TOL_OUT[dtype]
+    # and the compacted copy of E = everything gives the same bits as the aliased weights
+    cs = L.compact(torch.arange(d_ff, dtype=torch.int32, device=dev()))
+    assert torch.equal(L.decode([cs, cs], x), y)
+
+
+def test_decode_many_steps_back_to_back_with_overlap():
+    d, d_ff, k = 1024, 2816, 1408
+    L, host = make_layer(d, d_ff, "bf16")
+    e_np = np.arange(0, d_ff, 2, dtype=np.int32)
+    cs = L.compact(torch.from_numpy(e_np).to(dev()))
+    xs = rand((16, d), torch.bfloat16, 11).to(dev())
+    ys = torch.empty_like(xs)
+    arr = G.compact_array([cs])
+    torch.cuda.synchronize()
+    for t in range(16):
+        G.griffin_ff_decode(L.desc, arr, None, xs[t:t + 1], ys[t:t + 1], L.ws, G.DECODE_OVERLAP_WEIGHT_PREFETCH)
+    assert L.status() == G.OK
+    c = O.compact_experts(e_np, h64(host, "wg"), h64(host, "wu"), h64(host, "wd"))
+    ref = O.ff_pruned(np64(xs), c, "swiglu")
+    assert rel_l2(np64(ys), ref) < TOL_OUT["bf16"]
+
+
+# ---------------------------------------------------------------- prefill ---
+
+PREFILL_SHAPES = [(64, 256, 688), (1, 64, 96), (37, 72, 200), (130, 512, 1032), (256, 1024, 2816)]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("act", ["swiglu", "geglu_tanh", "reglu"])
+@pytest.mark.parametrize("S,d,d_ff", PREFILL_SHAPES)
+def test_prefill_score_matches_oracle(dtype, act, S, d, d_ff):
+    L, host = make_layer(d, d_ff, dtype, act=act, bias=(S == 37), seed=S + d, S_max=S)
+    x = rand((S, d), TD[dtype], 5) + rand((1, d), TD[dtype], 6, 4.0 / d ** 0.5)
+    y, s = L.prefill(x)
+    ref_y, ref_z = O.ff_dense(np64(x), h64(host, "wg"), h64(host, "wu"), h64(host, "wd"), act,
+                              h64(host, "bg"), h64(host, "bu"), h64(host, "bd"))
+    ref_s = O.flock_score(ref_z)
+    assert rel_l2(np64(y), ref_y) < TOL_OUT[dtype]
+    s = np64(s)
+    # relative to the typical score: entries near zero carry no relative information
+    assert np.max(np.abs(s - ref_s)) / np.sqrt(S / d_ff) < 3 * TOL_SCORE[dtype]
+    big = ref_s > 0.1 * np.sqrt(S / d_ff)
+    assert np.max(np.abs(s[big] - ref_s[big]) / ref_s[big]) < 3 * TOL_SCORE[dtype]
+    assert abs(float(np.sum(s * s)) - S) < 1e-3 * S     # rows of Zbar are unit vectors
+    _, s2 = L.prefill(x, want_y=False)
+    assert np.array_equal(np64(s2), s)                   # deterministic; y is optional
+
+
+def test_prefill_zero_row_contributes_nothing():
+    S, d, d_ff = 16, 64, 96
+    L, host = make_layer(d, d_ff, "f32", S_max=S)
+    x = rand((S, d), torch.float32, 8)
+    x[3] = 0.0
+    y, s = L.prefill(x)
+    s = np64(s)
+    assert np.all(np.isfinite(s)) and abs(float(np.sum(s * s)) - (S - 1)) < 1e-4 * S
+    _, z = O.ff_dense(np64(x), h64(host, "wg"), h64(host, "wu"), h64(host, "wd"), "swiglu")
+    assert np.max(np.abs(s - O.flock_score(z))) < 1e-5
+    assert torch.all(y[3] == 0)
