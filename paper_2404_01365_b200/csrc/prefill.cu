@@ -1,15 +1,17 @@
 // Prompt-phase FF and selection statistic (Section 4.2, Eqs. 1, 3 and 6 of the GRIFFIN paper).
 //
 //   1. Z = sigma(X W_g^T + b_g) * (X W_1^T + b_1)          [S, d_ff]  (Eq. 3), stored in the
-//      storage dtype; the same kernel leaves, per token and per column tile, the partial
-//      sum of squares of the stored row                                 (for ||Z_i||^2)
+//      storage dtype as the operand of step 2 and, for bf16 storage, once more in fp32
+//      for the statistic (a bf16-rounded Z would move s by up to 2^-8, more than the
+//      margin by which neighbouring neurons differ); the same kernel leaves, per token
+//      and per column tile, the partial sum of squares of the fp32 row   (for ||Z_i||^2)
 //   2. Y = Z W_2^T + b_2                                    [S, d]     (Eq. 1)
 //   3. inv_i = 1 / ||Z_i||_2^2  (0 for an all-zero row)
 //   4. colpart[chunk, j] = sum over the chunk's tokens of Z_ij^2 * inv_i
 //   5. s_j = sqrt(sum over chunks of colpart[chunk, j])                 (Eq. 6)
 //
 // The row normaliser spans every column tile, so the column sums cannot finish inside
-// step 1: steps 3-5 re-read Z (which mostly still sits in L2).  All partial sums are kept
+// step 1: steps 3-5 re-read the fp32 Z (which mostly still sits in L2).  All partial sums are kept
 // and added in a fixed order, so s is deterministic.
 //
 // This file holds the fp32-FMA (SIMT) matrix kernels, which serve the fp32 storage type
@@ -35,6 +37,8 @@ PrefillScratch prefill_scratch(const griffin_ff_desc *desc, int S) {
     size_t off = 0;
     ps.z_off = off;
     off = align_up(off + (size_t)S * desc->d_ff * esz, 256);
+    ps.zf_off = off;
+    if (desc->dtype != GRIFFIN_DT_F32) off = align_up(off + (size_t)S * desc->d_ff * sizeof(float), 256);
     ps.rowsq_off = off;
     off = align_up(off + (size_t)S * ps.n_col_tiles * sizeof(float), 256);
     ps.inv_off = off;
@@ -72,6 +76,7 @@ template <typename T>
 __global__ void __launch_bounds__(PF_THREADS) ff1_simt_kernel(const T *__restrict__ x, const T *__restrict__ w_gate,
                                                               const T *__restrict__ w_up, const T *__restrict__ b_gate,
                                                               const T *__restrict__ b_up, T *__restrict__ z,
+                                                              float *__restrict__ zf,  // fp32 copy, or null
                                                               float *__restrict__ rowsq, int S, int d, int d_ff,
                                                               int n_col_tiles, int act) {
     __shared__ float xs[PF_BK][PF_BM + PF_PAD], gs[PF_BK][PF_BN + PF_PAD], us[PF_BK][PF_BN + PF_PAD];
@@ -111,10 +116,10 @@ __global__ void __launch_bounds__(PF_THREADS) ff1_simt_kernel(const T *__restric
                 float g = ga[i][j], u = ua[i][j];
                 if (b_gate) g += Elem<T>::to_float(b_gate[col]);
                 if (b_up) u += Elem<T>::to_float(b_up[col]);
-                const T zt = Elem<T>::from_float(sigma_rt(act, g) * u);
-                z[(size_t)row * d_ff + col] = zt;
-                const float zf = Elem<T>::to_float(zt);  // the norm is that of the stored row
-                sq = fmaf(zf, zf, sq);
+                const float zv = sigma_rt(act, g) * u;
+                z[(size_t)row * d_ff + col] = Elem<T>::from_float(zv);
+                if (zf) zf[(size_t)row * d_ff + col] = zv;
+                sq = fmaf(zv, zv, sq);
             }
         }
         red[ty * 4 + i][tx] = sq;
@@ -178,28 +183,23 @@ __global__ void row_inv_kernel(const float *__restrict__ rowsq, int S, int n_col
     if (lane == 0) inv[row] = sq > 0.f ? 1.0f / sq : 0.f;
 }
 
-// Step 4: a thread owns 16 bytes' worth of neighbouring columns over one chunk of tokens.
-template <typename T>
-__global__ void __launch_bounds__(128) col_partial_kernel(const T *__restrict__ z, const float *__restrict__ inv, int S,
-                                                          int d_ff, float *__restrict__ colpart) {
-    constexpr int VEC = Elem<T>::VEC;
-    const int col = (blockIdx.x * 128 + threadIdx.x) * VEC;
+// Step 4: a thread owns four neighbouring columns of the fp32 Z over one chunk of tokens.
+__global__ void __launch_bounds__(128) col_partial_kernel(const float *__restrict__ z, const float *__restrict__ inv,
+                                                          int S, int d_ff, float *__restrict__ colpart) {
+    const int col = (blockIdx.x * 128 + threadIdx.x) * 4;
     if (col >= d_ff) return;
     const int r0 = blockIdx.y * PF_ROW_CHUNK, r1 = min(S, r0 + PF_ROW_CHUNK);
-    float acc[VEC];
-#pragma unroll
-    for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 4
     for (int r = r0; r < r1; ++r) {
-        float f[VEC];
-        Elem<T>::unpack(*reinterpret_cast<const uint4 *>(z + (size_t)r * d_ff + col), f);
+        const float4 f = *reinterpret_cast<const float4 *>(z + (size_t)r * d_ff + col);
         const float w = __ldg(inv + r);
-#pragma unroll
-        for (int e = 0; e < VEC; ++e) acc[e] = fmaf(f[e] * f[e], w, acc[e]);
+        acc.x = fmaf(f.x * f.x, w, acc.x);
+        acc.y = fmaf(f.y * f.y, w, acc.y);
+        acc.z = fmaf(f.z * f.z, w, acc.z);
+        acc.w = fmaf(f.w * f.w, w, acc.w);
     }
-    float *dst = colpart + (size_t)blockIdx.y * d_ff + col;
-#pragma unroll
-    for (int e = 0; e < VEC; ++e) dst[e] = acc[e];
+    *reinterpret_cast<float4 *>(colpart + (size_t)blockIdx.y * d_ff + col) = acc;
 }
 
 // Step 5.
@@ -218,6 +218,8 @@ static griffin_status prefill_typed(const griffin_ff_desc *desc, const griffin_f
     const int d = desc->d, d_ff = desc->d_ff;
     const PrefillScratch ps = prefill_scratch(desc, S);
     T *z = reinterpret_cast<T *>(scratch + ps.z_off);
+    constexpr bool kBf16 = std::is_same<T, __nv_bfloat16>::value;
+    float *zf = kBf16 ? reinterpret_cast<float *>(scratch + ps.zf_off) : nullptr;
     float *rowsq = reinterpret_cast<float *>(scratch + ps.rowsq_off);
     float *inv = reinterpret_cast<float *>(scratch + ps.inv_off);
     float *colpart = reinterpret_cast<float *>(scratch + ps.colpart_off);
@@ -225,10 +227,10 @@ static griffin_status prefill_typed(const griffin_ff_desc *desc, const griffin_f
     int n_col_tiles = 0;
     bool ff2_done = false;
     bool use_tc = false;
-    if constexpr (std::is_same<T, __nv_bfloat16>::value) use_tc = prefill_tc_supported(desc, S);
+    if constexpr (kBf16) use_tc = prefill_tc_supported(desc, S);
     if (use_tc) {
-        if constexpr (std::is_same<T, __nv_bfloat16>::value) {
-            griffin_status st = launch_prefill_tc(desc, w, x, S, y, z, rowsq, &n_col_tiles, ws, stream);
+        if constexpr (kBf16) {
+            griffin_status st = launch_prefill_tc(desc, w, x, S, y, z, zf, rowsq, &n_col_tiles, ws, stream);
             if (st != GRIFFIN_OK) return st;
         }
         ff2_done = true;
@@ -237,7 +239,7 @@ static griffin_status prefill_typed(const griffin_ff_desc *desc, const griffin_f
         const dim3 g1(n_col_tiles, (S + PF_BM - 1) / PF_BM);
         ff1_simt_kernel<T><<<g1, PF_THREADS, 0, stream>>>(
             static_cast<const T *>(x), static_cast<const T *>(w->w_gate), static_cast<const T *>(w->w_up),
-            static_cast<const T *>(w->b_gate), static_cast<const T *>(w->b_up), z, rowsq, S, d, d_ff, n_col_tiles,
+            static_cast<const T *>(w->b_gate), static_cast<const T *>(w->b_up), z, zf, rowsq, S, d, d_ff, n_col_tiles,
             desc->act);
         if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
     }
@@ -250,9 +252,9 @@ static griffin_status prefill_typed(const griffin_ff_desc *desc, const griffin_f
     }
     row_inv_kernel<<<(S + 7) / 8, 256, 0, stream>>>(rowsq, S, n_col_tiles, inv);
     if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
-    constexpr int VEC = Elem<T>::VEC;
-    const dim3 g4((d_ff + 128 * VEC - 1) / (128 * VEC), ps.n_row_chunks);
-    col_partial_kernel<T><<<g4, 128, 0, stream>>>(z, inv, S, d_ff, colpart);
+    const float *z32 = kBf16 ? zf : reinterpret_cast<const float *>(z);
+    const dim3 g4((d_ff + 511) / 512, ps.n_row_chunks);
+    col_partial_kernel<<<g4, 128, 0, stream>>>(z32, inv, S, d_ff, colpart);
     if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
     score_finish_kernel<<<(d_ff + 255) / 256, 256, 0, stream>>>(colpart, ps.n_row_chunks, d_ff, score);
     if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;

@@ -3,7 +3,7 @@
 namespace griffin {
 bool prefill_tc_supported(const griffin_ff_desc *, int) { return false; }
 griffin_status launch_prefill_tc(const griffin_ff_desc *, const griffin_ff_weights *, const void *, int, void *,
-                                 __nv_bfloat16 *, float *, int *, void *, cudaStream_t) {
+                                 __nv_bfloat16 *, float *, float *, int *, void *, cudaStream_t) {
     return GRIFFIN_ERR_UNSUPPORTED;
 }
 }  // namespace griffin

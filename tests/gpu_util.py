@@ -6,8 +6,13 @@ from oracle import griffin_oracle as O
 from paper_2404_01365_b200 import binding as G
 
 TOL_OUT = {"f32": 1e-4, "bf16": 2e-2}      # relative L2 of outputs
-TOL_SCORE = {"f32": 1e-5, "bf16": 1e-3}    # relative L-inf of the statistic
-TIE_WINDOW = 1e-3                           # expert sets may differ only this close to the k-th score
+
+
+def score_tol(dtype):
+    """Relative tolerance on each s_j.  The statistic is computed from fp32 activations in both
+    storage types; what is left is fp32 accumulation noise over d (dot products), d_ff (row
+    norm) and S (column sum) terms."""
+    return 1e-5 if dtype == "f32" else 2e-5
 
 
 def dev():

@@ -5,7 +5,7 @@ import torch
 
 from oracle import griffin_oracle as O
 from paper_2404_01365_b200 import binding as G
-from gpu_util import (GpuLayer, TOL_OUT, TOL_SCORE, check_expert_set, dev, np64, rand, rel_l2)
+from gpu_util import (GpuLayer, TOL_OUT, check_expert_set, dev, np64, rand, rel_l2, score_tol)
 
 pytestmark = pytest.mark.gpu
 
@@ -139,7 +139,7 @@ def test_decode_matches_oracle(dtype, d, d_ff, k, B):
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_decode_with_all_neurons_is_the_dense_ff(dtype):
     d, d_ff = 512, 1536
-    L, host = make_layer(d, d_ff, dtype, act="geglu_tanh", bias=True)
+    L, host = make_layer(d, d_ff, dtype, act="geglu_tanh", bias=True, n_seq=2)
     x = rand((2, d), TD[dtype], 3)
     y = L.decode([L.dense_set(), L.dense_set()], x)
     ref, _ = O.ff_dense(np64(x), h64(host, "wg"), h64(host, "wu"), h64(host, "wd"), "geglu_tanh",
@@ -184,11 +184,8 @@ def test_prefill_score_matches_oracle(dtype, act, S, d, d_ff):
     ref_s = O.flock_score(ref_z)
     assert rel_l2(np64(y), ref_y) < TOL_OUT[dtype]
     s = np64(s)
-    # relative to the typical score: entries near zero carry no relative information
-    assert np.max(np.abs(s - ref_s)) / np.sqrt(S / d_ff) < 3 * TOL_SCORE[dtype]
-    big = ref_s > 0.1 * np.sqrt(S / d_ff)
-    assert np.max(np.abs(s[big] - ref_s[big]) / ref_s[big]) < 3 * TOL_SCORE[dtype]
-    assert abs(float(np.sum(s * s)) - S) < 1e-3 * S     # rows of Zbar are unit vectors
+    assert np.all(np.abs(s - ref_s) <= score_tol(dtype) * ref_s + 1e-6 * np.sqrt(S / d_ff))
+    assert abs(float(np.sum(s * s)) - S) < 1e-5 * S     # rows of Zbar are unit vectors
     _, s2 = L.prefill(x, want_y=False)
     assert np.array_equal(np64(s2), s)                   # deterministic; y is optional
 
