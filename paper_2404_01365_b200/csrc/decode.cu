@@ -62,18 +62,22 @@ static size_t dec_smem_bytes(int n_stages, int stage_bytes) {
     return (size_t)n_stages * stage_bytes + 2 * n_stages * sizeof(uint64_t) + 2 * DEC_PART_FLOATS * sizeof(float) + 16;
 }
 
-// Barrier wait that gives up after WAIT_LIMIT_NS, or as soon as another thread of the CTA
+// Barrier wait that gives up after WAIT_LIMIT_CYCLES, or as soon as another thread of the CTA
 // has given up.  On a give-up the status word is raised and false is returned.
 __device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort, void *ws,
                                               int where) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_timer_ns();
+    // Fast path: plain polling.  The clock is only consulted every few thousand polls, so a
+    // wait that succeeds (every wait of a healthy run) never pays for reading it.
+#pragma unroll 1
+    for (int i = 0; i < 4096; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
     for (;;) {
 #pragma unroll 1
-        for (int i = 0; i < 128; ++i)
+        for (int i = 0; i < 4096; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort) return false;
-        if (global_timer_ns() - t0 > WAIT_LIMIT_NS) {
+        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
             *abort = 1;
             raise_status(ws, DEV_STATUS_TIMEOUT, where);
             return false;
@@ -93,9 +97,10 @@ __device__ __forceinline__ void producer_drain(const DecSmem &s, int n_stages, u
     for (uint32_t it = first; it < issued; ++it) {
         const int stage = it % n_stages;
         const uint32_t parity = (it / n_stages) & 1;
-        const unsigned long long t0 = global_timer_ns();
+        if (mbar_try_wait(&s.full[stage], parity)) continue;
+        const long long t0 = clock64();
         while (!mbar_try_wait(&s.full[stage], parity))
-            if (global_timer_ns() - t0 > WAIT_LIMIT_NS) break;
+            if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
     }
 }
 
@@ -391,10 +396,13 @@ static cudaError_t launch_maybe_overlapped(const void *func, dim3 grid, dim3 blo
     return cudaLaunchKernelExC(&cfg, func, args);
 }
 
+#ifndef GRIFFIN_DEC_STAGE_KB
+#define GRIFFIN_DEC_STAGE_KB 96
+#endif
 static int pick_stages(int stage_bytes) {
     // about 96 KB of stages: deep enough to cover HBM latency, small enough that the next
     // kernel's CTA fits beside this one on the SM and can prefetch its own weights
-    int n = (96 * 1024) / stage_bytes;
+    int n = (GRIFFIN_DEC_STAGE_KB * 1024) / stage_bytes;
     if (n < 2) n = 2;
     if (n > 12) n = 12;
     return n;
