@@ -2,6 +2,9 @@
 //   z_hat = sigma(W_g_hat x + b_g_hat) * (W_1_hat x + b_1_hat)        kernel "gate_up"
 //   y_hat = W_2_hat z_hat + b_2                                        kernel "down"
 //
+// This file holds the fp32-FMA kernels (fp32 storage) and the dispatcher; bf16 storage goes
+// through the warp-MMA kernels in decode_mma.cu, which share the pipeline design below.
+//
 // At batch 1..8 both products are matrix-vector products whose cost is the single pass
 // over the compact weights, so both kernels are built around keeping HBM busy:
 //   * one CTA per SM, persistent over its share of the work items;
@@ -13,96 +16,9 @@
 //     the previous kernel on the stream has finished; everything that depends on that
 //     kernel (x, z, y) is touched only after griddepcontrol.wait.
 // Results are deterministic: every sum has a fixed order.
-#include "common.cuh"
-#include "launch.h"
+#include "decode_common.cuh"
 
 namespace griffin {
-
-constexpr int DEC_CONSUMER_WARPS = 8;
-constexpr int DEC_CONSUMERS = DEC_CONSUMER_WARPS * 32;
-constexpr int DEC_THREADS = DEC_CONSUMERS + 32;  // + producer warp
-constexpr int DEC_MAX_ROWS = 64;                 // rows per work item (neurons / output rows)
-constexpr int DEC_DOWN_ITER = 2;                 // 16-byte vectors per consumer thread per row segment
-constexpr int DEC_PART_FLOATS = DEC_MAX_ROWS * DEC_CONSUMER_WARPS * 2;  // one parity buffer
-
-struct DecodeSeq {
-    const void *w_gate, *w_up, *w_down, *b_gate, *b_up;
-};
-struct DecodeParams {
-    DecodeSeq seq[GRIFFIN_MAX_BATCH];
-    const void *b_down;
-    const void *x;  // [B, d]
-    void *y;        // [B, d]
-    float *z;       // [B, ldk] fp32 scratch
-    void *ws;       // workspace header (status word), may be null
-    int d, k, ldk, B;
-    int n_slices;  // work items per sequence
-    int n_stages;
-    int kt_len;    // down kernel: elements per k-tile (multiple of 8)
-    int n_ktiles;
-};
-
-struct DecSmem {
-    uint8_t *stages;
-    uint64_t *full, *empty;
-    float *part;
-    volatile int *abort;
-};
-
-__device__ __forceinline__ DecSmem carve(uint8_t *smem, int n_stages, int stage_bytes) {
-    DecSmem s;
-    s.stages = smem;
-    s.full = reinterpret_cast<uint64_t *>(smem + (size_t)n_stages * stage_bytes);
-    s.empty = s.full + n_stages;
-    s.part = reinterpret_cast<float *>(s.empty + n_stages);
-    s.abort = reinterpret_cast<volatile int *>(s.part + 2 * DEC_PART_FLOATS);
-    return s;
-}
-static size_t dec_smem_bytes(int n_stages, int stage_bytes) {
-    return (size_t)n_stages * stage_bytes + 2 * n_stages * sizeof(uint64_t) + 2 * DEC_PART_FLOATS * sizeof(float) + 16;
-}
-
-// Barrier wait that gives up after WAIT_LIMIT_CYCLES, or as soon as another thread of the CTA
-// has given up.  On a give-up the status word is raised and false is returned.
-__device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort, void *ws,
-                                              int where) {
-    // Fast path: plain polling.  The clock is only consulted every few thousand polls, so a
-    // wait that succeeds (every wait of a healthy run) never pays for reading it.
-#pragma unroll 1
-    for (int i = 0; i < 4096; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    for (;;) {
-#pragma unroll 1
-        for (int i = 0; i < 4096; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
-        if (*abort) return false;
-        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
-            *abort = 1;
-            raise_status(ws, DEV_STATUS_TIMEOUT, where);
-            return false;
-        }
-    }
-}
-
-__device__ __forceinline__ void consumer_barrier() {
-    asm volatile("bar.sync 1, %0;" ::"n"(DEC_CONSUMERS) : "memory");
-}
-
-// After its last issue the producer stays until every copy it started has landed, so the
-// CTA's shared memory is never released under a copy in flight.  (Only matters after a
-// give-up: normally the consumers have already waited for every stage.)
-__device__ __forceinline__ void producer_drain(const DecSmem &s, int n_stages, uint32_t issued) {
-    const uint32_t first = issued > (uint32_t)n_stages ? issued - n_stages : 0;
-    for (uint32_t it = first; it < issued; ++it) {
-        const int stage = it % n_stages;
-        const uint32_t parity = (it / n_stages) & 1;
-        if (mbar_try_wait(&s.full[stage], parity)) continue;
-        const long long t0 = clock64();
-        while (!mbar_try_wait(&s.full[stage], parity))
-            if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
-    }
-}
 
 // ---------------------------------------------------------------------------------------
 // Kernel gate_up:
@@ -381,7 +297,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_down_kernel(const __grid_c
 // ---------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------
-static cudaError_t launch_maybe_overlapped(const void *func, dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+cudaError_t launch_maybe_overlapped(const void *func, dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
                                            bool overlap, void **args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
@@ -408,7 +324,7 @@ static int pick_stages(int stage_bytes) {
     return n;
 }
 
-static int slices_for(int rows, int grid) {
+int slices_for(int rows, int grid) {
     // a multiple of the grid, fine enough that one item has at most DEC_MAX_ROWS rows
     int per = (rows + grid * DEC_MAX_ROWS - 1) / (grid * DEC_MAX_ROWS);
     if (per < 1) per = 1;
@@ -416,28 +332,9 @@ static int slices_for(int rows, int grid) {
 }
 
 template <typename T>
-static griffin_status decode_typed(const griffin_ff_desc *desc, int B, const griffin_ff_compact *sets,
-                                   const void *b_down, const void *x, void *y, float *z, void *ws, uint32_t flags,
-                                   cudaStream_t stream) {
+static griffin_status decode_simt(DecodeParams &p, int act, uint32_t flags, cudaStream_t stream) {
     constexpr int VEC = Elem<T>::VEC;
-    DecodeParams p = {};
-    for (int b = 0; b < B; ++b) {
-        p.seq[b].w_gate = sets[b].w_gate_c;
-        p.seq[b].w_up = sets[b].w_up_c;
-        p.seq[b].w_down = sets[b].w_down_c;
-        p.seq[b].b_gate = sets[b].b_gate_c;
-        p.seq[b].b_up = sets[b].b_up_c;
-    }
-    p.b_down = b_down;
-    p.x = x;
-    p.y = y;
-    p.z = z;
-    p.ws = ws;
-    p.d = desc->d;
-    p.k = sets[0].k;
-    p.ldk = sets[0].ldk;
-    p.B = B;
-
+    const int B = p.B;
     const int sms = device_sm_count();
     if (sms <= 0) return GRIFFIN_ERR_CUDA;
     const bool overlap = (flags & GRIFFIN_DECODE_OVERLAP_WEIGHT_PREFETCH) != 0;
@@ -460,7 +357,6 @@ static griffin_status decode_typed(const griffin_ff_desc *desc, int B, const gri
             default: return GRIFFIN_ERR_UNSUPPORTED;
         }
         if (ensure_dynamic_smem(fn, smem) != cudaSuccess) return GRIFFIN_ERR_CUDA;
-        int act = desc->act;
         void *args[] = {&p, &act};
         if (launch_maybe_overlapped(fn, dim3(grid), dim3(DEC_THREADS), smem, stream, overlap, args) != cudaSuccess)
             return GRIFFIN_ERR_CUDA;
@@ -486,9 +382,25 @@ static griffin_status decode_typed(const griffin_ff_desc *desc, int B, const gri
 
 griffin_status launch_decode(const griffin_ff_desc *desc, int B, const griffin_ff_compact *sets, const void *b_down,
                              const void *x, void *y, float *z, void *ws, uint32_t flags, cudaStream_t stream) {
-    if (desc->dtype == GRIFFIN_DT_F32)
-        return decode_typed<float>(desc, B, sets, b_down, x, y, z, ws, flags, stream);
-    return decode_typed<__nv_bfloat16>(desc, B, sets, b_down, x, y, z, ws, flags, stream);
+    DecodeParams p = {};
+    for (int b = 0; b < B; ++b) {
+        p.seq[b].w_gate = sets[b].w_gate_c;
+        p.seq[b].w_up = sets[b].w_up_c;
+        p.seq[b].w_down = sets[b].w_down_c;
+        p.seq[b].b_gate = sets[b].b_gate_c;
+        p.seq[b].b_up = sets[b].b_up_c;
+    }
+    p.b_down = b_down;
+    p.x = x;
+    p.y = y;
+    p.z = z;
+    p.ws = ws;
+    p.d = desc->d;
+    p.k = sets[0].k;
+    p.ldk = sets[0].ldk;
+    p.B = B;
+    if (desc->dtype == GRIFFIN_DT_F32) return decode_simt<float>(p, desc->act, flags, stream);
+    return decode_bf16_mma(p, desc->act, flags, stream);
 }
 
 }  // namespace griffin

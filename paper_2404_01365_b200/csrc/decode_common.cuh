@@ -1,0 +1,108 @@
+// Pieces shared by the two families of decode kernels (fp32-FMA and warp-MMA).
+#pragma once
+
+#include "common.cuh"
+#include "launch.h"
+
+namespace griffin {
+
+constexpr int DEC_CONSUMER_WARPS = 8;
+constexpr int DEC_CONSUMERS = DEC_CONSUMER_WARPS * 32;
+constexpr int DEC_THREADS = DEC_CONSUMERS + 32;  // + producer warp
+constexpr int DEC_MAX_ROWS = 64;                 // rows per work item (neurons / output rows)
+constexpr int DEC_DOWN_ITER = 2;                 // 16-byte vectors per consumer thread per row segment
+constexpr int DEC_PART_FLOATS = DEC_MAX_ROWS * DEC_CONSUMER_WARPS * 2;  // one parity buffer
+
+struct DecodeSeq {
+    const void *w_gate, *w_up, *w_down, *b_gate, *b_up;
+};
+struct DecodeParams {
+    DecodeSeq seq[GRIFFIN_MAX_BATCH];
+    const void *b_down;
+    const void *x;  // [B, d]
+    void *y;        // [B, d]
+    float *z;       // [B, ldk] fp32 scratch
+    void *ws;       // workspace header (status word), may be null
+    int d, k, ldk, B;
+    int n_slices;  // work items per sequence
+    int n_stages;
+    int kt_len;    // down kernel: elements per k-tile (multiple of 8)
+    int n_ktiles;
+};
+
+struct DecSmem {
+    uint8_t *stages;
+    uint64_t *full, *empty;
+    float *part;
+    volatile int *abort;
+};
+
+__device__ __forceinline__ DecSmem carve(uint8_t *smem, int n_stages, int stage_bytes) {
+    DecSmem s;
+    s.stages = smem;
+    s.full = reinterpret_cast<uint64_t *>(smem + (size_t)n_stages * stage_bytes);
+    s.empty = s.full + n_stages;
+    s.part = reinterpret_cast<float *>(s.empty + n_stages);
+    s.abort = reinterpret_cast<volatile int *>(s.part + 2 * DEC_PART_FLOATS);
+    return s;
+}
+static inline size_t dec_smem_bytes(int n_stages, int stage_bytes) {
+    return (size_t)n_stages * stage_bytes + 2 * n_stages * sizeof(uint64_t) + 2 * DEC_PART_FLOATS * sizeof(float) + 16;
+}
+
+// Barrier wait that gives up after WAIT_LIMIT_CYCLES, or as soon as another thread of the CTA
+// has given up.  On a give-up the status word is raised and false is returned.
+__device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort, void *ws,
+                                              int where) {
+    // Fast path: plain polling.  The clock is only consulted every few thousand polls, so a
+    // wait that succeeds (every wait of a healthy run) never pays for reading it.
+#pragma unroll 1
+    for (int i = 0; i < 4096; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 4096; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort) return false;
+        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+            *abort = 1;
+            raise_status(ws, DEV_STATUS_TIMEOUT, where);
+            return false;
+        }
+    }
+}
+
+__device__ __forceinline__ void consumer_barrier() {
+    asm volatile("bar.sync 1, %0;" ::"n"(DEC_CONSUMERS) : "memory");
+}
+
+// After its last issue the producer stays until every copy it started has landed, so the
+// CTA's shared memory is never released under a copy in flight.  (Only matters after a
+// give-up: normally the consumers have already waited for every stage.)
+__device__ __forceinline__ void producer_drain(const DecSmem &s, int n_stages, uint32_t issued) {
+    const uint32_t first = issued > (uint32_t)n_stages ? issued - n_stages : 0;
+    for (uint32_t it = first; it < issued; ++it) {
+        const int stage = it % n_stages;
+        const uint32_t parity = (it / n_stages) & 1;
+        if (mbar_try_wait(&s.full[stage], parity)) continue;
+        const long long t0 = clock64();
+        while (!mbar_try_wait(&s.full[stage], parity))
+            if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
+    }
+}
+
+
+// Launches `func`, optionally allowing it to start before the previous kernel on the stream
+// has completed (programmatic dependent launch).
+cudaError_t launch_maybe_overlapped(const void *func, dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                    bool overlap, void **args);
+
+// Number of work items per sequence: a multiple of the grid, fine enough that one item has at
+// most DEC_MAX_ROWS rows.
+int slices_for(int rows, int grid);
+
+// bf16 decode through warp-level MMA (decode_mma.cu).
+griffin_status decode_bf16_mma(DecodeParams &p, int act, uint32_t flags, cudaStream_t stream);
+
+}  // namespace griffin

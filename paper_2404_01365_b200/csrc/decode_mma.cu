@@ -1,0 +1,348 @@
+// Generation-phase pruned FF (Eqs. 4 and 5 of the GRIFFIN paper) for bf16 storage.
+//
+// Same pipeline as the fp32-FMA kernels (persistent CTA per SM, producer warp streaming
+// weight rows into a ring of shared-memory stages with 1-D bulk copies, 8 consumer warps,
+// programmatic dependent launch), but the consumers hand the staged rows to the warp-level
+// tensor-core instruction mma.sync.m16n8k16 instead of unpacking and multiplying element by
+// element.  The products are matrix-vector products, so this is not about FLOPs: it cuts the
+// instructions issued per staged byte several times over, which is what kept the FMA version
+// from reaching HBM speed.
+//
+// Stages are made of few, large, contiguous copies (measured on B200: every bulk copy costs
+// about 30 ns of issue time and every stage hand-over about 240 ns, whatever their size, so
+// a stage should carry 24-32 KB in two to four copies).  A stage therefore holds R "pairs"
+// of whole rows (or 16 KB chunks of long rows): for gate_up a pair is (gate row j, up row
+// j), for down it is (row c, row c+1) of W_2_hat.  Both rows of a pair meet the same vector
+// (x, or z).
+//
+// How one pair meets the vector in the MMA (M = 16, N = 8, K = 16):
+//   * A row is a sequence of 16-byte units (8 elements).  In a block of 32 units, lane l of
+//     a warp reads unit l of both rows and of the vector: every 8 consecutive lanes read 128
+//     contiguous bytes, so there are no bank conflicts and nothing needs padding.
+//   * With g = lane / 4 and t = lane % 4, the MMA takes the lane's row data as rows g
+//     (first real row) and g + 8 (second real row) of A, and its vector data as column g
+//     of B, both at K positions 2t, 2t+1, 2t+8, 2t+9: "virtual row" g of a real row is the
+//     set of units read by lanes 4g..4g+3, "virtual vector" g the matching units of x (or
+//     z).  The unit's first four elements feed one MMA and the last four a second one (the
+//     MMA sums over K, so any assignment of elements to K positions works as long as the
+//     row and the vector agree, and here the same lane supplies both).
+//   * C[m][n] pairs virtual row m with virtual vector n; only the diagonal m = n belongs to
+//     the dot product.  Lane (g, t = g / 2) holds it; three shuffles add the 8 diagonal
+//     entries.  The tensor core does 8x the needed multiplies, which is free here.
+//   * down: z is fp32; it is split into two bf16 numbers z_hi + z_lo and each block runs the
+//     MMAs once against each, into the same accumulators, so 16 bits of z survive.
+//   * 8 / R warps share a pair; their partial sums meet in shared memory at the end of a
+//     work item, in a fixed order.
+#include "decode_common.cuh"
+
+namespace griffin {
+
+constexpr int MMA_CHUNK_UNITS_MAX = 1024;  // 16 KB of one row per stage at most
+constexpr int MMA_STAGE_TARGET = 32 * 1024;
+#ifndef GRIFFIN_DEC_SMEM_KB
+#define GRIFFIN_DEC_SMEM_KB 113
+#endif
+constexpr int MMA_SMEM_TARGET = GRIFFIN_DEC_SMEM_KB * 1024;  // 113 KB = half an SM: the next kernel's CTA fits too
+
+struct MmaPlan {
+    int row_units;    // 16-byte units per real row
+    int n_chunks;     // pieces a row is cut into
+    int chunk_units;  // units per piece (the last may be shorter)
+    int R;            // pairs per stage: 1, 2 or 4
+    int stage_bytes;
+    int n_stages;
+    int vec_bytes;
+};
+
+struct MmaSmem {
+    uint8_t *stages;
+    uint8_t *vec;  // gate_up: x as bf16 [d]; down: z_hi [ldk] then z_lo [ldk]
+    uint64_t *full, *empty;
+    float2 *part;  // [2 parities][DEC_MAX_ROWS pairs][8 warps]
+    volatile int *abort;
+};
+__device__ __forceinline__ MmaSmem carve_mma(uint8_t *smem, const MmaPlan &pl) {
+    MmaSmem s;
+    s.stages = smem;
+    s.vec = smem + (size_t)pl.n_stages * pl.stage_bytes;
+    s.full = reinterpret_cast<uint64_t *>(s.vec + pl.vec_bytes);
+    s.empty = s.full + pl.n_stages;
+    s.part = reinterpret_cast<float2 *>(s.empty + pl.n_stages);
+    s.abort = reinterpret_cast<volatile int *>(s.part + 2 * DEC_MAX_ROWS * DEC_CONSUMER_WARPS);
+    return s;
+}
+static size_t mma_fixed_smem(int n_stages) {
+    return 2 * n_stages * sizeof(uint64_t) + 2 * DEC_MAX_ROWS * DEC_CONSUMER_WARPS * sizeof(float2) + 16;
+}
+
+static MmaPlan make_plan(int row_elems, int vec_bytes) {
+    MmaPlan pl;
+    pl.row_units = row_elems / 8;
+    pl.n_chunks = (pl.row_units + MMA_CHUNK_UNITS_MAX - 1) / MMA_CHUNK_UNITS_MAX;
+    pl.chunk_units = (pl.row_units + pl.n_chunks - 1) / pl.n_chunks;
+    const int pair_bytes = 2 * pl.chunk_units * 16;
+    pl.R = pair_bytes * 4 <= MMA_STAGE_TARGET ? 4 : (pair_bytes * 2 <= MMA_STAGE_TARGET ? 2 : 1);
+    pl.stage_bytes = pl.R * pair_bytes;
+    pl.vec_bytes = vec_bytes;
+    int n = ((int)MMA_SMEM_TARGET - vec_bytes - (int)mma_fixed_smem(8)) / pl.stage_bytes;
+    pl.n_stages = n < 2 ? 2 : (n > 8 ? 8 : n);
+    return pl;
+}
+
+__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// Adds the diagonal of the 16 x 8 accumulator tile: returns (sum over g of C[g][g],
+// sum over g of C[g + 8][g]) in lane 0.  Lane (g, t) holds columns 2t, 2t+1 of rows g, g+8.
+__device__ __forceinline__ float2 diagonal_sum(const float (&c)[4], int g, int t) {
+    float v0 = 0.f, v1 = 0.f;
+    if (t == (g >> 1)) {
+        v0 = (g & 1) ? c[1] : c[0];
+        v1 = (g & 1) ? c[3] : c[2];
+    }
+    // the 8 lanes that hold a diagonal entry are 0, 4, 9, 13, 18, 22, 27, 31
+    v0 += __shfl_xor_sync(0xffffffffu, v0, 4);
+    v1 += __shfl_xor_sync(0xffffffffu, v1, 4);
+    v0 += __shfl_xor_sync(0xffffffffu, v0, 9);
+    v1 += __shfl_xor_sync(0xffffffffu, v1, 9);
+    v0 += __shfl_xor_sync(0xffffffffu, v0, 18);
+    v1 += __shfl_xor_sync(0xffffffffu, v1, 18);
+    return make_float2(v0, v1);
+}
+
+// This warp's share of one pair's chunk: blocks q, q + wpn, ... of 32 units each.
+//   row0,row1 : the two staged rows; vec0 : vector units for this chunk; vec1 : second vector
+//   (down's z_lo); n_units : valid units in this chunk
+template <bool TWO_VECTORS>
+__device__ __forceinline__ void pair_mma(float (&acc)[4], const uint4 *row0, const uint4 *row1, const uint4 *vec0,
+                                         const uint4 *vec1, int n_units, int q, int wpn, int lane) {
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+#pragma unroll 2
+    for (int b = q; b * 32 < n_units; b += wpn) {
+        const int u = b * 32 + lane;  // a warp reads 512 contiguous bytes
+        uint4 r0 = zero, r1 = zero, v = zero, w = zero;
+        if (u < n_units) {  // past the end both operands are zero (stale bytes could be NaN)
+            r0 = row0[u];
+            r1 = row1[u];
+            v = vec0[u];
+            if (TWO_VECTORS) w = vec1[u];
+        }
+        mma_bf16(acc, r0.x, r1.x, r0.y, r1.y, v.x, v.y);
+        mma_bf16(acc, r0.z, r1.z, r0.w, r1.w, v.z, v.w);
+        if (TWO_VECTORS) {
+            mma_bf16(acc, r0.x, r1.x, r0.y, r1.y, w.x, w.y);
+            mma_bf16(acc, r0.z, r1.z, r0.w, r1.w, w.z, w.w);
+        }
+    }
+}
+
+__device__ __forceinline__ void producer_drain_mma(const MmaSmem &s, int n_stages, uint32_t issued) {
+    const uint32_t first = issued > (uint32_t)n_stages ? issued - n_stages : 0;
+    for (uint32_t it = first; it < issued; ++it) {
+        const int stage = it % n_stages;
+        const uint32_t parity = (it / n_stages) & 1;
+        if (mbar_try_wait(&s.full[stage], parity)) continue;
+        const long long t0 = clock64();
+        while (!mbar_try_wait(&s.full[stage], parity))
+            if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
+    }
+}
+
+// DOWN = false: gate_up, z[b, j] = sigma(gate_j . x + b_gate_j) * (up_j . x + b_up_j);
+//               item = (sequence, slice of neurons), pair = neuron.
+// DOWN = true : down, y[b, c] = w_down_c[c, :] . z[b] + b_down[c];
+//               item = (sequence, chunk of output rows), pair = two consecutive rows.
+template <bool DOWN>
+__global__ void __launch_bounds__(DEC_THREADS) decode_mma_kernel(const __grid_constant__ DecodeParams p,
+                                                                 const __grid_constant__ MmaPlan pl, int act) {
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    const MmaSmem s = carve_mma(smem_raw, pl);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        for (int i = 0; i < pl.n_stages; ++i) {
+            mbar_init(&s.full[i], 1);
+            mbar_init(&s.empty[i], DEC_CONSUMER_WARPS);
+        }
+        *s.abort = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+    pdl_launch_dependents();
+
+    const int n_items = p.B * p.n_slices;
+    const int total_rows = DOWN ? p.d : p.k;  // what the slices partition
+    const size_t row_bytes = (size_t)pl.row_units * 16;
+    const int chunk_bytes_max = pl.chunk_units * 16;
+    const int wpn = DEC_CONSUMER_WARPS / pl.R;  // warps per pair
+
+    if (warp == DEC_CONSUMER_WARPS) {
+        // ---- producer warp: weights only, never waits for the previous grid.  Lane l < 2R
+        //      copies row (l & 1) of pair (l >> 1).
+        uint32_t it = 0;
+        bool ok = true;
+        const int my_pair = lane >> 1, my_row = lane & 1;
+        for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+            const int b = item / p.n_slices, sl = item - b * p.n_slices;
+            const int r0 = (int)((long long)sl * total_rows / p.n_slices);
+            const int r1 = (int)((long long)(sl + 1) * total_rows / p.n_slices);
+            const int n_pairs = DOWN ? (r1 - r0 + 1) / 2 : r1 - r0;
+            const uint8_t *mat = static_cast<const uint8_t *>(DOWN ? p.seq[b].w_down
+                                                                   : (my_row ? p.seq[b].w_up : p.seq[b].w_gate));
+            for (int pg = 0; ok && pg < n_pairs; pg += pl.R) {
+                const int pair = pg + my_pair;
+                const int grow = DOWN ? r0 + 2 * pair + my_row : r0 + pair;  // row in the matrix
+                const bool mine = lane < 2 * pl.R && pair < n_pairs && grow < r1;
+                // rows copied in this stage (the same for every chunk of the group)
+                const int rows_in_stage = DOWN ? min(2 * pl.R, r1 - r0 - 2 * pg) : 2 * min(pl.R, n_pairs - pg);
+                for (int c = 0; c < pl.n_chunks; ++c, ++it) {
+                    const int units = min(pl.chunk_units, pl.row_units - c * pl.chunk_units);
+                    const int stage = it % pl.n_stages;
+                    const uint32_t use = it / pl.n_stages;
+                    int go = 1;
+                    if (lane == 0) {
+                        if (use > 0 && !wait_or_abort(&s.empty[stage], (use - 1) & 1, s.abort, p.ws, DOWN ? 7 : 5)) go = 0;
+                        if (go) mbar_arrive_expect_tx(&s.full[stage], (uint32_t)(rows_in_stage * units * 16));
+                    }
+                    go = __shfl_sync(0xffffffffu, go, 0);
+                    if (!go) {
+                        ok = false;
+                        break;
+                    }
+                    if (mine)
+                        bulk_g2s(s.stages + (size_t)stage * pl.stage_bytes + (size_t)lane * chunk_bytes_max,
+                                 mat + (size_t)grow * row_bytes + (size_t)c * chunk_bytes_max, (uint32_t)units * 16,
+                                 &s.full[stage]);
+                }
+            }
+        }
+        if (lane == 0) producer_drain_mma(s, pl.n_stages, it);
+        return;
+    }
+
+    // ---- consumers
+    pdl_wait_prior_grids();  // x / z and the outputs belong to earlier work on the stream
+    const int g = lane >> 2, t = lane & 3;
+    const int my_pair = warp / wpn, q = warp - my_pair * wpn;
+    // the scratch holds, per sequence, z_hi [ldk] then z_lo [ldk] in bf16 (same bytes as fp32 [ldk])
+    __nv_bfloat16 *zbits = reinterpret_cast<__nv_bfloat16 *>(p.z);
+    uint32_t it = 0;
+    int item_parity = 0, cur_b = -1;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, item_parity ^= 1) {
+        const int b = item / p.n_slices, sl = item - b * p.n_slices;
+        const int r0 = (int)((long long)sl * total_rows / p.n_slices);
+        const int r1 = (int)((long long)(sl + 1) * total_rows / p.n_slices);
+        const int n_pairs = DOWN ? (r1 - r0 + 1) / 2 : r1 - r0;
+        float2 *part = s.part + item_parity * (DEC_MAX_ROWS * DEC_CONSUMER_WARPS);
+        if (b != cur_b) {  // stage this sequence's vector in shared memory
+            if (cur_b >= 0) consumer_barrier();  // nobody still reads the previous one
+            if (!DOWN) {
+                const uint4 *src =
+                    reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(p.x) + (size_t)b * p.d);
+                for (int v = tid; v < pl.row_units; v += DEC_CONSUMERS) reinterpret_cast<uint4 *>(s.vec)[v] = src[v];
+            } else {  // z_hi [ldk] then z_lo [ldk], as gate_up left them
+                const uint4 *src = reinterpret_cast<const uint4 *>(zbits + (size_t)b * 2 * p.ldk);
+                for (int v = tid; v < 2 * pl.row_units; v += DEC_CONSUMERS) reinterpret_cast<uint4 *>(s.vec)[v] = src[v];
+            }
+            consumer_barrier();
+            cur_b = b;
+        }
+        const uint4 *vec0 = reinterpret_cast<const uint4 *>(s.vec);
+        const uint4 *vec1 = vec0 + pl.row_units;  // z_lo (down only)
+        bool ok = true;
+        for (int pg = 0; ok && pg < n_pairs; pg += pl.R) {
+            const bool have = pg + my_pair < n_pairs;
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int c = 0; c < pl.n_chunks; ++c, ++it) {
+                const int stage = it % pl.n_stages;
+                if (!wait_or_abort(&s.full[stage], (it / pl.n_stages) & 1, s.abort, p.ws, DOWN ? 8 : 6)) {
+                    ok = false;
+                    break;
+                }
+                if (have) {
+                    const int units = min(pl.chunk_units, pl.row_units - c * pl.chunk_units);
+                    const uint4 *row0 = reinterpret_cast<const uint4 *>(s.stages + (size_t)stage * pl.stage_bytes +
+                                                                        (size_t)(2 * my_pair) * chunk_bytes_max);
+                    const uint4 *row1 = row0 + pl.chunk_units;
+                    pair_mma<DOWN>(acc, row0, row1, vec0 + c * pl.chunk_units, vec1 + c * pl.chunk_units, units, q, wpn,
+                                   lane);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&s.empty[stage]);
+            }
+            if (ok && have) {
+                const float2 d2 = diagonal_sum(acc, g, t);
+                if (lane == 0) part[(pg + my_pair) * DEC_CONSUMER_WARPS + q] = d2;
+            }
+        }
+        consumer_barrier();
+        if (!ok || *s.abort) break;
+        if (tid < r1 - r0) {
+            const int pair = DOWN ? tid >> 1 : tid;
+            float a0 = 0.f, a1 = 0.f;
+            for (int w = 0; w < wpn; ++w) {
+                const float2 v = part[pair * DEC_CONSUMER_WARPS + w];
+                a0 += v.x;
+                a1 += v.y;
+            }
+            if (!DOWN) {
+                const int j = r0 + tid;
+                if (p.seq[b].b_gate) a0 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[b].b_gate)[j]);
+                if (p.seq[b].b_up) a1 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[b].b_up)[j]);
+                // z leaves as two bf16 numbers, z_hi + z_lo, ready to be the down kernel's vector
+                const float zv = sigma_rt(act, a0) * a1;
+                const __nv_bfloat16 h = __float2bfloat16_rn(zv);
+                zbits[(size_t)b * 2 * p.ldk + j] = h;
+                zbits[(size_t)b * 2 * p.ldk + p.ldk + j] = __float2bfloat16_rn(zv - __bfloat162float(h));
+            } else {
+                const int c = r0 + tid;
+                float acc = (tid & 1) ? a1 : a0;
+                if (p.b_down) acc += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.b_down)[c]);
+                static_cast<__nv_bfloat16 *>(p.y)[(size_t)b * p.d + c] = __float2bfloat16_rn(acc);
+            }
+        }
+        if (!DOWN) {  // the last slice also clears the padding of z (at most 7 entries)
+            const int pad = tid - (DEC_CONSUMERS - 8);
+            if (sl == p.n_slices - 1 && pad >= 0 && p.k + pad < p.ldk) {
+                zbits[(size_t)b * 2 * p.ldk + p.k + pad] = __float2bfloat16_rn(0.f);
+                zbits[(size_t)b * 2 * p.ldk + p.ldk + p.k + pad] = __float2bfloat16_rn(0.f);
+            }
+        }
+    }
+}
+
+template <bool DOWN>
+static griffin_status launch_one(DecodeParams &p, const MmaPlan &pl, int act, int sms, bool overlap,
+                                 cudaStream_t stream) {
+    const int rows = DOWN ? p.d : p.k;
+    // an item holds at most DEC_MAX_ROWS pairs' worth of partial sums
+    p.n_slices = slices_for(rows, sms);
+    const int grid = min(sms, p.B * p.n_slices);
+    const size_t smem = (size_t)pl.n_stages * pl.stage_bytes + pl.vec_bytes + mma_fixed_smem(pl.n_stages);
+    if (smem > 227 * 1024) return GRIFFIN_ERR_UNSUPPORTED;
+    const void *fn = (const void *)decode_mma_kernel<DOWN>;
+    if (ensure_dynamic_smem(fn, smem) != cudaSuccess) return GRIFFIN_ERR_CUDA;
+    MmaPlan plan = pl;
+    void *args[] = {&p, &plan, &act};
+    if (launch_maybe_overlapped(fn, dim3(grid), dim3(DEC_THREADS), smem, stream, overlap, args) != cudaSuccess)
+        return GRIFFIN_ERR_CUDA;
+    return GRIFFIN_OK;
+}
+
+griffin_status decode_bf16_mma(DecodeParams &p, int act, uint32_t flags, cudaStream_t stream) {
+    const int sms = device_sm_count();
+    if (sms <= 0) return GRIFFIN_ERR_CUDA;
+    const bool overlap = (flags & GRIFFIN_DECODE_OVERLAP_WEIGHT_PREFETCH) != 0;
+    const MmaPlan gu = make_plan(p.d, p.d * 2);
+    griffin_status st = launch_one<false>(p, gu, act, sms, overlap, stream);
+    if (st != GRIFFIN_OK) return st;
+    // down may always start early: gate_up never writes weights
+    const MmaPlan dn = make_plan(p.ldk, p.ldk * 4);
+    return launch_one<true>(p, dn, act, sms, true, stream);
+}
+
+}  // namespace griffin
