@@ -173,6 +173,34 @@ griffin_status griffin_ff_decode(const griffin_ff_desc *desc, int32_t B,
                                  const void *x, void *y, void *workspace, size_t ws_bytes,
                                  uint32_t flags, void *stream);
 
+/* The paper has no counterpart to this call: it is griffin_ff_decode for callers that have
+ * no device memory to give as a workspace and may not allocate any.  That is the situation
+ * of code that lives inside somebody else's process under a fixed memory budget (an
+ * inference server that hands a plug-in its inputs and outputs and nothing else), and of
+ * latency-critical loops that must stay clear of cudaMalloc / cudaFree because those calls
+ * take the allocator's lock and synchronise the whole device.
+ *
+ * Same arguments, same kernels and same results as griffin_ff_decode, minus the workspace:
+ * the activations z_hat go through an array that is part of the library image itself
+ * (GRIFFIN_STATIC_SCRATCH_BYTES of device memory on every GPU that loads the library, held
+ * until the process exits).  The call allocates and frees nothing.
+ *   - Limit: B * ldk * 4 bytes must fit in GRIFFIN_STATIC_SCRATCH_BYTES, otherwise
+ *     GRIFFIN_ERR_UNSUPPORTED is returned and nothing is enqueued (B = 8 sequences of up to
+ *     32768 experts fit; use griffin_ff_decode with a workspace beyond that).
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  It keeps whatever the previous call left
+ *     there; nothing in it needs to start at zero, because every entry the second kernel
+ *     reads has been written by the first kernel of the same call.  Two calls that overlap
+ *     on the GPU (different streams) race on it: keep calls on one device ordered.
+ *   - There is no status word: should a bounded wait inside a kernel give up, the call's
+ *     output is incomplete and nothing reports it.  Callers that need that report use
+ *     griffin_ff_decode. */
+#define GRIFFIN_STATIC_SCRATCH_BYTES (1u << 20)
+griffin_status griffin_ff_decode_static(const griffin_ff_desc *desc, int32_t B,
+                                        const griffin_ff_compact *sets /*host*/, const void *b_down,
+                                        const void *x, void *y, uint32_t flags, void *stream);
+
 /* Synchronises `stream`, then reads the workspace's device status word.  GRIFFIN_OK,
  * GRIFFIN_ERR_TIMEOUT (a bounded wait inside a kernel gave up), GRIFFIN_ERR_INVALID_ARG
  * (a kernel met an out-of-range expert index) or GRIFFIN_ERR_CUDA. */

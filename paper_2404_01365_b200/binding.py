@@ -27,6 +27,7 @@ EXPORTS = (
     "griffin_status_string", "griffin_version", "griffin_k_from_keep_ratio", "griffin_compact_ldk",
     "griffin_workspace_bytes", "griffin_workspace_init", "griffin_ff_prefill_score", "griffin_select_topk",
     "griffin_combine_scores", "griffin_compact_experts", "griffin_ff_decode", "griffin_check_device_status",
+    "griffin_ff_decode_static",
 )
 
 
@@ -85,6 +86,8 @@ def load(path=None):
     lib.griffin_compact_experts.argtypes = [C.POINTER(FFDesc), C.POINTER(FFWeights), vp, C.POINTER(FFCompact), vp, vp]
     lib.griffin_ff_decode.restype = C.c_int
     lib.griffin_ff_decode.argtypes = [C.POINTER(FFDesc), i32, C.POINTER(FFCompact), vp, vp, vp, vp, sz, u32, vp]
+    lib.griffin_ff_decode_static.restype = C.c_int
+    lib.griffin_ff_decode_static.argtypes = [C.POINTER(FFDesc), i32, C.POINTER(FFCompact), vp, vp, vp, u32, vp]
     lib.griffin_check_device_status.restype = C.c_int
     lib.griffin_check_device_status.argtypes = [vp, vp]
     _lib = lib
@@ -206,6 +209,17 @@ def griffin_ff_decode(desc, sets, b_down, x, y, ws, flags=DECODE_DEFAULT, stream
     arr = sets if isinstance(sets, C.Array) else compact_array(sets)
     _check(load().griffin_ff_decode(C.byref(desc), len(arr), arr, _ptr(b_down), _ptr(x), _ptr(y), _ptr(ws),
                                     ws.numel(), int(flags), _stream(stream)), "griffin_ff_decode")
+
+
+STATIC_SCRATCH_BYTES = 1 << 20
+
+
+def griffin_ff_decode_static(desc, sets, b_down, x, y, flags=DECODE_DEFAULT, stream=None):
+    """griffin_ff_decode for callers that cannot allocate a workspace: the scratch is a fixed
+    array inside the library (see include/griffin_ff.h for its limit and sharing rules)."""
+    arr = sets if isinstance(sets, C.Array) else compact_array(sets)
+    _check(load().griffin_ff_decode_static(C.byref(desc), len(arr), arr, _ptr(b_down), _ptr(x), _ptr(y), int(flags),
+                                           _stream(stream)), "griffin_ff_decode_static")
 
 
 def griffin_check_device_status(ws, stream=None):

@@ -186,6 +186,24 @@ griffin_status griffin_ff_decode(const griffin_ff_desc *desc, int32_t B, const g
     return launch_decode(desc, B, sets, b_down, x, y, z, workspace, flags, static_cast<cudaStream_t>(stream));
 }
 
+griffin_status griffin_ff_decode_static(const griffin_ff_desc *desc, int32_t B, const griffin_ff_compact *sets,
+                                        const void *b_down, const void *x, void *y, uint32_t flags, void *stream) {
+    griffin_status st = check_desc(desc);
+    if (st != GRIFFIN_OK) return st;
+    if (sets == nullptr || x == nullptr || y == nullptr) return GRIFFIN_ERR_INVALID_ARG;
+    if (B < 1) return GRIFFIN_ERR_INVALID_ARG;
+    if (B > GRIFFIN_MAX_BATCH || desc->d > GRIFFIN_MAX_D) return GRIFFIN_ERR_UNSUPPORTED;
+    if (flags & ~GRIFFIN_DECODE_OVERLAP_WEIGHT_PREFETCH) return GRIFFIN_ERR_INVALID_ARG;
+    for (int b = 0; b < B; ++b) {
+        st = check_compact(desc, &sets[b]);
+        if (st != GRIFFIN_OK) return st;
+        if (sets[b].k != sets[0].k || sets[b].ldk != sets[0].ldk) return GRIFFIN_ERR_INVALID_ARG;
+    }
+    if (!aligned16(x) || !aligned16(y)) return GRIFFIN_ERR_ALIGNMENT;
+    // the size check against GRIFFIN_STATIC_SCRATCH_BYTES happens in the launcher, before any CUDA call
+    return launch_decode_static(desc, B, sets, b_down, x, y, flags, static_cast<cudaStream_t>(stream));
+}
+
 griffin_status griffin_check_device_status(const void *workspace, void *stream) {
     if (workspace == nullptr) return GRIFFIN_ERR_WORKSPACE;
     WsHeader h;

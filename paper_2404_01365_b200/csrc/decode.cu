@@ -403,4 +403,34 @@ griffin_status launch_decode(const griffin_ff_desc *desc, int B, const griffin_f
     return decode_bf16_mma(p, desc->act, flags, stream);
 }
 
+// ---------------------------------------------------------------------------------------
+// Decode without a caller-provided workspace: z lives in a static device array that is part
+// of this library's image (one copy per GPU that loads it).  In host code the array's name
+// is only a stand-in; the address a kernel may use comes from cudaGetSymbolAddress, asked
+// once per device with that device current.
+// ---------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_decode_scratch[GRIFFIN_STATIC_SCRATCH_BYTES];
+
+static float *static_scratch_of_current_device() {
+    static float *addr[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (addr[dev] == nullptr) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_decode_scratch) != cudaSuccess) return nullptr;
+        addr[dev] = static_cast<float *>(p);
+    }
+    return addr[dev];
+}
+
+griffin_status launch_decode_static(const griffin_ff_desc *desc, int B, const griffin_ff_compact *sets,
+                                    const void *b_down, const void *x, void *y, uint32_t flags, cudaStream_t stream) {
+    if ((size_t)B * (size_t)sets[0].ldk * sizeof(float) > (size_t)GRIFFIN_STATIC_SCRATCH_BYTES)
+        return GRIFFIN_ERR_UNSUPPORTED;
+    float *z = static_scratch_of_current_device();
+    if (z == nullptr) return GRIFFIN_ERR_CUDA;
+    // same launcher as the workspace variant; no status word (ws = null)
+    return launch_decode(desc, B, sets, b_down, x, y, z, nullptr, flags, stream);
+}
+
 }  // namespace griffin

@@ -19,6 +19,10 @@ cudaError_t ensure_dynamic_smem(const void *fn, size_t bytes);
 griffin_status launch_decode(const griffin_ff_desc *desc, int B, const griffin_ff_compact *sets, const void *b_down,
                              const void *x, void *y, float *z, void *ws, uint32_t flags, cudaStream_t stream);
 
+// Decode with the z scratch in the library's own static device array (no workspace).
+griffin_status launch_decode_static(const griffin_ff_desc *desc, int B, const griffin_ff_compact *sets,
+                                    const void *b_down, const void *x, void *y, uint32_t flags, cudaStream_t stream);
+
 griffin_status launch_select_topk(const float *score, int n_seq, int d_ff, int k, int32_t *idx, cudaStream_t stream);
 
 griffin_status launch_combine_scores(const float *score, const int32_t *prompt_len_host, int n_seq, int d_ff,
