@@ -1,0 +1,114 @@
+"""End-to-end parity of the whole path (prompt FF + statistic -> top-k -> compaction -> decode)
+against the CPU oracle, driven through the same runner and launch configuration bench.py
+times (decode calls with overlapped weight prefetch after the first step).
+
+Small versions of every workload are checked in full; the full-size workloads are checked on
+one block each (first, middle or last), all prompt rows, and decode steps {0, 1, T/2, T-1}.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import griffin_oracle as O
+from paper_2404_01365_b200 import binding as G, synth
+from paper_2404_01365_b200.runner import FFStack
+from gpu_util import TOL_OUT, check_expert_set, dev, np64, rel_l2, score_tol
+
+pytestmark = pytest.mark.gpu
+
+
+def run_block(w, layer, keep, n_seq, oracle_seqs, steps):
+    """One block of workload `w`: n_seq sequences on the GPU; the oracle follows the sequences
+    in `oracle_seqs` through the prompt phase, and every sequence through the decode steps
+    (with the expert set the GPU selected, so that decode is judged on its own)."""
+    k = G.griffin_k_from_keep_ratio(w.d_ff, keep)
+    assert k == O.k_from_keep_ratio(w.d_ff, keep)
+    wg, wu, wd = synth.make_weights(w, layer)
+    stack = FFStack(w.d, w.d_ff, w.act, w.dtype, 1, n_seq, w.S, k, dev())
+    stack.add_block(wg.to(dev()), wu.to(dev()), wd.to(dev()))
+    X = [synth.make_prompt(w, layer, q) for q in range(n_seq)]
+    XD = torch.stack([synth.make_decode_inputs(w, layer, q) for q in range(n_seq)], 1)  # [T, n_seq, d]
+    Y = torch.empty((n_seq, w.S, w.d), device=dev(), dtype=w.torch_dtype)
+    for q in range(n_seq):
+        stack.prefill_score(0, q, X[q].to(dev()), Y[q])
+    stack.select_all()
+    for q in range(n_seq):
+        stack.compact(0, q)
+    xd_dev = XD.to(dev())
+    yd = torch.empty_like(xd_dev)
+    for t in range(w.T):
+        stack.decode(0, xd_dev[t], yd[t], overlap=t > 0)
+    assert stack.status() == G.OK
+    E = stack.idx[0].cpu().numpy()
+    S_gpu = np64(stack.score[0])
+
+    wg64, wu64, wd64 = np64(wg), np64(wu), np64(wd)
+    swaps = 0
+    for q in oracle_seqs:
+        y_ref, z_ref = O.ff_dense(np64(X[q]), wg64, wu64, wd64, w.act)
+        s_ref = O.flock_score(z_ref)
+        assert rel_l2(np64(Y[q]), y_ref) < TOL_OUT[w.dtype], ("prefill output", q)
+        tol = score_tol(w.dtype)
+        assert np.all(np.abs(S_gpu[q] - s_ref) <= tol * s_ref + 1e-6 * np.sqrt(w.S / w.d_ff)), ("statistic", q)
+        assert abs(float(np.sum(S_gpu[q] ** 2)) - w.S) < 1e-4 * w.S
+        swaps += check_expert_set(E[q], s_ref, k)
+    for q in range(n_seq):
+        assert np.all(np.diff(E[q]) > 0) and E[q].min() >= 0 and E[q].max() < w.d_ff
+        c = O.compact_experts(E[q], wg64, wu64, wd64)
+        for t in steps:
+            ref = O.ff_pruned(np64(XD[t, q]), c, w.act)
+            assert rel_l2(np64(yd[t, q]), ref) < TOL_OUT[w.dtype], ("decode", q, t)
+    if n_seq > 1 and k < w.d_ff:   # each sequence picked its own experts
+        assert any(not np.array_equal(E[0], E[q]) for q in range(1, n_seq))
+    return swaps
+
+
+def test_tiny_workload_in_full():
+    w = synth.WORKLOADS["tiny_swiglu_f32"]
+    swaps = run_block(w, 0, 0.5, 1, [0], range(w.T))
+    assert swaps == 0      # fp32 end to end: the expert set is the oracle's
+
+
+SMALL = {
+    "llama2_7b": dict(d=512, d_ff=1376, S=96, T=6),
+    "gemma_7b": dict(d=384, d_ff=3072, S=128, T=6),
+    "llama2_13b": dict(d=640, d_ff=1728, S=160, T=4),
+    "mistral_7b": dict(d=512, d_ff=1792, S=200, T=4),
+}
+
+
+@pytest.mark.parametrize("name", list(SMALL))
+def test_small_versions_of_every_workload(name):
+    base = synth.WORKLOADS[name]
+    w = synth.scaled(base, **SMALL[name])
+    for keep in base.keeps:
+        for layer in (0, base.L - 1):
+            run_block(w, layer, keep, base.B, range(base.B), range(w.T))
+
+
+def _steps(T):
+    return sorted({0, 1, T // 2, T - 1})
+
+
+def test_full_size_llama2_7b_blocks():
+    w = synth.WORKLOADS["llama2_7b"]
+    for layer in (0, w.L // 2, w.L - 1):
+        run_block(w, layer, 0.5, 1, [0], _steps(w.T))
+
+
+def test_full_size_gemma_7b_block():
+    w = synth.WORKLOADS["gemma_7b"]
+    run_block(w, w.L - 1, 0.5, 1, [0], _steps(w.T))
+
+
+def test_full_size_llama2_13b_block_batch8():
+    w = synth.WORKLOADS["llama2_13b"]
+    # 8 sequences with 8 distinct expert sets decoded together; the oracle follows the prompt
+    # phase of two of them (0.87 TFLOP of fp64 each) and the decode of all eight
+    run_block(w, w.L // 2, 0.5, w.B, [0, w.B - 1], _steps(w.T))
+
+
+@pytest.mark.parametrize("keep", [0.25, 0.5, 0.75, 1.0])
+def test_full_size_mistral_7b_block_keep_sweep(keep):
+    w = synth.WORKLOADS["mistral_7b"]
+    run_block(w, 0, keep, w.B, [0] if keep != 0.5 else [0, 3], _steps(w.T))
