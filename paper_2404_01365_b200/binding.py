@@ -58,7 +58,7 @@ def load(path=None):
     global _lib
     if _lib is not None:
         return _lib
-    path = path or _build.LIB_PATH
+    path = path or os.environ.get("GRIFFIN_FF_LIB") or _build.LIB_PATH
     if not os.path.exists(path):
         raise RuntimeError(f"{path} is missing: build it with `python -m paper_2404_01365_b200.build` "
                            "(there is no fallback path)")

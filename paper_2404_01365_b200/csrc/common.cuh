@@ -20,8 +20,10 @@ constexpr int DEV_STATUS_TIMEOUT = 1;    // a bounded wait gave up
 constexpr int DEV_STATUS_BAD_INDEX = 2;  // an expert index outside [0, d_ff)
 
 struct WsHeader {
-    int status;  // DEV_STATUS_*
-    int detail;  // where it happened (kernel-specific code)
+    int status;           // DEV_STATUS_*
+    int detail;           // where it happened (kernel-specific code)
+    unsigned int arrive;  // grid barrier of the fused decode kernel: CTAs that finished the first half
+    unsigned int depart;  // ... and CTAs that have seen everybody arrive (the last one resets both)
 };
 
 __device__ __forceinline__ void raise_status(void *ws, int status, int detail) {

@@ -409,16 +409,17 @@ griffin_status launch_decode(const griffin_ff_desc *desc, int B, const griffin_f
 // is only a stand-in; the address a kernel may use comes from cudaGetSymbolAddress, asked
 // once per device with that device current.
 // ---------------------------------------------------------------------------------------
-static __device__ __align__(256) unsigned char g_static_decode_scratch[GRIFFIN_STATIC_SCRATCH_BYTES];
+// 256 bytes of header (what a workspace starts with; zero at load time and self-cleaning) + the scratch proper
+static __device__ __align__(256) unsigned char g_static_decode_scratch[256 + GRIFFIN_STATIC_SCRATCH_BYTES];
 
-static float *static_scratch_of_current_device() {
-    static float *addr[64] = {nullptr};
+static unsigned char *static_scratch_of_current_device() {
+    static unsigned char *addr[64] = {nullptr};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
     if (addr[dev] == nullptr) {
         void *p = nullptr;
         if (cudaGetSymbolAddress(&p, g_static_decode_scratch) != cudaSuccess) return nullptr;
-        addr[dev] = static_cast<float *>(p);
+        addr[dev] = static_cast<unsigned char *>(p);
     }
     return addr[dev];
 }
@@ -427,10 +428,10 @@ griffin_status launch_decode_static(const griffin_ff_desc *desc, int B, const gr
                                     const void *b_down, const void *x, void *y, uint32_t flags, cudaStream_t stream) {
     if ((size_t)B * (size_t)sets[0].ldk * sizeof(float) > (size_t)GRIFFIN_STATIC_SCRATCH_BYTES)
         return GRIFFIN_ERR_UNSUPPORTED;
-    float *z = static_scratch_of_current_device();
-    if (z == nullptr) return GRIFFIN_ERR_CUDA;
-    // same launcher as the workspace variant; no status word (ws = null)
-    return launch_decode(desc, B, sets, b_down, x, y, z, nullptr, flags, stream);
+    unsigned char *base = static_scratch_of_current_device();
+    if (base == nullptr) return GRIFFIN_ERR_CUDA;
+    // same launcher as the workspace variant: header first, z behind it
+    return launch_decode(desc, B, sets, b_down, x, y, reinterpret_cast<float *>(base + 256), base, flags, stream);
 }
 
 }  // namespace griffin

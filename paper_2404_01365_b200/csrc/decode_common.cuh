@@ -25,6 +25,7 @@ struct DecodeParams {
     void *ws;       // workspace header (status word), may be null
     int d, k, ldk, B;
     int n_slices;  // work items per sequence
+    int n_slices_dn;  // fused bf16 kernel: work items per sequence of the down half
     int n_stages;
     int kt_len;    // down kernel: elements per k-tile (multiple of 8)
     int n_ktiles;

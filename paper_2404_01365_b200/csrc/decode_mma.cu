@@ -115,28 +115,40 @@ __device__ __forceinline__ float2 diagonal_sum(const float (&c)[4], int g, int t
     return make_float2(v0, v1);
 }
 
-// This warp's share of one pair's chunk: blocks q, q + wpn, ... of 32 units each.
+// This warp's share of one pair's chunk: blocks q, q + wpn, ... of 32 units each, never more
+// than MMA_BLOCKS_PER_WARP of them (a stage holds at most 32 / R blocks per row and 8 / R warps
+// share the pair).  All shared-memory reads are issued before the first MMA and the MMAs go
+// to four independent accumulators, so the latencies overlap instead of adding up: measured,
+// the serial version spent about 200 cycles per block and made the consumers, not HBM, the
+// bottleneck.
 //   row0,row1 : the two staged rows; vec0 : vector units for this chunk; vec1 : second vector
 //   (down's z_lo); n_units : valid units in this chunk
+constexpr int MMA_BLOCKS_PER_WARP = 4;
 template <bool TWO_VECTORS>
-__device__ __forceinline__ void pair_mma(float (&acc)[4], const uint4 *row0, const uint4 *row1, const uint4 *vec0,
+__device__ __forceinline__ void pair_mma(float (&acc)[4][4], const uint4 *row0, const uint4 *row1, const uint4 *vec0,
                                          const uint4 *vec1, int n_units, int q, int wpn, int lane) {
     const uint4 zero = make_uint4(0, 0, 0, 0);
-#pragma unroll 2
-    for (int b = q; b * 32 < n_units; b += wpn) {
-        const int u = b * 32 + lane;  // a warp reads 512 contiguous bytes
-        uint4 r0 = zero, r1 = zero, v = zero, w = zero;
+    uint4 r0[MMA_BLOCKS_PER_WARP], r1[MMA_BLOCKS_PER_WARP], v[MMA_BLOCKS_PER_WARP], w[MMA_BLOCKS_PER_WARP];
+#pragma unroll
+    for (int i = 0; i < MMA_BLOCKS_PER_WARP; ++i) {
+        const int u = (q + i * wpn) * 32 + lane;  // a warp reads 512 contiguous bytes
+        r0[i] = zero; r1[i] = zero; v[i] = zero; w[i] = zero;
         if (u < n_units) {  // past the end both operands are zero (stale bytes could be NaN)
-            r0 = row0[u];
-            r1 = row1[u];
-            v = vec0[u];
-            if (TWO_VECTORS) w = vec1[u];
+            r0[i] = row0[u];
+            r1[i] = row1[u];
+            v[i] = vec0[u];
+            if (TWO_VECTORS) w[i] = vec1[u];
         }
-        mma_bf16(acc, r0.x, r1.x, r0.y, r1.y, v.x, v.y);
-        mma_bf16(acc, r0.z, r1.z, r0.w, r1.w, v.z, v.w);
-        if (TWO_VECTORS) {
-            mma_bf16(acc, r0.x, r1.x, r0.y, r1.y, w.x, w.y);
-            mma_bf16(acc, r0.z, r1.z, r0.w, r1.w, w.z, w.w);
+    }
+#pragma unroll
+    for (int i = 0; i < MMA_BLOCKS_PER_WARP; ++i) {
+        if ((q + i * wpn) * 32 < n_units) {  // warp-uniform
+            mma_bf16(acc[(2 * i) & 3], r0[i].x, r1[i].x, r0[i].y, r1[i].y, v[i].x, v[i].y);
+            mma_bf16(acc[(2 * i + 1) & 3], r0[i].z, r1[i].z, r0[i].w, r1[i].w, v[i].z, v[i].w);
+            if (TWO_VECTORS) {
+                mma_bf16(acc[(2 * i) & 3], r0[i].x, r1[i].x, r0[i].y, r1[i].y, w[i].x, w[i].y);
+                mma_bf16(acc[(2 * i + 1) & 3], r0[i].z, r1[i].z, r0[i].w, r1[i].w, w[i].z, w[i].w);
+            }
         }
     }
 }
@@ -153,89 +165,90 @@ __device__ __forceinline__ void producer_drain_mma(const MmaSmem &s, int n_stage
     }
 }
 
-// DOWN = false: gate_up, z[b, j] = sigma(gate_j . x + b_gate_j) * (up_j . x + b_up_j);
-//               item = (sequence, slice of neurons), pair = neuron.
-// DOWN = true : down, y[b, c] = w_down_c[c, :] . z[b] + b_down[c];
-//               item = (sequence, chunk of output rows), pair = two consecutive rows.
-template <bool DOWN>
-__global__ void __launch_bounds__(DEC_THREADS) decode_mma_kernel(const __grid_constant__ DecodeParams p,
-                                                                 const __grid_constant__ MmaPlan pl, int act) {
-    extern __shared__ __align__(128) uint8_t smem_raw[];
-    const MmaSmem s = carve_mma(smem_raw, pl);
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (tid == 0) {
-        for (int i = 0; i < pl.n_stages; ++i) {
-            mbar_init(&s.full[i], 1);
-            mbar_init(&s.empty[i], DEC_CONSUMER_WARPS);
-        }
-        *s.abort = 0;
-        mbar_fence_init();
-    }
-    __syncthreads();
-    pdl_launch_dependents();
+// The two halves of a decode call share one kernel, one ring and one stage counter:
+//   DOWN = false: gate_up, z[b, j] = sigma(gate_j . x + b_gate_j) * (up_j . x + b_up_j);
+//                 item = (sequence, slice of neurons), pair = neuron.
+//   DOWN = true : down, y[b, c] = w_down_c[c, :] . z[b] + b_down[c];
+//                 item = (sequence, chunk of output rows), pair = two consecutive rows.
+struct FusedPlan {
+    MmaPlan gu, dn;   // per-half geometry (their n_stages / stage_bytes are overridden below)
+    int slot_bytes;   // ring slot = the larger of the two halves' stages
+    int n_stages;
+    int vec_bytes;    // the larger of x (d * 2) and z_hi | z_lo (ldk * 4)
+};
 
-    const int n_items = p.B * p.n_slices;
-    const int total_rows = DOWN ? p.d : p.k;  // what the slices partition
+__device__ __forceinline__ MmaSmem carve_fused(uint8_t *smem, const FusedPlan &fp) {
+    MmaSmem s;
+    s.stages = smem;
+    s.vec = smem + (size_t)fp.n_stages * fp.slot_bytes;
+    s.full = reinterpret_cast<uint64_t *>(s.vec + fp.vec_bytes);
+    s.empty = s.full + fp.n_stages;
+    s.part = reinterpret_cast<float2 *>(s.empty + fp.n_stages);
+    s.abort = reinterpret_cast<volatile int *>(s.part + 2 * DEC_MAX_ROWS * DEC_CONSUMER_WARPS);
+    return s;
+}
+
+// Producer side of one half.  Lane l < 2R copies row (l & 1) of pair (l >> 1).  Weights only.
+template <bool DOWN>
+__device__ __forceinline__ bool produce_half(const DecodeParams &p, const MmaPlan &pl, const MmaSmem &s, int n_stages,
+                                             int slot_bytes, int n_slices, uint32_t &it, int lane) {
+    const int n_items = p.B * n_slices;
+    const int total_rows = DOWN ? p.d : p.k;
     const size_t row_bytes = (size_t)pl.row_units * 16;
     const int chunk_bytes_max = pl.chunk_units * 16;
-    const int wpn = DEC_CONSUMER_WARPS / pl.R;  // warps per pair
-
-    if (warp == DEC_CONSUMER_WARPS) {
-        // ---- producer warp: weights only, never waits for the previous grid.  Lane l < 2R
-        //      copies row (l & 1) of pair (l >> 1).
-        uint32_t it = 0;
-        bool ok = true;
-        const int my_pair = lane >> 1, my_row = lane & 1;
-        for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
-            const int b = item / p.n_slices, sl = item - b * p.n_slices;
-            const int r0 = (int)((long long)sl * total_rows / p.n_slices);
-            const int r1 = (int)((long long)(sl + 1) * total_rows / p.n_slices);
-            const int n_pairs = DOWN ? (r1 - r0 + 1) / 2 : r1 - r0;
-            const uint8_t *mat = static_cast<const uint8_t *>(DOWN ? p.seq[b].w_down
-                                                                   : (my_row ? p.seq[b].w_up : p.seq[b].w_gate));
-            for (int pg = 0; ok && pg < n_pairs; pg += pl.R) {
-                const int pair = pg + my_pair;
-                const int grow = DOWN ? r0 + 2 * pair + my_row : r0 + pair;  // row in the matrix
-                const bool mine = lane < 2 * pl.R && pair < n_pairs && grow < r1;
-                // rows copied in this stage (the same for every chunk of the group)
-                const int rows_in_stage = DOWN ? min(2 * pl.R, r1 - r0 - 2 * pg) : 2 * min(pl.R, n_pairs - pg);
-                for (int c = 0; c < pl.n_chunks; ++c, ++it) {
-                    const int units = min(pl.chunk_units, pl.row_units - c * pl.chunk_units);
-                    const int stage = it % pl.n_stages;
-                    const uint32_t use = it / pl.n_stages;
-                    int go = 1;
-                    if (lane == 0) {
-                        if (use > 0 && !wait_or_abort(&s.empty[stage], (use - 1) & 1, s.abort, p.ws, DOWN ? 7 : 5)) go = 0;
-                        if (go) mbar_arrive_expect_tx(&s.full[stage], (uint32_t)(rows_in_stage * units * 16));
-                    }
-                    go = __shfl_sync(0xffffffffu, go, 0);
-                    if (!go) {
-                        ok = false;
-                        break;
-                    }
-                    if (mine)
-                        bulk_g2s(s.stages + (size_t)stage * pl.stage_bytes + (size_t)lane * chunk_bytes_max,
-                                 mat + (size_t)grow * row_bytes + (size_t)c * chunk_bytes_max, (uint32_t)units * 16,
-                                 &s.full[stage]);
+    const int my_pair = lane >> 1, my_row = lane & 1;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+        const int b = item / n_slices, sl = item - b * n_slices;
+        const int r0 = (int)((long long)sl * total_rows / n_slices);
+        const int r1 = (int)((long long)(sl + 1) * total_rows / n_slices);
+        const int n_pairs = DOWN ? (r1 - r0 + 1) / 2 : r1 - r0;
+        const uint8_t *mat =
+            static_cast<const uint8_t *>(DOWN ? p.seq[b].w_down : (my_row ? p.seq[b].w_up : p.seq[b].w_gate));
+        for (int pg = 0; pg < n_pairs; pg += pl.R) {
+            const int pair = pg + my_pair;
+            const int grow = DOWN ? r0 + 2 * pair + my_row : r0 + pair;  // row in the matrix
+            const bool mine = lane < 2 * pl.R && pair < n_pairs && grow < r1;
+            // rows copied in this stage (the same for every chunk of the group)
+            const int rows_in_stage = DOWN ? min(2 * pl.R, r1 - r0 - 2 * pg) : 2 * min(pl.R, n_pairs - pg);
+            for (int c = 0; c < pl.n_chunks; ++c, ++it) {
+                const int units = min(pl.chunk_units, pl.row_units - c * pl.chunk_units);
+                const int stage = it % n_stages;
+                const uint32_t use = it / n_stages;
+                int go = 1;
+                if (lane == 0) {
+                    if (use > 0 && !wait_or_abort(&s.empty[stage], (use - 1) & 1, s.abort, p.ws, DOWN ? 7 : 5)) go = 0;
+                    if (go) mbar_arrive_expect_tx(&s.full[stage], (uint32_t)(rows_in_stage * units * 16));
                 }
+                go = __shfl_sync(0xffffffffu, go, 0);
+                if (!go) return false;
+                if (mine)
+                    bulk_g2s(s.stages + (size_t)stage * slot_bytes + (size_t)lane * chunk_bytes_max,
+                             mat + (size_t)grow * row_bytes + (size_t)c * chunk_bytes_max, (uint32_t)units * 16,
+                             &s.full[stage]);
             }
         }
-        if (lane == 0) producer_drain_mma(s, pl.n_stages, it);
-        return;
     }
+    return true;
+}
 
-    // ---- consumers
-    pdl_wait_prior_grids();  // x / z and the outputs belong to earlier work on the stream
+// Consumer side of one half (all 8 consumer warps).  Returns false after a give-up.
+template <bool DOWN>
+__device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPlan &pl, const MmaSmem &s, int n_stages,
+                                             int slot_bytes, int n_slices, uint32_t &it, int &item_parity, int act,
+                                             int tid, int warp, int lane) {
+    const int n_items = p.B * n_slices;
+    const int total_rows = DOWN ? p.d : p.k;
+    const int chunk_bytes_max = pl.chunk_units * 16;
+    const int wpn = DEC_CONSUMER_WARPS / pl.R;  // warps per pair
     const int g = lane >> 2, t = lane & 3;
     const int my_pair = warp / wpn, q = warp - my_pair * wpn;
     // the scratch holds, per sequence, z_hi [ldk] then z_lo [ldk] in bf16 (same bytes as fp32 [ldk])
     __nv_bfloat16 *zbits = reinterpret_cast<__nv_bfloat16 *>(p.z);
-    uint32_t it = 0;
-    int item_parity = 0, cur_b = -1;
+    int cur_b = -1;
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, item_parity ^= 1) {
-        const int b = item / p.n_slices, sl = item - b * p.n_slices;
-        const int r0 = (int)((long long)sl * total_rows / p.n_slices);
-        const int r1 = (int)((long long)(sl + 1) * total_rows / p.n_slices);
+        const int b = item / n_slices, sl = item - b * n_slices;
+        const int r0 = (int)((long long)sl * total_rows / n_slices);
+        const int r1 = (int)((long long)(sl + 1) * total_rows / n_slices);
         const int n_pairs = DOWN ? (r1 - r0 + 1) / 2 : r1 - r0;
         float2 *part = s.part + item_parity * (DEC_MAX_ROWS * DEC_CONSUMER_WARPS);
         if (b != cur_b) {  // stage this sequence's vector in shared memory
@@ -244,9 +257,10 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_mma_kernel(const __grid_co
                 const uint4 *src =
                     reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(p.x) + (size_t)b * p.d);
                 for (int v = tid; v < pl.row_units; v += DEC_CONSUMERS) reinterpret_cast<uint4 *>(s.vec)[v] = src[v];
-            } else {  // z_hi [ldk] then z_lo [ldk], as gate_up left them
+            } else {  // z_hi [ldk] then z_lo [ldk], written by other CTAs of this grid: read through L2
                 const uint4 *src = reinterpret_cast<const uint4 *>(zbits + (size_t)b * 2 * p.ldk);
-                for (int v = tid; v < 2 * pl.row_units; v += DEC_CONSUMERS) reinterpret_cast<uint4 *>(s.vec)[v] = src[v];
+                for (int v = tid; v < 2 * pl.row_units; v += DEC_CONSUMERS)
+                    reinterpret_cast<uint4 *>(s.vec)[v] = __ldcg(src + v);
             }
             consumer_barrier();
             cur_b = b;
@@ -256,16 +270,16 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_mma_kernel(const __grid_co
         bool ok = true;
         for (int pg = 0; ok && pg < n_pairs; pg += pl.R) {
             const bool have = pg + my_pair < n_pairs;
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+            float acc[4][4] = {};
             for (int c = 0; c < pl.n_chunks; ++c, ++it) {
-                const int stage = it % pl.n_stages;
-                if (!wait_or_abort(&s.full[stage], (it / pl.n_stages) & 1, s.abort, p.ws, DOWN ? 8 : 6)) {
+                const int stage = it % n_stages;
+                if (!wait_or_abort(&s.full[stage], (it / n_stages) & 1, s.abort, p.ws, DOWN ? 8 : 6)) {
                     ok = false;
                     break;
                 }
                 if (have) {
                     const int units = min(pl.chunk_units, pl.row_units - c * pl.chunk_units);
-                    const uint4 *row0 = reinterpret_cast<const uint4 *>(s.stages + (size_t)stage * pl.stage_bytes +
+                    const uint4 *row0 = reinterpret_cast<const uint4 *>(s.stages + (size_t)stage * slot_bytes +
                                                                         (size_t)(2 * my_pair) * chunk_bytes_max);
                     const uint4 *row1 = row0 + pl.chunk_units;
                     pair_mma<DOWN>(acc, row0, row1, vec0 + c * pl.chunk_units, vec1 + c * pl.chunk_units, units, q, wpn,
@@ -275,12 +289,15 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_mma_kernel(const __grid_co
                 if (lane == 0) mbar_arrive(&s.empty[stage]);
             }
             if (ok && have) {
-                const float2 d2 = diagonal_sum(acc, g, t);
+                float sum[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) sum[e] = (acc[0][e] + acc[1][e]) + (acc[2][e] + acc[3][e]);
+                const float2 d2 = diagonal_sum(sum, g, t);
                 if (lane == 0) part[(pg + my_pair) * DEC_CONSUMER_WARPS + q] = d2;
             }
         }
         consumer_barrier();
-        if (!ok || *s.abort) break;
+        if (!ok || *s.abort) return false;
         if (tid < r1 - r0) {
             const int pair = DOWN ? tid >> 1 : tid;
             float a0 = 0.f, a1 = 0.f;
@@ -293,7 +310,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_mma_kernel(const __grid_co
                 const int j = r0 + tid;
                 if (p.seq[b].b_gate) a0 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[b].b_gate)[j]);
                 if (p.seq[b].b_up) a1 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[b].b_up)[j]);
-                // z leaves as two bf16 numbers, z_hi + z_lo, ready to be the down kernel's vector
+                // z leaves as two bf16 numbers, z_hi + z_lo, ready to be the down half's vector
                 const float zv = sigma_rt(act, a0) * a1;
                 const __nv_bfloat16 h = __float2bfloat16_rn(zv);
                 zbits[(size_t)b * 2 * p.ldk + j] = h;
@@ -307,42 +324,107 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_mma_kernel(const __grid_co
         }
         if (!DOWN) {  // the last slice also clears the padding of z (at most 7 entries)
             const int pad = tid - (DEC_CONSUMERS - 8);
-            if (sl == p.n_slices - 1 && pad >= 0 && p.k + pad < p.ldk) {
+            if (sl == n_slices - 1 && pad >= 0 && p.k + pad < p.ldk) {
                 zbits[(size_t)b * 2 * p.ldk + p.k + pad] = __float2bfloat16_rn(0.f);
                 zbits[(size_t)b * 2 * p.ldk + p.ldk + p.k + pad] = __float2bfloat16_rn(0.f);
             }
         }
     }
+    return true;
 }
 
-template <bool DOWN>
-static griffin_status launch_one(DecodeParams &p, const MmaPlan &pl, int act, int sms, bool overlap,
-                                 cudaStream_t stream) {
-    const int rows = DOWN ? p.d : p.k;
-    // an item holds at most DEC_MAX_ROWS pairs' worth of partial sums
-    p.n_slices = slices_for(rows, sms);
-    const int grid = min(sms, p.B * p.n_slices);
-    const size_t smem = (size_t)pl.n_stages * pl.stage_bytes + pl.vec_bytes + mma_fixed_smem(pl.n_stages);
-    if (smem > 227 * 1024) return GRIFFIN_ERR_UNSUPPORTED;
-    const void *fn = (const void *)decode_mma_kernel<DOWN>;
-    if (ensure_dynamic_smem(fn, smem) != cudaSuccess) return GRIFFIN_ERR_CUDA;
-    MmaPlan plan = pl;
-    void *args[] = {&p, &plan, &act};
-    if (launch_maybe_overlapped(fn, dim3(grid), dim3(DEC_THREADS), smem, stream, overlap, args) != cudaSuccess)
-        return GRIFFIN_ERR_CUDA;
-    return GRIFFIN_OK;
+__device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int *p) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Grid-wide meeting point between the two halves, called by one thread per CTA after the
+// CTA's z entries have been written and fenced.  Bounded: gives up after WAIT_LIMIT_CYCLES.
+// The counters clean up after themselves: the last CTA to leave resets both.
+__device__ __forceinline__ bool grid_meet(WsHeader *h, unsigned int n_ctas, volatile int *abort, void *ws) {
+    atomicAdd(&h->arrive, 1u);
+    const long long t0 = clock64();
+    while (ld_acquire_u32(&h->arrive) < n_ctas) {
+        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+            *abort = 1;
+            raise_status(ws, DEV_STATUS_TIMEOUT, 9);
+            return false;
+        }
+    }
+    if (atomicAdd(&h->depart, 1u) == n_ctas - 1) {  // everybody has seen the full count
+        h->depart = 0;
+        h->arrive = 0;
+        __threadfence();
+    }
+    return true;
+}
+
+__global__ void __launch_bounds__(DEC_THREADS) decode_fused_kernel(const __grid_constant__ DecodeParams p,
+                                                                   const __grid_constant__ FusedPlan fp, int act) {
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    const MmaSmem s = carve_fused(smem_raw, fp);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        for (int i = 0; i < fp.n_stages; ++i) {
+            mbar_init(&s.full[i], 1);
+            mbar_init(&s.empty[i], DEC_CONSUMER_WARPS);
+        }
+        *s.abort = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+    pdl_launch_dependents();
+
+    if (warp == DEC_CONSUMER_WARPS) {
+        // ---- producer warp: weights only, so it never waits for the previous grid, nor for
+        //      the meeting point: the first stages of W_2_hat are on their way while the
+        //      consumers are still waiting for the other CTAs' z
+        uint32_t it = 0;
+        if (produce_half<false>(p, fp.gu, s, fp.n_stages, fp.slot_bytes, p.n_slices, it, lane))
+            produce_half<true>(p, fp.dn, s, fp.n_stages, fp.slot_bytes, p.n_slices_dn, it, lane);
+        if (lane == 0) producer_drain_mma(s, fp.n_stages, it);
+        return;
+    }
+
+    // ---- consumers
+    pdl_wait_prior_grids();  // x, the z scratch and the outputs belong to earlier work on the stream
+    uint32_t it = 0;
+    int item_parity = 0;
+    if (!consume_half<false>(p, fp.gu, s, fp.n_stages, fp.slot_bytes, p.n_slices, it, item_parity, act, tid, warp, lane))
+        return;
+    __threadfence();  // this CTA's z entries are visible device-wide before it reports in
+    consumer_barrier();
+    if (tid == 0) grid_meet(static_cast<WsHeader *>(p.ws), gridDim.x, s.abort, p.ws);
+    consumer_barrier();
+    if (*s.abort) return;
+    consume_half<true>(p, fp.dn, s, fp.n_stages, fp.slot_bytes, p.n_slices_dn, it, item_parity, act, tid, warp, lane);
 }
 
 griffin_status decode_bf16_mma(DecodeParams &p, int act, uint32_t flags, cudaStream_t stream) {
     const int sms = device_sm_count();
     if (sms <= 0) return GRIFFIN_ERR_CUDA;
+    if (p.ws == nullptr) return GRIFFIN_ERR_WORKSPACE;  // the meeting point's counters live in the header
     const bool overlap = (flags & GRIFFIN_DECODE_OVERLAP_WEIGHT_PREFETCH) != 0;
-    const MmaPlan gu = make_plan(p.d, p.d * 2);
-    griffin_status st = launch_one<false>(p, gu, act, sms, overlap, stream);
-    if (st != GRIFFIN_OK) return st;
-    // down may always start early: gate_up never writes weights
-    const MmaPlan dn = make_plan(p.ldk, p.ldk * 4);
-    return launch_one<true>(p, dn, act, sms, true, stream);
+    FusedPlan fp;
+    fp.gu = make_plan(p.d, p.d * 2);
+    fp.dn = make_plan(p.ldk, p.ldk * 4);
+    fp.slot_bytes = max(fp.gu.stage_bytes, fp.dn.stage_bytes);
+    fp.vec_bytes = max(p.d * 2, p.ldk * 4);
+    int n = ((int)MMA_SMEM_TARGET - fp.vec_bytes - (int)mma_fixed_smem(8)) / fp.slot_bytes;
+    fp.n_stages = n < 2 ? 2 : (n > 8 ? 8 : n);
+    p.n_slices = slices_for(p.k, sms);
+    p.n_slices_dn = slices_for(p.d, sms);
+    // every CTA of the grid must be able to run at the same time (they meet half-way): one per SM
+    const int grid = sms;
+    const size_t smem = (size_t)fp.n_stages * fp.slot_bytes + fp.vec_bytes + mma_fixed_smem(fp.n_stages);
+    if (smem > 227 * 1024) return GRIFFIN_ERR_UNSUPPORTED;
+    const void *fn = (const void *)decode_fused_kernel;
+    if (ensure_dynamic_smem(fn, smem) != cudaSuccess) return GRIFFIN_ERR_CUDA;
+    void *args[] = {&p, &fp, &act};
+    if (launch_maybe_overlapped(fn, dim3(grid), dim3(DEC_THREADS), smem, stream, overlap, args) != cudaSuccess)
+        return GRIFFIN_ERR_CUDA;
+    return GRIFFIN_OK;
 }
 
 }  // namespace griffin
