@@ -37,12 +37,13 @@
 
 namespace griffin {
 
+constexpr int DEC_GROUP_WARPS = 4;           // consumer warps per group (two groups)
 constexpr int MMA_CHUNK_UNITS_MAX = 1024;  // 16 KB of one row per stage at most
 constexpr int MMA_STAGE_TARGET = 32 * 1024;
 #ifndef GRIFFIN_DEC_SMEM_KB
-#define GRIFFIN_DEC_SMEM_KB 113
+#define GRIFFIN_DEC_SMEM_KB 200
 #endif
-constexpr int MMA_SMEM_TARGET = GRIFFIN_DEC_SMEM_KB * 1024;  // 113 KB = half an SM: the next kernel's CTA fits too
+constexpr int MMA_SMEM_TARGET = GRIFFIN_DEC_SMEM_KB * 1024;  // shared memory the ring, the vector and the rest may take
 
 struct MmaPlan {
     int row_units;    // 16-byte units per real row
@@ -115,53 +116,66 @@ __device__ __forceinline__ float2 diagonal_sum(const float (&c)[4], int g, int t
     return make_float2(v0, v1);
 }
 
-// This warp's share of one pair's chunk: blocks q, q + wpn, ... of 32 units each, never more
-// than MMA_BLOCKS_PER_WARP of them (a stage holds at most 32 / R blocks per row and 8 / R warps
-// share the pair).  All shared-memory reads are issued before the first MMA and the MMAs go
-// to four independent accumulators, so the latencies overlap instead of adding up: measured,
-// the serial version spent about 200 cycles per block and made the consumers, not HBM, the
-// bottleneck.
+// This warp's share of one pair's chunk: blocks q, q + wpg, ... of 32 units each, never more
+// than MMA_BLOCKS_PER_WARP of them (a stage holds at most 32 / R blocks per row and the 4 / R
+// warps of a consumer group share the pair).  They are taken in batches of four: all
+// shared-memory reads of a batch are issued before its first MMA, and the MMAs go to four
+// independent accumulators, so latencies overlap instead of adding up.
 //   row0,row1 : the two staged rows; vec0 : vector units for this chunk; vec1 : second vector
-//   (down's z_lo); n_units : valid units in this chunk
-constexpr int MMA_BLOCKS_PER_WARP = 4;
-template <bool TWO_VECTORS>
+//   (down's z_lo); xr : the vector's units held in registers (gate_up, where x is the same for
+//   every neuron of the item); n_units : valid units in this chunk
+constexpr int MMA_BLOCKS_PER_WARP = 8;
+constexpr int MMA_BATCH = 4;
+template <bool DOWN>
 __device__ __forceinline__ void pair_mma(float (&acc)[4][4], const uint4 *row0, const uint4 *row1, const uint4 *vec0,
-                                         const uint4 *vec1, int n_units, int q, int wpn, int lane) {
+                                         const uint4 *vec1, const uint4 (&xr)[MMA_BLOCKS_PER_WARP], int n_units, int q,
+                                         int wpg, int lane) {
     const uint4 zero = make_uint4(0, 0, 0, 0);
-    uint4 r0[MMA_BLOCKS_PER_WARP], r1[MMA_BLOCKS_PER_WARP], v[MMA_BLOCKS_PER_WARP], w[MMA_BLOCKS_PER_WARP];
 #pragma unroll
-    for (int i = 0; i < MMA_BLOCKS_PER_WARP; ++i) {
-        const int u = (q + i * wpn) * 32 + lane;  // a warp reads 512 contiguous bytes
-        r0[i] = zero; r1[i] = zero; v[i] = zero; w[i] = zero;
-        if (u < n_units) {  // past the end both operands are zero (stale bytes could be NaN)
-            r0[i] = row0[u];
-            r1[i] = row1[u];
-            v[i] = vec0[u];
-            if (TWO_VECTORS) w[i] = vec1[u];
+    for (int b0 = 0; b0 < MMA_BLOCKS_PER_WARP; b0 += MMA_BATCH) {
+        if ((q + b0 * wpg) * 32 >= n_units) break;  // warp-uniform
+        uint4 r0[MMA_BATCH], r1[MMA_BATCH], v[MMA_BATCH], w[MMA_BATCH];
+#pragma unroll
+        for (int i = 0; i < MMA_BATCH; ++i) {
+            const int u = (q + (b0 + i) * wpg) * 32 + lane;  // a warp reads 512 contiguous bytes
+            r0[i] = zero; r1[i] = zero; v[i] = zero; w[i] = zero;
+            if (u < n_units) {  // past the end both operands are zero (stale bytes could be NaN)
+                r0[i] = row0[u];
+                r1[i] = row1[u];
+                if (DOWN) {
+                    v[i] = vec0[u];
+                    w[i] = vec1[u];
+                } else {
+                    v[i] = xr[b0 + i];
+                }
+            }
         }
-    }
 #pragma unroll
-    for (int i = 0; i < MMA_BLOCKS_PER_WARP; ++i) {
-        if ((q + i * wpn) * 32 < n_units) {  // warp-uniform
-            mma_bf16(acc[(2 * i) & 3], r0[i].x, r1[i].x, r0[i].y, r1[i].y, v[i].x, v[i].y);
-            mma_bf16(acc[(2 * i + 1) & 3], r0[i].z, r1[i].z, r0[i].w, r1[i].w, v[i].z, v[i].w);
-            if (TWO_VECTORS) {
-                mma_bf16(acc[(2 * i) & 3], r0[i].x, r1[i].x, r0[i].y, r1[i].y, w[i].x, w[i].y);
-                mma_bf16(acc[(2 * i + 1) & 3], r0[i].z, r1[i].z, r0[i].w, r1[i].w, w[i].z, w[i].w);
+        for (int i = 0; i < MMA_BATCH; ++i) {
+            if ((q + (b0 + i) * wpg) * 32 < n_units) {  // warp-uniform
+                mma_bf16(acc[(2 * i) & 3], r0[i].x, r1[i].x, r0[i].y, r1[i].y, v[i].x, v[i].y);
+                mma_bf16(acc[(2 * i + 1) & 3], r0[i].z, r1[i].z, r0[i].w, r1[i].w, v[i].z, v[i].w);
+                if (DOWN) {
+                    mma_bf16(acc[(2 * i) & 3], r0[i].x, r1[i].x, r0[i].y, r1[i].y, w[i].x, w[i].y);
+                    mma_bf16(acc[(2 * i + 1) & 3], r0[i].z, r1[i].z, r0[i].w, r1[i].w, w[i].z, w[i].w);
+                }
             }
         }
     }
 }
 
-__device__ __forceinline__ void producer_drain_mma(const MmaSmem &s, int n_stages, uint32_t issued) {
-    const uint32_t first = issued > (uint32_t)n_stages ? issued - n_stages : 0;
-    for (uint32_t it = first; it < issued; ++it) {
-        const int stage = it % n_stages;
-        const uint32_t parity = (it / n_stages) & 1;
-        if (mbar_try_wait(&s.full[stage], parity)) continue;
-        const long long t0 = clock64();
-        while (!mbar_try_wait(&s.full[stage], parity))
-            if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
+__device__ __forceinline__ void producer_drain_mma(const MmaSmem &s, int n_stages, const uint32_t (&issued)[2]) {
+    const int ns2 = n_stages >> 1;
+    for (int grp = 0; grp < 2; ++grp) {
+        const uint32_t first = issued[grp] > (uint32_t)ns2 ? issued[grp] - ns2 : 0;
+        for (uint32_t it = first; it < issued[grp]; ++it) {
+            const int stage = grp * ns2 + (int)(it % ns2);
+            const uint32_t parity = (it / ns2) & 1;
+            if (mbar_try_wait(&s.full[stage], parity)) continue;
+            const long long t0 = clock64();
+            while (!mbar_try_wait(&s.full[stage], parity))
+                if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
+        }
     }
 }
 
@@ -191,7 +205,7 @@ __device__ __forceinline__ MmaSmem carve_fused(uint8_t *smem, const FusedPlan &f
 // Producer side of one half.  Lane l < 2R copies row (l & 1) of pair (l >> 1).  Weights only.
 template <bool DOWN>
 __device__ __forceinline__ bool produce_half(const DecodeParams &p, const MmaPlan &pl, const MmaSmem &s, int n_stages,
-                                             int slot_bytes, int n_slices, uint32_t &it, int lane) {
+                                             int slot_bytes, int n_slices, uint32_t (&itg)[2], uint32_t &pgc, int lane) {
     const int n_items = p.B * n_slices;
     const int total_rows = DOWN ? p.d : p.k;
     const size_t row_bytes = (size_t)pl.row_units * 16;
@@ -204,16 +218,22 @@ __device__ __forceinline__ bool produce_half(const DecodeParams &p, const MmaPla
         const int n_pairs = DOWN ? (r1 - r0 + 1) / 2 : r1 - r0;
         const uint8_t *mat =
             static_cast<const uint8_t *>(DOWN ? p.seq[b].w_down : (my_row ? p.seq[b].w_up : p.seq[b].w_gate));
-        for (int pg = 0; pg < n_pairs; pg += pl.R) {
+        for (int pg = 0; pg < n_pairs; pg += pl.R, ++pgc) {
+            // consumer group (pgc & 1) owns this pair group; each group has its own half of the
+            // ring and its own count of stage uses, so that every barrier sees one strictly
+            // sequential user (a group skipping over the other's stages would otherwise wait on
+            // a parity that an older phase already satisfies)
+            const int grp = pgc & 1;
+            const int ns2 = n_stages >> 1;
             const int pair = pg + my_pair;
             const int grow = DOWN ? r0 + 2 * pair + my_row : r0 + pair;  // row in the matrix
             const bool mine = lane < 2 * pl.R && pair < n_pairs && grow < r1;
             // rows copied in this stage (the same for every chunk of the group)
             const int rows_in_stage = DOWN ? min(2 * pl.R, r1 - r0 - 2 * pg) : 2 * min(pl.R, n_pairs - pg);
-            for (int c = 0; c < pl.n_chunks; ++c, ++it) {
+            for (int c = 0; c < pl.n_chunks; ++c, ++itg[grp]) {
                 const int units = min(pl.chunk_units, pl.row_units - c * pl.chunk_units);
-                const int stage = it % n_stages;
-                const uint32_t use = it / n_stages;
+                const int stage = grp * ns2 + (int)(itg[grp] % ns2);
+                const uint32_t use = itg[grp] / ns2;
                 int go = 1;
                 if (lane == 0) {
                     if (use > 0 && !wait_or_abort(&s.empty[stage], (use - 1) & 1, s.abort, p.ws, DOWN ? 7 : 5)) go = 0;
@@ -234,14 +254,17 @@ __device__ __forceinline__ bool produce_half(const DecodeParams &p, const MmaPla
 // Consumer side of one half (all 8 consumer warps).  Returns false after a give-up.
 template <bool DOWN>
 __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPlan &pl, const MmaSmem &s, int n_stages,
-                                             int slot_bytes, int n_slices, uint32_t &it, int &item_parity, int act,
-                                             int tid, int warp, int lane) {
+                                             int slot_bytes, int n_slices, uint32_t &myit, uint32_t &pgc,
+                                             int &item_parity, int act, int tid, int warp, int lane) {
     const int n_items = p.B * n_slices;
     const int total_rows = DOWN ? p.d : p.k;
     const int chunk_bytes_max = pl.chunk_units * 16;
-    const int wpn = DEC_CONSUMER_WARPS / pl.R;  // warps per pair
+    // The 8 consumer warps form two groups of 4 that take alternate stages (pair groups), so
+    // that one group's waiting, shuffling and hand-back overlaps the other group's reads.
+    const int group = warp / DEC_GROUP_WARPS, wig = warp - group * DEC_GROUP_WARPS;
+    const int wpg = DEC_GROUP_WARPS / pl.R;  // warps of a group per pair
     const int g = lane >> 2, t = lane & 3;
-    const int my_pair = warp / wpn, q = warp - my_pair * wpn;
+    const int my_pair = wig / wpg, q = wig - my_pair * wpg;
     // the scratch holds, per sequence, z_hi [ldk] then z_lo [ldk] in bf16 (same bytes as fp32 [ldk])
     __nv_bfloat16 *zbits = reinterpret_cast<__nv_bfloat16 *>(p.z);
     int cur_b = -1;
@@ -267,13 +290,23 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
         }
         const uint4 *vec0 = reinterpret_cast<const uint4 *>(s.vec);
         const uint4 *vec1 = vec0 + pl.row_units;  // z_lo (down only)
+        uint4 xr[MMA_BLOCKS_PER_WARP];
+        if (!DOWN) {  // x does not change within the item: this lane's units of it stay in registers
+#pragma unroll
+            for (int i = 0; i < MMA_BLOCKS_PER_WARP; ++i) {
+                const int u = (q + i * wpg) * 32 + lane;
+                xr[i] = u < pl.row_units ? vec0[u] : make_uint4(0, 0, 0, 0);
+            }
+        }
         bool ok = true;
-        for (int pg = 0; ok && pg < n_pairs; pg += pl.R) {
+        for (int pg = 0; ok && pg < n_pairs; pg += pl.R, ++pgc) {
+            if ((int)(pgc & 1) != group) continue;  // the other group's stage(s)
+            const int ns2 = n_stages >> 1;
             const bool have = pg + my_pair < n_pairs;
             float acc[4][4] = {};
-            for (int c = 0; c < pl.n_chunks; ++c, ++it) {
-                const int stage = it % n_stages;
-                if (!wait_or_abort(&s.full[stage], (it / n_stages) & 1, s.abort, p.ws, DOWN ? 8 : 6)) {
+            for (int c = 0; c < pl.n_chunks; ++c, ++myit) {
+                const int stage = group * ns2 + (int)(myit % ns2);  // this group's half of the ring
+                if (!wait_or_abort(&s.full[stage], (myit / ns2) & 1, s.abort, p.ws, DOWN ? 8 : 6)) {
                     ok = false;
                     break;
                 }
@@ -282,8 +315,8 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
                     const uint4 *row0 = reinterpret_cast<const uint4 *>(s.stages + (size_t)stage * slot_bytes +
                                                                         (size_t)(2 * my_pair) * chunk_bytes_max);
                     const uint4 *row1 = row0 + pl.chunk_units;
-                    pair_mma<DOWN>(acc, row0, row1, vec0 + c * pl.chunk_units, vec1 + c * pl.chunk_units, units, q, wpn,
-                                   lane);
+                    pair_mma<DOWN>(acc, row0, row1, vec0 + c * pl.chunk_units, vec1 + c * pl.chunk_units, xr, units, q,
+                                   wpg, lane);
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&s.empty[stage]);
@@ -301,7 +334,7 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
         if (tid < r1 - r0) {
             const int pair = DOWN ? tid >> 1 : tid;
             float a0 = 0.f, a1 = 0.f;
-            for (int w = 0; w < wpn; ++w) {
+            for (int w = 0; w < wpg; ++w) {
                 const float2 v = part[pair * DEC_CONSUMER_WARPS + w];
                 a0 += v.x;
                 a1 += v.y;
@@ -368,7 +401,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_fused_kernel(const __grid_
     if (tid == 0) {
         for (int i = 0; i < fp.n_stages; ++i) {
             mbar_init(&s.full[i], 1);
-            mbar_init(&s.empty[i], DEC_CONSUMER_WARPS);
+            mbar_init(&s.empty[i], DEC_GROUP_WARPS);  // the group that owns the stage hands it back
         }
         *s.abort = 0;
         mbar_fence_init();
@@ -380,25 +413,27 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_fused_kernel(const __grid_
         // ---- producer warp: weights only, so it never waits for the previous grid, nor for
         //      the meeting point: the first stages of W_2_hat are on their way while the
         //      consumers are still waiting for the other CTAs' z
-        uint32_t it = 0;
-        if (produce_half<false>(p, fp.gu, s, fp.n_stages, fp.slot_bytes, p.n_slices, it, lane))
-            produce_half<true>(p, fp.dn, s, fp.n_stages, fp.slot_bytes, p.n_slices_dn, it, lane);
-        if (lane == 0) producer_drain_mma(s, fp.n_stages, it);
+        uint32_t itg[2] = {0, 0}, pgc = 0;
+        if (produce_half<false>(p, fp.gu, s, fp.n_stages, fp.slot_bytes, p.n_slices, itg, pgc, lane))
+            produce_half<true>(p, fp.dn, s, fp.n_stages, fp.slot_bytes, p.n_slices_dn, itg, pgc, lane);
+        if (lane == 0) producer_drain_mma(s, fp.n_stages, itg);
         return;
     }
 
     // ---- consumers
     pdl_wait_prior_grids();  // x, the z scratch and the outputs belong to earlier work on the stream
-    uint32_t it = 0;
+    uint32_t myit = 0, pgc = 0;  // stage uses of this warp's group; pair groups seen by everybody
     int item_parity = 0;
-    if (!consume_half<false>(p, fp.gu, s, fp.n_stages, fp.slot_bytes, p.n_slices, it, item_parity, act, tid, warp, lane))
+    if (!consume_half<false>(p, fp.gu, s, fp.n_stages, fp.slot_bytes, p.n_slices, myit, pgc, item_parity, act, tid, warp,
+                             lane))
         return;
     __threadfence();  // this CTA's z entries are visible device-wide before it reports in
     consumer_barrier();
     if (tid == 0) grid_meet(static_cast<WsHeader *>(p.ws), gridDim.x, s.abort, p.ws);
     consumer_barrier();
     if (*s.abort) return;
-    consume_half<true>(p, fp.dn, s, fp.n_stages, fp.slot_bytes, p.n_slices_dn, it, item_parity, act, tid, warp, lane);
+    consume_half<true>(p, fp.dn, s, fp.n_stages, fp.slot_bytes, p.n_slices_dn, myit, pgc, item_parity, act, tid, warp,
+                       lane);
 }
 
 griffin_status decode_bf16_mma(DecodeParams &p, int act, uint32_t flags, cudaStream_t stream) {
@@ -412,7 +447,7 @@ griffin_status decode_bf16_mma(DecodeParams &p, int act, uint32_t flags, cudaStr
     fp.slot_bytes = max(fp.gu.stage_bytes, fp.dn.stage_bytes);
     fp.vec_bytes = max(p.d * 2, p.ldk * 4);
     int n = ((int)MMA_SMEM_TARGET - fp.vec_bytes - (int)mma_fixed_smem(8)) / fp.slot_bytes;
-    fp.n_stages = n < 2 ? 2 : (n > 8 ? 8 : n);
+    fp.n_stages = (n < 2 ? 2 : (n > 8 ? 8 : n)) & ~1;  // two halves, one per consumer group
     p.n_slices = slices_for(p.k, sms);
     p.n_slices_dn = slices_for(p.d, sms);
     // every CTA of the grid must be able to run at the same time (they meet half-way): one per SM

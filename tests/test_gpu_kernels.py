@@ -111,6 +111,8 @@ DECODE_SHAPES = [
     (4096, 11008, 5504, 1),  # Llama-2-7B shape
     (5120, 2048, 1024, 8),   # widest d of the workloads, batch 8
     (8192, 1024, 512, 1),    # largest supported d
+    (512, 9008, 9008, 1),    # rows of W_2_hat longer than one stage chunk (two chunks)
+    (256, 20000, 16400, 2),  # three chunks per row, two sequences
 ]
 
 
