@@ -117,6 +117,29 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
 // Every device-side wait gives up after this many SM clock cycles (about 2 s).
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;
 
+// Barrier wait that gives up after WAIT_LIMIT_CYCLES, or as soon as another thread of the CTA
+// has given up.  On a give-up the status word is raised and false is returned.
+__device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort, void *ws,
+                                              int where) {
+    // Fast path: plain polling.  The clock is only consulted every few thousand polls, so a
+    // wait that succeeds (every wait of a healthy run) never pays for reading it.
+#pragma unroll 1
+    for (int i = 0; i < 4096; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 4096; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort) return false;
+        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+            *abort = 1;
+            raise_status(ws, DEV_STATUS_TIMEOUT, where);
+            return false;
+        }
+    }
+}
+
 // 1-D bulk copy global -> shared memory of this CTA; completion is counted on `bar` in
 // bytes.  dst and src 16-byte aligned, bytes a multiple of 16.
 __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t bytes, uint64_t *bar) {

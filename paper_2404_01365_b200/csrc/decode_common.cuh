@@ -51,29 +51,6 @@ static inline size_t dec_smem_bytes(int n_stages, int stage_bytes) {
     return (size_t)n_stages * stage_bytes + 2 * n_stages * sizeof(uint64_t) + 2 * DEC_PART_FLOATS * sizeof(float) + 16;
 }
 
-// Barrier wait that gives up after WAIT_LIMIT_CYCLES, or as soon as another thread of the CTA
-// has given up.  On a give-up the status word is raised and false is returned.
-__device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort, void *ws,
-                                              int where) {
-    // Fast path: plain polling.  The clock is only consulted every few thousand polls, so a
-    // wait that succeeds (every wait of a healthy run) never pays for reading it.
-#pragma unroll 1
-    for (int i = 0; i < 4096; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    for (;;) {
-#pragma unroll 1
-        for (int i = 0; i < 4096; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
-        if (*abort) return false;
-        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
-            *abort = 1;
-            raise_status(ws, DEV_STATUS_TIMEOUT, where);
-            return false;
-        }
-    }
-}
-
 __device__ __forceinline__ void consumer_barrier() {
     asm volatile("bar.sync 1, %0;" ::"n"(DEC_CONSUMERS) : "memory");
 }

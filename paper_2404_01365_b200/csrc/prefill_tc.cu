@@ -1,9 +1,404 @@
-// Placeholder: tensor-core path not wired yet.
+// Prompt-phase FF on the 5th-generation tensor cores (Eqs. 1 and 3 of the GRIFFIN paper), bf16
+// storage, fp32 accumulation:
+//   kernel<DUAL = true > : Z = sigma(X W_g^T + b_g) * (X W_1^T + b_1), also Z in fp32 and the
+//                          per-tile partial sums of squares of its rows (for the statistic)
+//   kernel<DUAL = false> : Y = Z W_2^T + b_2
+//
+// One persistent CTA per SM, 192 threads in three roles:
+//   warp 0      TMA producer: cp.async.bulk.tensor (2-D tiles, 128-byte swizzle, no multicast)
+//               of a 128 x 64 tile of the left operand and a BN x 64 tile of the weights
+//               into a ring of shared-memory stages;
+//   warp 1      MMA issuer: one elected thread issues tcgen05.mma (M = 128, N = BN, K = 16,
+//               operands from shared memory through matrix descriptors, accumulator in TMEM),
+//               releases each stage with tcgen05.commit; it also owns the TMEM allocation;
+//   warps 2-5   epilogue: tcgen05.ld of the accumulator (one row per thread), activation and
+//               gating (or bias), stores.  TMEM holds two accumulator stages, so the epilogue
+//               of one tile runs under the MMAs of the next.
+// For DUAL the gate and up tiles of the same 128 neurons are loaded one behind the other, so
+// that a single N = 256 MMA against the shared X tile fills columns 0..127 with the gate
+// and 128..255 with the up pre-activations: the epilogue thread that owns a row finds both.
+//
+// Every wait is bounded; after a give-up the CTA still frees its TMEM before it returns.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "launch.h"
 #include "prefill_tc.h"
+
 namespace griffin {
-bool prefill_tc_supported(const griffin_ff_desc *, int) { return false; }
-griffin_status launch_prefill_tc(const griffin_ff_desc *, const griffin_ff_weights *, const void *, int, void *,
-                                 __nv_bfloat16 *, float *, float *, int *, void *, cudaStream_t) {
-    return GRIFFIN_ERR_UNSUPPORTED;
+
+constexpr int TC_BM = 128;        // rows (tokens) per tile
+constexpr int TC_BK = 64;         // K per stage: 64 bf16 = one 128-byte swizzle row
+constexpr int TC_THREADS = 192;
+constexpr int TC_STAGES = 4;
+
+// ---- PTX wrappers -------------------------------------------------------------------------
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int x, int y, uint64_t *bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+            smem_u32(dst)),
+        "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
 }
+__device__ __forceinline__ void tmem_alloc(uint32_t *dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)),
+                 "r"(ncols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// D[tmem] (+)= A[smem] * B[smem]; accumulate = 0 overwrites D
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// the barrier gets one arrival once every MMA issued so far by this thread has completed
+__device__ __forceinline__ void umma_commit(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+// 32 lanes x 32 columns of fp32: thread i of the warp receives row (lane base + i)
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 bf16) and
+// which was written by TMA with the 128-byte swizzle: rows 128 bytes apart, groups of 8 rows
+// 1024 bytes apart (stride byte offset), descriptor version 1, layout type 2 (128B swizzle).
+// The tile must start on a 1024-byte boundary; stepping K by 16 elements adds 32 bytes to
+// the start address.
+__device__ __forceinline__ uint64_t smem_desc_sw128(const void *tile, int k16) {
+    const uint32_t addr = smem_u32(tile) + (uint32_t)k16 * 32u;
+    return (uint64_t)((addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, M x N.
+__host__ __device__ constexpr uint32_t umma_idesc(int M, int N) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+struct TcParams {
+    int S;            // rows of the left operand and of the output
+    int n_total;      // columns of the output (d_ff for DUAL, d otherwise)
+    int K;            // reduction length (d for DUAL, d_ff otherwise), multiple of 64
+    int m_tiles, n_tiles;
+    const __nv_bfloat16 *bias0, *bias1;  // DUAL: b_gate, b_up; otherwise b_down, unused (may be null)
+    __nv_bfloat16 *out;                  // Z or Y, [S, n_total]
+    float *zf;                           // DUAL: Z in fp32, [S, n_total]
+    float *rowsq;                        // DUAL: [S, n_tiles] partial sums of squares of the fp32 rows
+    int act;
+    void *ws;
+};
+
+struct TcSmem {
+    uint8_t *stages;
+    uint64_t *full, *empty, *acc_full, *acc_empty;
+    uint32_t *tmem_slot;
+    volatile int *abort;
+};
+constexpr size_t TC_TAIL_BYTES = (2 * TC_STAGES + 4) * sizeof(uint64_t) + 16;
+
+template <bool DUAL, int BN>
+__global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant__ CUtensorMap map_a,
+                                                           const __grid_constant__ CUtensorMap map_b0,
+                                                           const __grid_constant__ CUtensorMap map_b1,
+                                                           const __grid_constant__ TcParams p) {
+    constexpr int NT = DUAL ? 256 : BN;            // MMA N = TMEM columns of one accumulator stage
+    constexpr int B_ROWS = DUAL ? 128 : BN;        // rows of one weight tile load
+    constexpr int A_BYTES = TC_BM * TC_BK * 2;     // 16 KB
+    constexpr int STAGE_BYTES = A_BYTES + NT * TC_BK * 2;
+    constexpr uint32_t IDESC = umma_idesc(TC_BM, NT);
+
+    extern __shared__ uint8_t smem_raw[];
+    TcSmem s;
+    s.stages = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    s.full = reinterpret_cast<uint64_t *>(s.stages + (size_t)TC_STAGES * STAGE_BYTES);
+    s.empty = s.full + TC_STAGES;
+    s.acc_full = s.empty + TC_STAGES;
+    s.acc_empty = s.acc_full + 2;
+    s.tmem_slot = reinterpret_cast<uint32_t *>(s.acc_empty + 2);
+    s.abort = reinterpret_cast<volatile int *>(s.tmem_slot + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        for (int i = 0; i < TC_STAGES; ++i) {
+            mbar_init(&s.full[i], 1);
+            mbar_init(&s.empty[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&s.acc_full[i], 1);
+            mbar_init(&s.acc_empty[i], 4);  // one arrival per epilogue warp
+        }
+        *s.abort = 0;
+        mbar_fence_init();
+    }
+    if (warp == 1) tmem_alloc(s.tmem_slot, 2 * NT);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *s.tmem_slot;
+
+    const int n_tiles_total = p.m_tiles * p.n_tiles;
+    const int kb_total = p.K / TC_BK;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < n_tiles_total; tile += gridDim.x) {
+                const int m = tile % p.m_tiles, n = tile / p.m_tiles;  // tiles sharing weights are neighbours
+                for (int kb = 0; kb < kb_total; ++kb, ++it) {
+                    const int stage = it % TC_STAGES;
+                    const uint32_t use = it / TC_STAGES;
+                    if (use > 0 && !wait_or_abort(&s.empty[stage], (use - 1) & 1, s.abort, p.ws, 20)) {
+                        ok = false;
+                        break;
+                    }
+                    uint8_t *a = s.stages + (size_t)stage * STAGE_BYTES;
+                    mbar_arrive_expect_tx(&s.full[stage], STAGE_BYTES);
+                    tma_load_2d(a, &map_a, kb * TC_BK, m * TC_BM, &s.full[stage]);
+                    tma_load_2d(a + A_BYTES, &map_b0, kb * TC_BK, n * B_ROWS, &s.full[stage]);
+                    if (DUAL) tma_load_2d(a + A_BYTES + B_ROWS * TC_BK * 2, &map_b1, kb * TC_BK, n * B_ROWS, &s.full[stage]);
+                }
+            }
+            // stay until every copy that was started has landed
+            const uint32_t first = it > TC_STAGES ? it - TC_STAGES : 0;
+            for (uint32_t j = first; j < it; ++j) {
+                const long long t0 = clock64();
+                while (!mbar_try_wait(&s.full[j % TC_STAGES], (j / TC_STAGES) & 1))
+                    if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            uint32_t it = 0, tcount = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < n_tiles_total; tile += gridDim.x, ++tcount) {
+                const int acc = tcount & 1;
+                const uint32_t acc_use = tcount >> 1;
+                if (acc_use > 0 && !wait_or_abort(&s.acc_empty[acc], (acc_use - 1) & 1, s.abort, p.ws, 21)) break;
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * NT);
+                for (int kb = 0; kb < kb_total; ++kb, ++it) {
+                    const int stage = it % TC_STAGES;
+                    if (!wait_or_abort(&s.full[stage], (it / TC_STAGES) & 1, s.abort, p.ws, 22)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after_sync();
+                    const uint8_t *a = s.stages + (size_t)stage * STAGE_BYTES;
+#pragma unroll
+                    for (int k16 = 0; k16 < TC_BK / 16; ++k16)
+                        umma_bf16(d_tmem, smem_desc_sw128(a, k16), smem_desc_sw128(a + A_BYTES, k16), IDESC,
+                                  (kb | k16) != 0 ? 1u : 0u);
+                    umma_commit(&s.empty[stage]);  // the stage may be refilled once these MMAs have read it
+                }
+                if (ok) umma_commit(&s.acc_full[acc]);
+            }
+        }
+    } else {
+        // ---------------- epilogue (warps 2..5) ----------------
+        const int wq = warp & 3;                 // the TMEM lane quarter this warp may read
+        const int row_in_tile = wq * 32 + lane;  // one output row per thread
+        uint32_t tcount = 0;
+        for (int tile = blockIdx.x; tile < n_tiles_total; tile += gridDim.x, ++tcount) {
+            const int m = tile % p.m_tiles, n = tile / p.m_tiles;
+            const int acc = tcount & 1;
+            if (!wait_or_abort(&s.acc_full[acc], (tcount >> 1) & 1, s.abort, p.ws, 23)) break;
+            tc_fence_after_sync();
+            const int row = m * TC_BM + row_in_tile;
+            const bool live = row < p.S;
+            const uint32_t taddr = tmem_base + ((uint32_t)(wq * 32) << 16) + (uint32_t)(acc * NT);
+            if (DUAL) {
+                float sq = 0.f;
+#pragma unroll 1
+                for (int c = 0; c < 128; c += 32) {
+                    float g[32], u[32];
+                    tmem_ld32(taddr + c, g);
+                    tmem_ld32(taddr + 128 + c, u);
+                    const int col = n * 128 + c;
+                    uint32_t packed[16];
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        float g0 = g[i], g1 = g[i + 1], u0 = u[i], u1 = u[i + 1];
+                        if (p.bias0) { g0 += __bfloat162float(p.bias0[col + i]); g1 += __bfloat162float(p.bias0[col + i + 1]); }
+                        if (p.bias1) { u0 += __bfloat162float(p.bias1[col + i]); u1 += __bfloat162float(p.bias1[col + i + 1]); }
+                        const float z0 = sigma_rt(p.act, g0) * u0, z1 = sigma_rt(p.act, g1) * u1;
+                        g[i] = z0;
+                        g[i + 1] = z1;
+                        sq = fmaf(z0, z0, sq);
+                        sq = fmaf(z1, z1, sq);
+                        const __nv_bfloat162 h = __floats2bfloat162_rn(z0, z1);
+                        packed[i >> 1] = *reinterpret_cast<const uint32_t *>(&h);
+                    }
+                    if (live) {
+                        uint4 *zo = reinterpret_cast<uint4 *>(p.out + (size_t)row * p.n_total + col);
+                        float4 *fo = reinterpret_cast<float4 *>(p.zf + (size_t)row * p.n_total + col);
+#pragma unroll
+                        for (int v = 0; v < 4; ++v)
+                            zo[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+#pragma unroll
+                        for (int v = 0; v < 8; ++v) fo[v] = make_float4(g[4 * v], g[4 * v + 1], g[4 * v + 2], g[4 * v + 3]);
+                    }
+                }
+                if (live) p.rowsq[(size_t)row * p.n_tiles + n] = sq;
+            } else {
+#pragma unroll 1
+                for (int c = 0; c < BN; c += 32) {
+                    float a[32];
+                    tmem_ld32(taddr + c, a);
+                    const int col = n * BN + c;
+                    uint32_t packed[16];
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        float y0 = a[i], y1 = a[i + 1];
+                        if (p.bias0) { y0 += __bfloat162float(p.bias0[col + i]); y1 += __bfloat162float(p.bias0[col + i + 1]); }
+                        const __nv_bfloat162 h = __floats2bfloat162_rn(y0, y1);
+                        packed[i >> 1] = *reinterpret_cast<const uint32_t *>(&h);
+                    }
+                    if (live) {
+                        uint4 *yo = reinterpret_cast<uint4 *>(p.out + (size_t)row * p.n_total + col);
+#pragma unroll
+                        for (int v = 0; v < 4; ++v)
+                            yo[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+                    }
+                }
+            }
+            tc_fence_before_sync();  // this warp's TMEM reads are done
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&s.acc_empty[acc]);
+        }
+    }
+
+    // ---------------- teardown: everybody meets, the allocating warp frees TMEM ----------------
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, 2 * NT);
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver's tensor-map encoder, looked up through the runtime (the library does not link libcuda).
+static EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    return fn;
+}
+
+// Row-major bf16 matrix [rows, cols] (cols contiguous); box = box_rows x 64 columns, 128-byte swizzle,
+// out-of-range elements read as zero.
+static bool make_map(CUtensorMap *map, const void *base, int rows, int cols, int box_rows) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (enc == nullptr) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool prefill_tc_supported(const griffin_ff_desc *desc, int S) {
+    if (desc->dtype != GRIFFIN_DT_BF16 || S < 1) return false;
+    if (desc->d % 128 != 0 || desc->d_ff % 128 != 0) return false;  // whole tiles in N, whole stages in K
+    return encode_tiled_fn() != nullptr;
+}
+
+template <bool DUAL, int BN>
+static griffin_status launch_tc(const CUtensorMap &ma, const CUtensorMap &mb0, const CUtensorMap &mb1, const TcParams &p,
+                                int sms, cudaStream_t stream) {
+    constexpr int NT = DUAL ? 256 : BN;
+    const size_t smem = 1024 + (size_t)TC_STAGES * (TC_BM * TC_BK * 2 + NT * TC_BK * 2) + TC_TAIL_BYTES;
+    const void *fn = (const void *)ff_tc_kernel<DUAL, BN>;
+    if (ensure_dynamic_smem(fn, smem) != cudaSuccess) return GRIFFIN_ERR_CUDA;
+    const int tiles = p.m_tiles * p.n_tiles;
+    ff_tc_kernel<DUAL, BN><<<tiles < sms ? tiles : sms, TC_THREADS, smem, stream>>>(ma, mb0, mb1, p);
+    return cudaGetLastError() == cudaSuccess ? GRIFFIN_OK : GRIFFIN_ERR_CUDA;
+}
+
+griffin_status launch_prefill_tc(const griffin_ff_desc *desc, const griffin_ff_weights *w, const void *x, int S,
+                                 void *y, __nv_bfloat16 *z, float *zf, float *rowsq, int *n_col_tiles, void *ws,
+                                 cudaStream_t stream) {
+    const int d = desc->d, d_ff = desc->d_ff;
+    const int sms = device_sm_count();
+    if (sms <= 0) return GRIFFIN_ERR_CUDA;
+    const int m_tiles = (S + TC_BM - 1) / TC_BM;
+    CUtensorMap mx, mg, mu;
+    if (!make_map(&mx, x, S, d, TC_BM) || !make_map(&mg, w->w_gate, d_ff, d, 128) ||
+        !make_map(&mu, w->w_up, d_ff, d, 128))
+        return GRIFFIN_ERR_CUDA;
+    TcParams p = {};
+    p.S = S;
+    p.n_total = d_ff;
+    p.K = d;
+    p.m_tiles = m_tiles;
+    p.n_tiles = d_ff / 128;
+    p.bias0 = static_cast<const __nv_bfloat16 *>(w->b_gate);
+    p.bias1 = static_cast<const __nv_bfloat16 *>(w->b_up);
+    p.out = z;
+    p.zf = zf;
+    p.rowsq = rowsq;
+    p.act = desc->act;
+    p.ws = ws;
+    *n_col_tiles = p.n_tiles;
+    griffin_status st = launch_tc<true, 128>(mx, mg, mu, p, sms, stream);
+    if (st != GRIFFIN_OK || y == nullptr) return st;
+
+    // Y = Z W_2^T + b_2: wide tiles when there are enough of them to fill the GPU, else narrow ones
+    const bool wide = d % 256 == 0 && (d / 256) * m_tiles >= sms;
+    const int bn = wide ? 256 : 128;
+    CUtensorMap mz, md;
+    if (!make_map(&mz, z, S, d_ff, TC_BM) || !make_map(&md, w->w_down, d, d_ff, bn)) return GRIFFIN_ERR_CUDA;
+    TcParams q = {};
+    q.S = S;
+    q.n_total = d;
+    q.K = d_ff;
+    q.m_tiles = m_tiles;
+    q.n_tiles = d / bn;
+    q.bias0 = static_cast<const __nv_bfloat16 *>(w->b_down);
+    q.out = static_cast<__nv_bfloat16 *>(y);
+    q.act = desc->act;
+    q.ws = ws;
+    return wide ? launch_tc<false, 256>(mz, md, md, q, sms, stream) : launch_tc<false, 128>(mz, md, md, q, sms, stream);
+}
+
 }  // namespace griffin
