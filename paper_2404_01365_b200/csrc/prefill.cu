@@ -183,23 +183,40 @@ __global__ void row_inv_kernel(const float *__restrict__ rowsq, int S, int n_col
     if (lane == 0) inv[row] = sq > 0.f ? 1.0f / sq : 0.f;
 }
 
-// Step 4: a thread owns four neighbouring columns of the fp32 Z over one chunk of tokens.
-__global__ void __launch_bounds__(128) col_partial_kernel(const float *__restrict__ z, const float *__restrict__ inv,
+// Step 4: a CTA owns 128 neighbouring columns of the fp32 Z over one chunk of tokens; each of
+// its 8 warps takes every 8th token of the chunk (one float4 per lane, all loads of a warp in
+// flight together) and the warps' sums meet in shared memory in a fixed order.
+__global__ void __launch_bounds__(256) col_partial_kernel(const float *__restrict__ z, const float *__restrict__ inv,
                                                           int S, int d_ff, float *__restrict__ colpart) {
-    const int col = (blockIdx.x * 128 + threadIdx.x) * 4;
-    if (col >= d_ff) return;
+    __shared__ float4 red[8][32];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int col = (blockIdx.x * 32 + lane) * 4;
     const int r0 = blockIdx.y * PF_ROW_CHUNK, r1 = min(S, r0 + PF_ROW_CHUNK);
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 4
-    for (int r = r0; r < r1; ++r) {
-        const float4 f = *reinterpret_cast<const float4 *>(z + (size_t)r * d_ff + col);
-        const float w = __ldg(inv + r);
-        acc.x = fmaf(f.x * f.x, w, acc.x);
-        acc.y = fmaf(f.y * f.y, w, acc.y);
-        acc.z = fmaf(f.z * f.z, w, acc.z);
-        acc.w = fmaf(f.w * f.w, w, acc.w);
+    if (col < d_ff) {
+#pragma unroll
+        for (int i = 0; i < PF_ROW_CHUNK / 8; ++i) {
+            const int r = r0 + warp + 8 * i;
+            if (r < r1) {
+                const float4 f = *reinterpret_cast<const float4 *>(z + (size_t)r * d_ff + col);
+                const float w = __ldg(inv + r);
+                acc.x = fmaf(f.x * f.x, w, acc.x);
+                acc.y = fmaf(f.y * f.y, w, acc.y);
+                acc.z = fmaf(f.z * f.z, w, acc.z);
+                acc.w = fmaf(f.w * f.w, w, acc.w);
+            }
+        }
     }
-    *reinterpret_cast<float4 *>(colpart + (size_t)blockIdx.y * d_ff + col) = acc;
+    red[warp][lane] = acc;
+    __syncthreads();
+    if (warp == 0 && col < d_ff) {
+        float4 t = red[0][lane];
+#pragma unroll
+        for (int w = 1; w < 8; ++w) {
+            t.x += red[w][lane].x; t.y += red[w][lane].y; t.z += red[w][lane].z; t.w += red[w][lane].w;
+        }
+        *reinterpret_cast<float4 *>(colpart + (size_t)blockIdx.y * d_ff + col) = t;
+    }
 }
 
 // Step 5.
@@ -253,8 +270,8 @@ static griffin_status prefill_typed(const griffin_ff_desc *desc, const griffin_f
     row_inv_kernel<<<(S + 7) / 8, 256, 0, stream>>>(rowsq, S, n_col_tiles, inv);
     if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
     const float *z32 = kBf16 ? zf : reinterpret_cast<const float *>(z);
-    const dim3 g4((d_ff + 511) / 512, ps.n_row_chunks);
-    col_partial_kernel<<<g4, 128, 0, stream>>>(z32, inv, S, d_ff, colpart);
+    const dim3 g4((d_ff + 127) / 128, ps.n_row_chunks);
+    col_partial_kernel<<<g4, 256, 0, stream>>>(z32, inv, S, d_ff, colpart);
     if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
     score_finish_kernel<<<(d_ff + 255) / 256, 256, 0, stream>>>(colpart, ps.n_row_chunks, d_ff, score);
     if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;

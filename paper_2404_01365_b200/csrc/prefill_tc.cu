@@ -30,7 +30,10 @@ namespace griffin {
 constexpr int TC_BM = 128;        // rows (tokens) per tile
 constexpr int TC_BK = 64;         // K per stage: 64 bf16 = one 128-byte swizzle row
 constexpr int TC_THREADS = 192;
-constexpr int TC_STAGES = 4;
+#ifndef GRIFFIN_TC_STAGES
+#define GRIFFIN_TC_STAGES 4
+#endif
+constexpr int TC_STAGES = GRIFFIN_TC_STAGES;
 
 // ---- PTX wrappers -------------------------------------------------------------------------
 __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int x, int y, uint64_t *bar) {
