@@ -33,7 +33,7 @@ griffin_status launch_compact(const griffin_ff_desc *desc, const griffin_ff_weig
 
 // Carve-up of the workspace behind its header for the prompt-phase path.
 struct PrefillScratch {
-    size_t z_off, zf_off, rowsq_off, inv_off, colpart_off, total;  // byte offsets from the scratch base
+    size_t z_off, zf_off, rowsq_off, inv_off, colpart_off, ypart_off, total;  // byte offsets from the scratch base
     int n_col_tiles;                                        // partial row sums kept per token
     int n_row_chunks;                                       // partial column sums kept per neuron
 };

@@ -45,6 +45,12 @@ PrefillScratch prefill_scratch(const griffin_ff_desc *desc, int S) {
     off = align_up(off + (size_t)S * sizeof(float), 256);
     ps.colpart_off = off;
     off = align_up(off + (size_t)ps.n_row_chunks * desc->d_ff * sizeof(float), 256);
+    ps.ypart_off = off;  // fp32 partial outputs of a K-split down projection (bf16 tensor-core path)
+    if (desc->dtype != GRIFFIN_DT_F32) {
+        int bn = 0, splits = 1;
+        gemm2_plan(S, desc->d, &bn, &splits);
+        if (splits > 1) off = align_up(off + (size_t)splits * S * desc->d * sizeof(float), 256);
+    }
     ps.total = off;
     return ps;
 }
@@ -247,7 +253,8 @@ static griffin_status prefill_typed(const griffin_ff_desc *desc, const griffin_f
     if constexpr (kBf16) use_tc = prefill_tc_supported(desc, S);
     if (use_tc) {
         if constexpr (kBf16) {
-            griffin_status st = launch_prefill_tc(desc, w, x, S, y, z, zf, rowsq, &n_col_tiles, ws, stream);
+            griffin_status st = launch_prefill_tc(desc, w, x, S, y, z, zf, rowsq, reinterpret_cast<float *>(scratch + ps.ypart_off),
+                                                  &n_col_tiles, ws, stream);
             if (st != GRIFFIN_OK) return st;
         }
         ff2_done = true;

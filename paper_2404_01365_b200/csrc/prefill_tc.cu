@@ -109,6 +109,8 @@ struct TcParams {
     __nv_bfloat16 *out;                  // Z or Y, [S, n_total]
     float *zf;                           // DUAL: Z in fp32, [S, n_total]
     float *rowsq;                        // DUAL: [S, n_tiles] partial sums of squares of the fp32 rows
+    int splits;                          // K splits (1 unless the plain GEMM has too few tiles)
+    float *part;                         // splits > 1: fp32 partial outputs [splits, S, n_total]
     int act;
     void *ws;
 };
@@ -161,7 +163,7 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
     tc_fence_after_sync();
     const uint32_t tmem_base = *s.tmem_slot;
 
-    const int n_tiles_total = p.m_tiles * p.n_tiles;
+    const int n_tiles_total = p.m_tiles * p.n_tiles * p.splits;  // work items: (m, n, K split)
     const int kb_total = p.K / TC_BK;
 
     if (warp == 0) {
@@ -170,8 +172,10 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
             uint32_t it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < n_tiles_total; tile += gridDim.x) {
-                const int m = tile % p.m_tiles, n = tile / p.m_tiles;  // tiles sharing weights are neighbours
-                for (int kb = 0; kb < kb_total; ++kb, ++it) {
+                const int m = tile % p.m_tiles, rest = tile / p.m_tiles;  // tiles sharing weights are neighbours
+                const int n = rest % p.n_tiles, sp = rest / p.n_tiles;
+                const int kb0 = sp * kb_total / p.splits, kb1 = (sp + 1) * kb_total / p.splits;
+                for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const int stage = it % TC_STAGES;
                     const uint32_t use = it / TC_STAGES;
                     if (use > 0 && !wait_or_abort(&s.empty[stage], (use - 1) & 1, s.abort, p.ws, 20)) {
@@ -204,7 +208,9 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
                 if (acc_use > 0 && !wait_or_abort(&s.acc_empty[acc], (acc_use - 1) & 1, s.abort, p.ws, 21)) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * NT);
-                for (int kb = 0; kb < kb_total; ++kb, ++it) {
+                const int sp = tile / (p.m_tiles * p.n_tiles);
+                const int kb0 = sp * kb_total / p.splits, kb1 = (sp + 1) * kb_total / p.splits;
+                for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const int stage = it % TC_STAGES;
                     if (!wait_or_abort(&s.full[stage], (it / TC_STAGES) & 1, s.abort, p.ws, 22)) {
                         ok = false;
@@ -215,7 +221,7 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
 #pragma unroll
                     for (int k16 = 0; k16 < TC_BK / 16; ++k16)
                         umma_bf16(d_tmem, smem_desc_sw128(a, k16), smem_desc_sw128(a + A_BYTES, k16), IDESC,
-                                  (kb | k16) != 0 ? 1u : 0u);
+                                  (kb > kb0 || k16 > 0) ? 1u : 0u);
                     umma_commit(&s.empty[stage]);  // the stage may be refilled once these MMAs have read it
                 }
                 if (ok) umma_commit(&s.acc_full[acc]);
@@ -227,7 +233,8 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
         const int row_in_tile = wq * 32 + lane;  // one output row per thread
         uint32_t tcount = 0;
         for (int tile = blockIdx.x; tile < n_tiles_total; tile += gridDim.x, ++tcount) {
-            const int m = tile % p.m_tiles, n = tile / p.m_tiles;
+            const int m = tile % p.m_tiles, rest = tile / p.m_tiles;
+            const int n = rest % p.n_tiles, sp = rest / p.n_tiles;
             const int acc = tcount & 1;
             if (!wait_or_abort(&s.acc_full[acc], (tcount >> 1) & 1, s.abort, p.ws, 23)) break;
             tc_fence_after_sync();
@@ -273,6 +280,14 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
                     float a[32];
                     tmem_ld32(taddr + c, a);
                     const int col = n * BN + c;
+                    if (p.splits > 1) {  // partial sums leave in fp32; bias and rounding happen in the reduction
+                        if (live) {
+                            float4 *po = reinterpret_cast<float4 *>(p.part + ((size_t)sp * p.S + row) * p.n_total + col);
+#pragma unroll
+                            for (int v = 0; v < 8; ++v) po[v] = make_float4(a[4 * v], a[4 * v + 1], a[4 * v + 2], a[4 * v + 3]);
+                        }
+                        continue;
+                    }
                     uint32_t packed[16];
 #pragma unroll
                     for (int i = 0; i < 32; i += 2) {
@@ -304,9 +319,39 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
     }
 }
 
+// y = bf16(sum over K splits of part + bias), four columns per thread, splits added in order.
+__global__ void splitk_reduce_kernel(const float *__restrict__ part, const __nv_bfloat16 *__restrict__ bias,
+                                     __nv_bfloat16 *__restrict__ y, int splits, size_t n_elems, int n_total) {
+    const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+    if (i >= n_elems) return;
+    float4 acc = *reinterpret_cast<const float4 *>(part + i);
+    for (int s = 1; s < splits; ++s) {
+        const float4 v = *reinterpret_cast<const float4 *>(part + (size_t)s * n_elems + i);
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    if (bias) {
+        const int c = (int)(i % n_total);
+        acc.x += __bfloat162float(bias[c]); acc.y += __bfloat162float(bias[c + 1]);
+        acc.z += __bfloat162float(bias[c + 2]); acc.w += __bfloat162float(bias[c + 3]);
+    }
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+    *reinterpret_cast<uint2 *>(y + i) =
+        make_uint2(*reinterpret_cast<const uint32_t *>(&lo), *reinterpret_cast<const uint32_t *>(&hi));
+}
+
 // ---------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------
+constexpr int TC_TARGET_CTAS = 148;  // SMs of a B200: what a grid should fill
+
+void gemm2_plan(int S, int d, int *bn, int *splits) {
+    const int m_tiles = (S + TC_BM - 1) / TC_BM;
+    *bn = d % 256 == 0 ? 256 : 128;
+    const int tiles = m_tiles * (d / *bn);
+    int sp = TC_TARGET_CTAS / (tiles > 0 ? tiles : 1);
+    *splits = sp < 1 ? 1 : (sp > 4 ? 4 : sp);
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -353,14 +398,14 @@ static griffin_status launch_tc(const CUtensorMap &ma, const CUtensorMap &mb0, c
     const size_t smem = 1024 + (size_t)TC_STAGES * (TC_BM * TC_BK * 2 + NT * TC_BK * 2) + TC_TAIL_BYTES;
     const void *fn = (const void *)ff_tc_kernel<DUAL, BN>;
     if (ensure_dynamic_smem(fn, smem) != cudaSuccess) return GRIFFIN_ERR_CUDA;
-    const int tiles = p.m_tiles * p.n_tiles;
+    const int tiles = p.m_tiles * p.n_tiles * p.splits;
     ff_tc_kernel<DUAL, BN><<<tiles < sms ? tiles : sms, TC_THREADS, smem, stream>>>(ma, mb0, mb1, p);
     return cudaGetLastError() == cudaSuccess ? GRIFFIN_OK : GRIFFIN_ERR_CUDA;
 }
 
 griffin_status launch_prefill_tc(const griffin_ff_desc *desc, const griffin_ff_weights *w, const void *x, int S,
-                                 void *y, __nv_bfloat16 *z, float *zf, float *rowsq, int *n_col_tiles, void *ws,
-                                 cudaStream_t stream) {
+                                 void *y, __nv_bfloat16 *z, float *zf, float *rowsq, float *ypart, int *n_col_tiles,
+                                 void *ws, cudaStream_t stream) {
     const int d = desc->d, d_ff = desc->d_ff;
     const int sms = device_sm_count();
     if (sms <= 0) return GRIFFIN_ERR_CUDA;
@@ -382,13 +427,14 @@ griffin_status launch_prefill_tc(const griffin_ff_desc *desc, const griffin_ff_w
     p.rowsq = rowsq;
     p.act = desc->act;
     p.ws = ws;
+    p.splits = 1;
     *n_col_tiles = p.n_tiles;
     griffin_status st = launch_tc<true, 128>(mx, mg, mu, p, sms, stream);
     if (st != GRIFFIN_OK || y == nullptr) return st;
 
-    // Y = Z W_2^T + b_2: wide tiles when there are enough of them to fill the GPU, else narrow ones
-    const bool wide = d % 256 == 0 && (d / 256) * m_tiles >= sms;
-    const int bn = wide ? 256 : 128;
+    // Y = Z W_2^T + b_2
+    int bn = 128, splits = 1;
+    gemm2_plan(S, d, &bn, &splits);
     CUtensorMap mz, md;
     if (!make_map(&mz, z, S, d_ff, TC_BM) || !make_map(&md, w->w_down, d, d_ff, bn)) return GRIFFIN_ERR_CUDA;
     TcParams q = {};
@@ -397,11 +443,18 @@ griffin_status launch_prefill_tc(const griffin_ff_desc *desc, const griffin_ff_w
     q.K = d_ff;
     q.m_tiles = m_tiles;
     q.n_tiles = d / bn;
-    q.bias0 = static_cast<const __nv_bfloat16 *>(w->b_down);
+    q.bias0 = splits > 1 ? nullptr : static_cast<const __nv_bfloat16 *>(w->b_down);
     q.out = static_cast<__nv_bfloat16 *>(y);
     q.act = desc->act;
     q.ws = ws;
-    return wide ? launch_tc<false, 256>(mz, md, md, q, sms, stream) : launch_tc<false, 128>(mz, md, md, q, sms, stream);
+    q.splits = splits;
+    q.part = splits > 1 ? ypart : nullptr;
+    st = bn == 256 ? launch_tc<false, 256>(mz, md, md, q, sms, stream) : launch_tc<false, 128>(mz, md, md, q, sms, stream);
+    if (st != GRIFFIN_OK || splits == 1) return st;
+    const size_t n_elems = (size_t)S * d;
+    splitk_reduce_kernel<<<(unsigned)((n_elems / 4 + 255) / 256), 256, 0, stream>>>(
+        ypart, static_cast<const __nv_bfloat16 *>(w->b_down), static_cast<__nv_bfloat16 *>(y), splits, n_elems, d);
+    return cudaGetLastError() == cudaSuccess ? GRIFFIN_OK : GRIFFIN_ERR_CUDA;
 }
 
 }  // namespace griffin

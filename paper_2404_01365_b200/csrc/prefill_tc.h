@@ -8,13 +8,18 @@
 
 namespace griffin {
 
+// Tiling of the down projection Y = Z W_2^T for S tokens: tile width (128 or 256 outputs) and the
+// number of K splits (1..4; more than one when whole tiles would leave most SMs idle).  Pure
+// arithmetic on the shape, so that workspace sizing and launch agree.
+void gemm2_plan(int S, int d, int *bn, int *splits);
+
 // Whether the tensor-core kernels take this shape (bf16, d and d_ff multiples of 64, ...).
 bool prefill_tc_supported(const griffin_ff_desc *desc, int S);
 
 // Steps 1 and 2 of the prompt phase: writes Z (bf16), its fp32 copy zf and the per-tile partial
 // row sums of squares rowsq [S, *n_col_tiles]; writes Y unless y is NULL.
 griffin_status launch_prefill_tc(const griffin_ff_desc *desc, const griffin_ff_weights *w, const void *x, int S,
-                                 void *y, __nv_bfloat16 *z, float *zf, float *rowsq, int *n_col_tiles, void *ws,
+                                 void *y, __nv_bfloat16 *z, float *zf, float *rowsq, float *ypart, int *n_col_tiles, void *ws,
                                  cudaStream_t stream);
 
 }  // namespace griffin
