@@ -167,7 +167,9 @@ griffin_status griffin_compact_experts(const griffin_ff_desc *desc, const griffi
  * sets: HOST array of B structs (entries may repeat to share a set); every set must have
  * the same k and ldk.  b_down [d] or NULL is shared by all sequences.  x [B, d] in,
  * y [B, d] out.  1 <= B <= GRIFFIN_MAX_BATCH, d <= GRIFFIN_MAX_D.  flags: GRIFFIN_DECODE_*.
- * The activations z_hat [B, ldk] live in the workspace as fp32 between the two kernels. */
+ * The activations z_hat [B, ldk] pass through the workspace (4 bytes per entry).  With bf16
+ * storage the call is one kernel whose CTAs (one per SM) meet half-way through a counter in
+ * the workspace header: run it on a GPU whose SMs it can all occupy. */
 griffin_status griffin_ff_decode(const griffin_ff_desc *desc, int32_t B,
                                  const griffin_ff_compact *sets /*host*/, const void *b_down,
                                  const void *x, void *y, void *workspace, size_t ws_bytes,

@@ -1,12 +1,17 @@
-// Generation-phase pruned FF (Eqs. 4 and 5 of the GRIFFIN paper) for bf16 storage.
+// Generation-phase pruned FF (Eqs. 4 and 5 of the GRIFFIN paper) for bf16 storage, as ONE kernel
+// per call:
+//   first half   z_hat = sigma(W_g_hat x + b_g_hat) * (W_1_hat x + b_1_hat)
+//   meeting      every CTA has written its z entries; all CTAs wait for each other (bounded)
+//   second half  y_hat = W_2_hat z_hat + b_2
 //
-// Same pipeline as the fp32-FMA kernels (persistent CTA per SM, producer warp streaming
-// weight rows into a ring of shared-memory stages with 1-D bulk copies, 8 consumer warps,
-// programmatic dependent launch), but the consumers hand the staged rows to the warp-level
-// tensor-core instruction mma.sync.m16n8k16 instead of unpacking and multiplying element by
-// element.  The products are matrix-vector products, so this is not about FLOPs: it cuts the
-// instructions issued per staged byte several times over, which is what kept the FMA version
-// from reaching HBM speed.
+// One persistent CTA per SM.  A producer warp streams weight rows into a ring of
+// shared-memory stages with 1-D bulk copies (TMA, no multicast) tracked by mbarriers; it
+// touches weights only, so it runs ahead of the previous kernel on the stream (programmatic
+// dependent launch) and of the meeting point.  Eight consumer warps, in two groups that take
+// alternate stages, hand the staged rows to the warp-level tensor-core instruction
+// mma.sync.m16n8k16 instead of unpacking and multiplying element by element.  The products are
+// matrix-vector products, so this is not about FLOPs: it cuts the instructions issued per
+// staged byte several times over, which is what kept an FMA version from reaching HBM speed.
 //
 // Stages are made of few, large, contiguous copies (measured on B200: every bulk copy costs
 // about 30 ns of issue time and every stage hand-over about 240 ns, whatever their size, so
@@ -29,10 +34,10 @@
 //   * C[m][n] pairs virtual row m with virtual vector n; only the diagonal m = n belongs to
 //     the dot product.  Lane (g, t = g / 2) holds it; three shuffles add the 8 diagonal
 //     entries.  The tensor core does 8x the needed multiplies, which is free here.
-//   * down: z is fp32; it is split into two bf16 numbers z_hi + z_lo and each block runs the
-//     MMAs once against each, into the same accumulators, so 16 bits of z survive.
-//   * 8 / R warps share a pair; their partial sums meet in shared memory at the end of a
-//     work item, in a fixed order.
+//   * second half: z crosses as two bf16 numbers z_hi + z_lo per entry and each block runs
+//     the MMAs once against each, into the same accumulators, so 16 bits of z survive.
+//   * The 4 / R warps of a group share a pair; their partial sums meet in shared memory at
+//     the end of a work item, in a fixed order, so results are bitwise reproducible.
 #include "decode_common.cuh"
 
 namespace griffin {
