@@ -123,6 +123,8 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, vo
                                               int where) {
     // Fast path: plain polling.  The clock is only consulted every few thousand polls, so a
     // wait that succeeds (every wait of a healthy run) never pays for reading it.
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort) return false;
 #pragma unroll 1
     for (int i = 0; i < 4096; ++i)
         if (mbar_try_wait(bar, parity)) return true;

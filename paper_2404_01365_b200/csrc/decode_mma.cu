@@ -44,7 +44,10 @@ namespace griffin {
 
 constexpr int DEC_GROUP_WARPS = 4;           // consumer warps per group (two groups)
 constexpr int MMA_CHUNK_UNITS_MAX = 1024;  // 16 KB of one row per stage at most
-constexpr int MMA_STAGE_TARGET = 32 * 1024;
+#ifndef GRIFFIN_DEC_STAGE_KB
+#define GRIFFIN_DEC_STAGE_KB 32
+#endif
+constexpr int MMA_STAGE_TARGET = GRIFFIN_DEC_STAGE_KB * 1024;
 #ifndef GRIFFIN_DEC_SMEM_KB
 #define GRIFFIN_DEC_SMEM_KB 200
 #endif
@@ -256,6 +259,11 @@ __device__ __forceinline__ bool produce_half(const DecodeParams &p, const MmaPla
     return true;
 }
 
+// barrier among the 128 threads of one consumer group (ids 2 and 3; 0 is __syncthreads, 1 all consumers)
+__device__ __forceinline__ void group_barrier(int group) {
+    asm volatile("bar.sync %0, %1;" ::"r"(2 + group), "n"(DEC_GROUP_WARPS * 32) : "memory");
+}
+
 // Consumer side of one half (all 8 consumer warps).  Returns false after a give-up.
 template <bool DOWN>
 __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPlan &pl, const MmaSmem &s, int n_stages,
@@ -279,8 +287,11 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
         const int r1 = (int)((long long)(sl + 1) * total_rows / n_slices);
         const int n_pairs = DOWN ? (r1 - r0 + 1) / 2 : r1 - r0;
         float2 *part = s.part + item_parity * (DEC_MAX_ROWS * DEC_CONSUMER_WARPS);
+        const uint32_t pgc0 = pgc;  // pair-group count at the start of the item: who owns which pair
+        // the groups finish an item independently; before a further item (partial-sum buffers
+        // and the staged vector are about to be reused) they meet
+        if (item != (int)blockIdx.x) consumer_barrier();
         if (b != cur_b) {  // stage this sequence's vector in shared memory
-            if (cur_b >= 0) consumer_barrier();  // nobody still reads the previous one
             if (!DOWN) {
                 const uint4 *src =
                     reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(p.x) + (size_t)b * p.d);
@@ -303,8 +314,11 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
                 xr[i] = u < pl.row_units ? vec0[u] : make_uint4(0, 0, 0, 0);
             }
         }
-        bool ok = true;
-        for (int pg = 0; ok && pg < n_pairs; pg += pl.R, ++pgc) {
+        // After a give-up anywhere in the CTA the remaining work is skipped, but every barrier is
+        // still visited in the same order by both groups, so that nobody is left waiting.
+        bool ok = !*s.abort;
+        for (int pg = 0; pg < n_pairs; pg += pl.R, ++pgc) {
+            if (!ok) continue;
             if ((int)(pgc & 1) != group) continue;  // the other group's stage(s)
             const int ns2 = n_stages >> 1;
             const bool have = pg + my_pair < n_pairs;
@@ -334,10 +348,14 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
                 if (lane == 0) part[(pg + my_pair) * DEC_CONSUMER_WARPS + q] = d2;
             }
         }
-        consumer_barrier();
-        if (!ok || *s.abort) return false;
-        if (tid < r1 - r0) {
-            const int pair = DOWN ? tid >> 1 : tid;
+        group_barrier(group);  // this group's partial sums are in place
+        if (*s.abort) ok = false;
+        // every thread of the group looks after the rows of the pairs its group owned
+        const int tig = tid - group * (DEC_GROUP_WARPS * 32);
+        const int my_row = tig;  // rows of the item: r0 + my_row (at most DEC_MAX_ROWS of them)
+        const int my_rows_pair = DOWN ? my_row >> 1 : my_row;
+        if (ok && my_row < r1 - r0 && (int)((pgc0 + my_rows_pair / pl.R) & 1) == group) {
+            const int pair = my_rows_pair;
             float a0 = 0.f, a1 = 0.f;
             for (int w = 0; w < wpg; ++w) {
                 const float2 v = part[pair * DEC_CONSUMER_WARPS + w];
@@ -345,7 +363,7 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
                 a1 += v.y;
             }
             if (!DOWN) {
-                const int j = r0 + tid;
+                const int j = r0 + my_row;
                 if (p.seq[b].b_gate) a0 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[b].b_gate)[j]);
                 if (p.seq[b].b_up) a1 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[b].b_up)[j]);
                 // z leaves as two bf16 numbers, z_hi + z_lo, ready to be the down half's vector
@@ -354,8 +372,8 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
                 zbits[(size_t)b * 2 * p.ldk + j] = h;
                 zbits[(size_t)b * 2 * p.ldk + p.ldk + j] = __float2bfloat16_rn(zv - __bfloat162float(h));
             } else {
-                const int c = r0 + tid;
-                float acc = (tid & 1) ? a1 : a0;
+                const int c = r0 + my_row;
+                float acc = (my_row & 1) ? a1 : a0;
                 if (p.b_down) acc += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.b_down)[c]);
                 static_cast<__nv_bfloat16 *>(p.y)[(size_t)b * p.d + c] = __float2bfloat16_rn(acc);
             }
@@ -368,7 +386,7 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
             }
         }
     }
-    return true;
+    return !*s.abort;
 }
 
 __device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int *p) {
@@ -383,7 +401,7 @@ __device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int *p) {
 __device__ __forceinline__ bool grid_meet(WsHeader *h, unsigned int n_ctas, volatile int *abort, void *ws) {
     atomicAdd(&h->arrive, 1u);
     const long long t0 = clock64();
-    while (ld_acquire_u32(&h->arrive) < n_ctas) {
+    while (!*abort && ld_acquire_u32(&h->arrive) < n_ctas) {
         if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
             *abort = 1;
             raise_status(ws, DEV_STATUS_TIMEOUT, 9);
@@ -398,7 +416,10 @@ __device__ __forceinline__ bool grid_meet(WsHeader *h, unsigned int n_ctas, vola
     return true;
 }
 
-__global__ void __launch_bounds__(DEC_THREADS) decode_fused_kernel(const __grid_constant__ DecodeParams p,
+#ifndef GRIFFIN_DEC_MIN_CTAS
+#define GRIFFIN_DEC_MIN_CTAS 1
+#endif
+__global__ void __launch_bounds__(DEC_THREADS, GRIFFIN_DEC_MIN_CTAS) decode_fused_kernel(const __grid_constant__ DecodeParams p,
                                                                    const __grid_constant__ FusedPlan fp, int act) {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     const MmaSmem s = carve_fused(smem_raw, fp);
@@ -429,14 +450,13 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_fused_kernel(const __grid_
     pdl_wait_prior_grids();  // x, the z scratch and the outputs belong to earlier work on the stream
     uint32_t myit = 0, pgc = 0;  // stage uses of this warp's group; pair groups seen by everybody
     int item_parity = 0;
-    if (!consume_half<false>(p, fp.gu, s, fp.n_stages, fp.slot_bytes, p.n_slices, myit, pgc, item_parity, act, tid, warp,
-                             lane))
-        return;
-    __threadfence();  // this CTA's z entries are visible device-wide before it reports in
-    consumer_barrier();
-    if (tid == 0) grid_meet(static_cast<WsHeader *>(p.ws), gridDim.x, s.abort, p.ws);
-    consumer_barrier();
-    if (*s.abort) return;
+    consume_half<false>(p, fp.gu, s, fp.n_stages, fp.slot_bytes, p.n_slices, myit, pgc, item_parity, act, tid, warp, lane);
+    // each group reports on its own: 2 arrivals per CTA
+    const int group = warp / DEC_GROUP_WARPS;
+    __threadfence();  // this group's z entries are visible device-wide before it reports in
+    group_barrier(group);
+    if ((tid & (DEC_GROUP_WARPS * 32 - 1)) == 0) grid_meet(static_cast<WsHeader *>(p.ws), 2 * gridDim.x, s.abort, p.ws);
+    consumer_barrier();  // both groups have seen everybody: the staged vector may be replaced by z
     consume_half<true>(p, fp.dn, s, fp.n_stages, fp.slot_bytes, p.n_slices_dn, myit, pgc, item_parity, act, tid, warp,
                        lane);
 }
