@@ -203,3 +203,19 @@ def test_prefill_zero_row_contributes_nothing():
     _, z = O.ff_dense(np64(x), h64(host, "wg"), h64(host, "wu"), h64(host, "wd"), "swiglu")
     assert np.max(np.abs(s - O.flock_score(z))) < 1e-5
     assert torch.all(y[3] == 0)
+
+
+def test_device_status_word_is_decoded():
+    # what a kernel leaves in the workspace header after a bounded wait gave up, or after it met a
+    # bad expert index, comes back as a status code; re-initialising the workspace clears it
+    L, _ = make_layer(64, 96, "bf16")
+    hdr = L.ws[:16].view(torch.int32)
+    assert L.status() == G.OK
+    hdr[0] = 1
+    assert L.status() == G.ERR_TIMEOUT
+    hdr[0] = 2
+    assert L.status() == G.ERR_INVALID_ARG
+    hdr[0] = 77
+    assert L.status() == G.ERR_CUDA
+    G.griffin_workspace_init(L.ws)
+    assert L.status() == G.OK and int(hdr[2]) == 0 and int(hdr[3]) == 0
