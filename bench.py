@@ -207,7 +207,8 @@ def run_ours(args, w, keep):
         raise RuntimeError("bench.py needs a CUDA device: the path has no CPU fallback")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
+    use_dist = "RANK" in os.environ and "MASTER_ADDR" in os.environ   # launched by torch.distributed.run
+    if use_dist:
         dist.init_process_group("nccl", device_id=dev)
     G.load()
 
@@ -247,7 +248,7 @@ def run_ours(args, w, keep):
 
     def barrier():
         torch.cuda.synchronize()
-        if world > 1:
+        if use_dist:
             dist.barrier()
         torch.cuda.synchronize()
 
@@ -302,7 +303,7 @@ def run_ours(args, w, keep):
 
     # ---- max over ranks ----------------------------------------------------------------------
     vals = torch.tensor([total_ms] + phase_ms + ([e2e[0]] if e2e else [0.0]), device=dev, dtype=torch.float64)
-    if world > 1:
+    if use_dist:
         dist.all_reduce(vals, op=dist.ReduceOp.MAX)
     total_ms, phase_ms, e2e_ms = float(vals[0]), [float(v) for v in vals[1:5]], float(vals[5])
 
@@ -364,7 +365,7 @@ def run_ours(args, w, keep):
                 "sample": f"{blocks} of {L} blocks, each: prompt S={S}, top-k, slicing, {T_sample} of {T} decode steps, "
                           f"batch 1; numpy fp64; {sec:.1f} s"}
         print(json.dumps(line), flush=True)
-    if world > 1:
+    if use_dist:
         dist.destroy_process_group()
 
 
