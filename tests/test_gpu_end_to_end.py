@@ -112,3 +112,40 @@ def test_full_size_llama2_13b_block_batch8():
 def test_full_size_mistral_7b_block_keep_sweep(keep):
     w = synth.WORKLOADS["mistral_7b"]
     run_block(w, 0, keep, w.B, [0] if keep != 0.5 else [0, 3], _steps(w.T))
+
+
+def test_shared_expert_set_for_a_batch():
+    """Batched GRIFFIN as the paper extends it (Eq. 7): the samples' statistics are combined into
+    s_bar = sum_i s_i / sqrt(S_i), ONE expert set is selected and every sequence decodes with
+    it (the same compact set passed for each sequence of the decode call)."""
+    w = synth.scaled(synth.WORKLOADS["mistral_7b"], d=512, d_ff=1792, T=3)
+    lengths = [200, 64, 131, 17]
+    n_seq, k = len(lengths), G.griffin_k_from_keep_ratio(w.d_ff, 0.5)
+    wg, wu, wd = synth.make_weights(w, 0)
+    stack = FFStack(w.d, w.d_ff, w.act, w.dtype, 1, n_seq, max(lengths), k, dev())
+    stack.add_block(wg.to(dev()), wu.to(dev()), wd.to(dev()))
+    wg64, wu64, wd64 = np64(wg), np64(wu), np64(wd)
+    s_ref = []
+    for q, S in enumerate(lengths):
+        x = synth.make_prompt(w, 0, q, S=S)
+        y = torch.empty((S, w.d), device=dev(), dtype=w.torch_dtype)
+        stack.prefill_score(0, q, x.to(dev()), y)
+        _, z = O.ff_dense(np64(x), wg64, wu64, wd64, w.act)
+        s_ref.append(O.flock_score(z))
+    s_bar = torch.empty((w.d_ff,), device=dev(), dtype=torch.float32)
+    G.griffin_combine_scores(stack.score[0], lengths, s_bar)
+    s_bar_ref = O.combine_scores(s_ref, lengths)
+    assert np.max(np.abs(np64(s_bar) - s_bar_ref) / s_bar_ref) < 1e-4
+    e = torch.empty((k,), device=dev(), dtype=torch.int32)
+    G.griffin_select_topk(s_bar, k, e)
+    check_expert_set(e.cpu().numpy(), s_bar_ref, k)
+    shared = stack.sets[0][0]
+    G.griffin_compact_experts(stack.desc, stack.weights[0], e, shared, stack.ws)
+    xd = torch.stack([synth.make_decode_inputs(w, 0, q)[0] for q in range(n_seq)])
+    yd = torch.empty((n_seq, w.d), device=dev(), dtype=w.torch_dtype)
+    G.griffin_ff_decode(stack.desc, [shared] * n_seq, None, xd.to(dev()), yd, stack.ws)
+    assert stack.status() == G.OK
+    c = O.compact_experts(e.cpu().numpy(), wg64, wu64, wd64)
+    ref = O.ff_pruned(np64(xd), c, w.act)
+    for q in range(n_seq):
+        assert rel_l2(np64(yd[q]), ref[q]) < TOL_OUT[w.dtype]
