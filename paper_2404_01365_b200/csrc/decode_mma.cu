@@ -124,52 +124,87 @@ __device__ __forceinline__ float2 diagonal_sum(const float (&c)[4], int g, int t
     return make_float2(v0, v1);
 }
 
-// This warp's share of one pair's chunk: blocks q, q + wpg, ... of 32 units each, never more
-// than MMA_BLOCKS_PER_WARP of them (a stage holds at most 32 / R blocks per row and the 4 / R
-// warps of a consumer group share the pair).  They are taken in batches of four: all
+// This warp's share of one pair's chunk: blocks q, q + WPG, ... of 32 units each, never more
+// than MMA_BLOCKS_PER_WARP of them (a stage holds at most 32 / R blocks per row and the
+// WPG = 4 / R warps of a consumer group share the pair).  The kernel is bound by the number of
+// instructions its few warps can issue, so the common case is kept to the loads and the MMAs
+// themselves: blocks are taken in batches of four whole blocks with no predicates and
+// compile-time offsets from per-lane base pointers; only what is left after the last whole
+// batch (at most four blocks, the last of which may be cut short by the end of the row) takes
+// the guarded path, where lanes past the end supply zeros (stale bytes could be NaN).  All
 // shared-memory reads of a batch are issued before its first MMA, and the MMAs go to four
 // independent accumulators, so latencies overlap instead of adding up.
-//   row0,row1 : the two staged rows; vec0 : vector units for this chunk; vec1 : second vector
-//   (down's z_lo); xr : the vector's units held in registers (gate_up, where x is the same for
-//   every neuron of the item); n_units : valid units in this chunk
+//   p0, p1 : this lane's unit of the first block of the two staged rows; pv, pw : the same for
+//   the vector held in shared memory (down: z_hi and z_lo); xr : the vector's units held in
+//   registers (gate_up, where x is the same for every neuron of the item); my_full : whole
+//   blocks of this warp; tail_lanes : lanes with data in the block after them (0: no such block)
 constexpr int MMA_BLOCKS_PER_WARP = 8;
 constexpr int MMA_BATCH = 4;
 template <bool DOWN>
-__device__ __forceinline__ void pair_mma(float (&acc)[4][4], const uint4 *row0, const uint4 *row1, const uint4 *vec0,
-                                         const uint4 *vec1, const uint4 (&xr)[MMA_BLOCKS_PER_WARP], int n_units, int q,
-                                         int wpg, int lane) {
-    const uint4 zero = make_uint4(0, 0, 0, 0);
+__device__ __forceinline__ void block_mma(float (&acc)[4][4], int i, const uint4 &r0, const uint4 &r1, const uint4 &v,
+                                          const uint4 &w) {
+    mma_bf16(acc[(2 * i) & 3], r0.x, r1.x, r0.y, r1.y, v.x, v.y);
+    mma_bf16(acc[(2 * i + 1) & 3], r0.z, r1.z, r0.w, r1.w, v.z, v.w);
+    if (DOWN) {
+        mma_bf16(acc[(2 * i) & 3], r0.x, r1.x, r0.y, r1.y, w.x, w.y);
+        mma_bf16(acc[(2 * i + 1) & 3], r0.z, r1.z, r0.w, r1.w, w.z, w.w);
+    }
+}
+template <bool DOWN, int WPG>
+__device__ __forceinline__ void pair_mma(float (&acc)[4][4], const uint4 *p0, const uint4 *p1, const uint4 *pv,
+                                         const uint4 *pw, const uint4 (&xr)[MMA_BLOCKS_PER_WARP], int my_full,
+                                         int tail_lanes, int lane) {
+    constexpr int BS = WPG * 32;  // units between consecutive blocks of this warp
 #pragma unroll
     for (int b0 = 0; b0 < MMA_BLOCKS_PER_WARP; b0 += MMA_BATCH) {
-        if ((q + b0 * wpg) * 32 >= n_units) break;  // warp-uniform
         uint4 r0[MMA_BATCH], r1[MMA_BATCH], v[MMA_BATCH], w[MMA_BATCH];
+        if (b0 + MMA_BATCH <= my_full) {  // warp-uniform: four whole blocks
 #pragma unroll
-        for (int i = 0; i < MMA_BATCH; ++i) {
-            const int u = (q + (b0 + i) * wpg) * 32 + lane;  // a warp reads 512 contiguous bytes
-            r0[i] = zero; r1[i] = zero; v[i] = zero; w[i] = zero;
-            if (u < n_units) {  // past the end both operands are zero (stale bytes could be NaN)
-                r0[i] = row0[u];
-                r1[i] = row1[u];
+            for (int i = 0; i < MMA_BATCH; ++i) {
+                r0[i] = p0[(b0 + i) * BS];
+                r1[i] = p1[(b0 + i) * BS];
                 if (DOWN) {
-                    v[i] = vec0[u];
-                    w[i] = vec1[u];
+                    v[i] = pv[(b0 + i) * BS];
+                    w[i] = pw[(b0 + i) * BS];
                 } else {
                     v[i] = xr[b0 + i];
                 }
             }
-        }
 #pragma unroll
-        for (int i = 0; i < MMA_BATCH; ++i) {
-            if ((q + (b0 + i) * wpg) * 32 < n_units) {  // warp-uniform
-                mma_bf16(acc[(2 * i) & 3], r0[i].x, r1[i].x, r0[i].y, r1[i].y, v[i].x, v[i].y);
-                mma_bf16(acc[(2 * i + 1) & 3], r0[i].z, r1[i].z, r0[i].w, r1[i].w, v[i].z, v[i].w);
-                if (DOWN) {
-                    mma_bf16(acc[(2 * i) & 3], r0[i].x, r1[i].x, r0[i].y, r1[i].y, w[i].x, w[i].y);
-                    mma_bf16(acc[(2 * i + 1) & 3], r0[i].z, r1[i].z, r0[i].w, r1[i].w, w[i].z, w[i].w);
+            for (int i = 0; i < MMA_BATCH; ++i) block_mma<DOWN>(acc, i, r0[i], r1[i], v[i], DOWN ? w[i] : v[i]);
+        } else if (b0 == 0 || b0 <= my_full) {  // a shorter batch ends the warp's blocks
+            const int n = my_full - b0 + (tail_lanes > 0 ? 1 : 0);  // blocks left, the cut one included
+            if (n > 0) {
+                const uint4 zero = make_uint4(0, 0, 0, 0);
+#pragma unroll
+                for (int i = 0; i < MMA_BATCH; ++i) {
+                    r0[i] = zero; r1[i] = zero; v[i] = zero; w[i] = zero;
+                    if (i < n && (b0 + i < my_full || lane < tail_lanes)) {
+                        r0[i] = p0[(b0 + i) * BS];
+                        r1[i] = p1[(b0 + i) * BS];
+                        if (DOWN) {
+                            v[i] = pv[(b0 + i) * BS];
+                            w[i] = pw[(b0 + i) * BS];
+                        } else {
+                            v[i] = xr[b0 + i];
+                        }
+                    }
                 }
+#pragma unroll
+                for (int i = 0; i < MMA_BATCH; ++i)
+                    if (i < n) block_mma<DOWN>(acc, i, r0[i], r1[i], v[i], DOWN ? w[i] : v[i]);  // warp-uniform
             }
         }
     }
+}
+
+// Whole blocks of warp q (of WPG) among the blocks of a chunk of `units` units, and the lanes
+// with data in its cut block, if the chunk's cut block is this warp's.
+template <int WPG>
+__device__ __forceinline__ void my_blocks(int units, int q, int &my_full, int &tail_lanes) {
+    const int whole = units >> 5, rem = units & 31;
+    my_full = whole > q ? (whole - q + WPG - 1) / WPG : 0;
+    tail_lanes = (rem != 0 && (whole % WPG) == q) ? rem : 0;
 }
 
 __device__ __forceinline__ void producer_drain_mma(const MmaSmem &s, int n_stages, const uint32_t (&issued)[2]) {
@@ -186,6 +221,21 @@ __device__ __forceinline__ void producer_drain_mma(const MmaSmem &s, int n_stage
         }
     }
 }
+
+// Position of one consumer group in its half of the ring: the slot used next, how often the
+// half has been gone round (its low bit is the barrier parity) and the uses so far.
+struct RingPos {
+    int slot;
+    uint32_t round;
+    uint32_t uses;
+    __device__ __forceinline__ void advance(int ns2) {
+        ++uses;
+        if (++slot == ns2) {
+            slot = 0;
+            ++round;
+        }
+    }
+};
 
 // The two halves of a decode call share one kernel, one ring and one stage counter:
 //   DOWN = false: gate_up, z[b, j] = sigma(gate_j . x + b_gate_j) * (up_j . x + b_up_j);
@@ -213,9 +263,10 @@ __device__ __forceinline__ MmaSmem carve_fused(uint8_t *smem, const FusedPlan &f
 // Producer side of one half.  Lane l < 2R copies row (l & 1) of pair (l >> 1).  Weights only.
 template <bool DOWN>
 __device__ __forceinline__ bool produce_half(const DecodeParams &p, const MmaPlan &pl, const MmaSmem &s, int n_stages,
-                                             int slot_bytes, int n_slices, uint32_t (&itg)[2], uint32_t &pgc, int lane) {
+                                             int slot_bytes, int n_slices, RingPos (&pos)[2], uint32_t &pgc, int lane) {
     const int n_items = p.B * n_slices;
     const int total_rows = DOWN ? p.d : p.k;
+    const int ns2 = n_stages >> 1;
     const size_t row_bytes = (size_t)pl.row_units * 16;
     const int chunk_bytes_max = pl.chunk_units * 16;
     const int my_pair = lane >> 1, my_row = lane & 1;
@@ -232,28 +283,32 @@ __device__ __forceinline__ bool produce_half(const DecodeParams &p, const MmaPla
             // sequential user (a group skipping over the other's stages would otherwise wait on
             // a parity that an older phase already satisfies)
             const int grp = pgc & 1;
-            const int ns2 = n_stages >> 1;
             const int pair = pg + my_pair;
             const int grow = DOWN ? r0 + 2 * pair + my_row : r0 + pair;  // row in the matrix
             const bool mine = lane < 2 * pl.R && pair < n_pairs && grow < r1;
             // rows copied in this stage (the same for every chunk of the group)
             const int rows_in_stage = DOWN ? min(2 * pl.R, r1 - r0 - 2 * pg) : 2 * min(pl.R, n_pairs - pg);
-            for (int c = 0; c < pl.n_chunks; ++c, ++itg[grp]) {
+            RingPos cur = grp ? pos[1] : pos[0];  // (constant indices keep both in registers)
+            for (int c = 0; c < pl.n_chunks; ++c, cur.advance(ns2)) {
                 const int units = min(pl.chunk_units, pl.row_units - c * pl.chunk_units);
-                const int stage = grp * ns2 + (int)(itg[grp] % ns2);
-                const uint32_t use = itg[grp] / ns2;
+                const int stage = grp * ns2 + cur.slot;
+                const uint32_t use = cur.round;
                 int go = 1;
                 if (lane == 0) {
                     if (use > 0 && !wait_or_abort(&s.empty[stage], (use - 1) & 1, s.abort, p.ws, DOWN ? 7 : 5)) go = 0;
                     if (go) mbar_arrive_expect_tx(&s.full[stage], (uint32_t)(rows_in_stage * units * 16));
                 }
                 go = __shfl_sync(0xffffffffu, go, 0);
-                if (!go) return false;
+                if (!go) {
+                    if (grp) pos[1] = cur; else pos[0] = cur;
+                    return false;
+                }
                 if (mine)
                     bulk_g2s(s.stages + (size_t)stage * slot_bytes + (size_t)lane * chunk_bytes_max,
                              mat + (size_t)grow * row_bytes + (size_t)c * chunk_bytes_max, (uint32_t)units * 16,
                              &s.full[stage]);
             }
+            if (grp) pos[1] = cur; else pos[0] = cur;
         }
     }
     return true;
@@ -265,9 +320,9 @@ __device__ __forceinline__ void group_barrier(int group) {
 }
 
 // Consumer side of one half (all 8 consumer warps).  Returns false after a give-up.
-template <bool DOWN>
+template <bool DOWN, int WPG>
 __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPlan &pl, const MmaSmem &s, int n_stages,
-                                             int slot_bytes, int n_slices, uint32_t &myit, uint32_t &pgc,
+                                             int slot_bytes, int n_slices, RingPos &pos, uint32_t &pgc,
                                              int &item_parity, int act, int tid, int warp, int lane) {
     const int n_items = p.B * n_slices;
     const int total_rows = DOWN ? p.d : p.k;
@@ -275,9 +330,14 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
     // The 8 consumer warps form two groups of 4 that take alternate stages (pair groups), so
     // that one group's waiting, shuffling and hand-back overlaps the other group's reads.
     const int group = warp / DEC_GROUP_WARPS, wig = warp - group * DEC_GROUP_WARPS;
-    const int wpg = DEC_GROUP_WARPS / pl.R;  // warps of a group per pair
+    constexpr int wpg = WPG;  // warps of a group per pair (4 / R)
+    const int ns2 = n_stages >> 1;
     const int g = lane >> 2, t = lane & 3;
     const int my_pair = wig / wpg, q = wig - my_pair * wpg;
+    // this lane's unit of this warp's first block, within a staged row and within the vector
+    const int lane_unit = q * 32 + lane;
+    int my_full, tail_lanes;  // this warp's blocks of a chunk (all chunks but a row's last are alike)
+    my_blocks<WPG>(pl.chunk_units, q, my_full, tail_lanes);
     // the scratch holds, per sequence, z_hi [ldk] then z_lo [ldk] in bf16 (same bytes as fp32 [ldk])
     __nv_bfloat16 *zbits = reinterpret_cast<__nv_bfloat16 *>(p.z);
     int cur_b = -1;
@@ -320,22 +380,24 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
         for (int pg = 0; pg < n_pairs; pg += pl.R, ++pgc) {
             if (!ok) continue;
             if ((int)(pgc & 1) != group) continue;  // the other group's stage(s)
-            const int ns2 = n_stages >> 1;
             const bool have = pg + my_pair < n_pairs;
             float acc[4][4] = {};
-            for (int c = 0; c < pl.n_chunks; ++c, ++myit) {
-                const int stage = group * ns2 + (int)(myit % ns2);  // this group's half of the ring
-                if (!wait_or_abort(&s.full[stage], (myit / ns2) & 1, s.abort, p.ws, DOWN ? 8 : 6)) {
+            if (pl.n_chunks > 1) my_blocks<WPG>(pl.chunk_units, q, my_full, tail_lanes);
+            for (int c = 0; c < pl.n_chunks; ++c, pos.advance(ns2)) {
+                const int stage = group * ns2 + pos.slot;  // this group's half of the ring
+                if (!wait_or_abort(&s.full[stage], pos.round & 1, s.abort, p.ws, DOWN ? 8 : 6)) {
                     ok = false;
                     break;
                 }
                 if (have) {
-                    const int units = min(pl.chunk_units, pl.row_units - c * pl.chunk_units);
-                    const uint4 *row0 = reinterpret_cast<const uint4 *>(s.stages + (size_t)stage * slot_bytes +
-                                                                        (size_t)(2 * my_pair) * chunk_bytes_max);
-                    const uint4 *row1 = row0 + pl.chunk_units;
-                    pair_mma<DOWN>(acc, row0, row1, vec0 + c * pl.chunk_units, vec1 + c * pl.chunk_units, xr, units, q,
-                                   wpg, lane);
+                    if (c == pl.n_chunks - 1 && c > 0)  // a long row's last chunk may be shorter
+                        my_blocks<WPG>(pl.row_units - c * pl.chunk_units, q, my_full, tail_lanes);
+                    const uint4 *p0 = reinterpret_cast<const uint4 *>(s.stages + (size_t)stage * slot_bytes +
+                                                                      (size_t)(2 * my_pair) * chunk_bytes_max) +
+                                      lane_unit;
+                    const uint4 *pv = vec0 + c * pl.chunk_units + lane_unit;
+                    pair_mma<DOWN, WPG>(acc, p0, p0 + pl.chunk_units, pv, pv + pl.row_units, xr, my_full, tail_lanes,
+                                        lane);
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&s.empty[stage]);
@@ -439,26 +501,36 @@ __global__ void __launch_bounds__(DEC_THREADS, GRIFFIN_DEC_MIN_CTAS) decode_fuse
         // ---- producer warp: weights only, so it never waits for the previous grid, nor for
         //      the meeting point: the first stages of W_2_hat are on their way while the
         //      consumers are still waiting for the other CTAs' z
-        uint32_t itg[2] = {0, 0}, pgc = 0;
-        if (produce_half<false>(p, fp.gu, s, fp.n_stages, fp.slot_bytes, p.n_slices, itg, pgc, lane))
-            produce_half<true>(p, fp.dn, s, fp.n_stages, fp.slot_bytes, p.n_slices_dn, itg, pgc, lane);
-        if (lane == 0) producer_drain_mma(s, fp.n_stages, itg);
+        RingPos pos[2] = {{0, 0, 0}, {0, 0, 0}};
+        uint32_t pgc = 0;
+        if (produce_half<false>(p, fp.gu, s, fp.n_stages, fp.slot_bytes, p.n_slices, pos, pgc, lane))
+            produce_half<true>(p, fp.dn, s, fp.n_stages, fp.slot_bytes, p.n_slices_dn, pos, pgc, lane);
+        const uint32_t issued[2] = {pos[0].uses, pos[1].uses};
+        if (lane == 0) producer_drain_mma(s, fp.n_stages, issued);
         return;
     }
 
     // ---- consumers
     pdl_wait_prior_grids();  // x, the z scratch and the outputs belong to earlier work on the stream
-    uint32_t myit = 0, pgc = 0;  // stage uses of this warp's group; pair groups seen by everybody
+    RingPos pos = {0, 0, 0};  // of this warp's group
+    uint32_t pgc = 0;         // pair groups seen by everybody
     int item_parity = 0;
-    consume_half<false>(p, fp.gu, s, fp.n_stages, fp.slot_bytes, p.n_slices, myit, pgc, item_parity, act, tid, warp, lane);
+    switch (fp.gu.R) {  // warps per pair as a compile-time constant: block offsets become immediates
+        case 4: consume_half<false, 1>(p, fp.gu, s, fp.n_stages, fp.slot_bytes, p.n_slices, pos, pgc, item_parity, act, tid, warp, lane); break;
+        case 2: consume_half<false, 2>(p, fp.gu, s, fp.n_stages, fp.slot_bytes, p.n_slices, pos, pgc, item_parity, act, tid, warp, lane); break;
+        default: consume_half<false, 4>(p, fp.gu, s, fp.n_stages, fp.slot_bytes, p.n_slices, pos, pgc, item_parity, act, tid, warp, lane); break;
+    }
     // each group reports on its own: 2 arrivals per CTA
     const int group = warp / DEC_GROUP_WARPS;
     __threadfence();  // this group's z entries are visible device-wide before it reports in
     group_barrier(group);
     if ((tid & (DEC_GROUP_WARPS * 32 - 1)) == 0) grid_meet(static_cast<WsHeader *>(p.ws), 2 * gridDim.x, s.abort, p.ws);
     consumer_barrier();  // both groups have seen everybody: the staged vector may be replaced by z
-    consume_half<true>(p, fp.dn, s, fp.n_stages, fp.slot_bytes, p.n_slices_dn, myit, pgc, item_parity, act, tid, warp,
-                       lane);
+    switch (fp.dn.R) {
+        case 4: consume_half<true, 1>(p, fp.dn, s, fp.n_stages, fp.slot_bytes, p.n_slices_dn, pos, pgc, item_parity, act, tid, warp, lane); break;
+        case 2: consume_half<true, 2>(p, fp.dn, s, fp.n_stages, fp.slot_bytes, p.n_slices_dn, pos, pgc, item_parity, act, tid, warp, lane); break;
+        default: consume_half<true, 4>(p, fp.dn, s, fp.n_stages, fp.slot_bytes, p.n_slices_dn, pos, pgc, item_parity, act, tid, warp, lane); break;
+    }
 }
 
 griffin_status decode_bf16_mma(DecodeParams &p, int act, uint32_t flags, cudaStream_t stream) {
