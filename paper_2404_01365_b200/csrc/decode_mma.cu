@@ -49,7 +49,7 @@ constexpr int MMA_CHUNK_UNITS_MAX = 1024;  // 16 KB of one row per stage at most
 #endif
 constexpr int MMA_STAGE_TARGET = GRIFFIN_DEC_STAGE_KB * 1024;
 #ifndef GRIFFIN_DEC_SMEM_KB
-#define GRIFFIN_DEC_SMEM_KB 200
+#define GRIFFIN_DEC_SMEM_KB 227
 #endif
 constexpr int MMA_SMEM_TARGET = GRIFFIN_DEC_SMEM_KB * 1024;  // shared memory the ring, the vector and the rest may take
 
@@ -106,22 +106,25 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// Adds the diagonal of the 16 x 8 accumulator tile: returns (sum over g of C[g][g],
-// sum over g of C[g + 8][g]) in lane 0.  Lane (g, t) holds columns 2t, 2t+1 of rows g, g+8.
-__device__ __forceinline__ float2 diagonal_sum(const float (&c)[4], int g, int t) {
+// Adds the diagonal of the 16 x 8 accumulator tile: the sum over g of C[g][g] ends up in lane
+// 0 and the sum over g of C[g + 8][g] in lane 4 (the value returned by other lanes means
+// nothing).  Lane (g, t) holds columns 2t, 2t+1 of rows g, g+8, so the 8 lanes that hold a
+// diagonal entry are 0, 4, 9, 13, 18, 22, 27, 31.  In the first exchange (xor 4) the lower
+// lane of each couple hands over its second-row entry and takes the partner's first-row
+// entry, so that from then on each lane carries one sum and three shuffles do for both rows.
+__device__ __forceinline__ float diagonal_sum(const float (&c)[4], int lane) {
+    const int g = lane >> 2, t = lane & 3;
     float v0 = 0.f, v1 = 0.f;
     if (t == (g >> 1)) {
         v0 = (g & 1) ? c[1] : c[0];
         v1 = (g & 1) ? c[3] : c[2];
     }
-    // the 8 lanes that hold a diagonal entry are 0, 4, 9, 13, 18, 22, 27, 31
-    v0 += __shfl_xor_sync(0xffffffffu, v0, 4);
-    v1 += __shfl_xor_sync(0xffffffffu, v1, 4);
-    v0 += __shfl_xor_sync(0xffffffffu, v0, 9);
-    v1 += __shfl_xor_sync(0xffffffffu, v1, 9);
-    v0 += __shfl_xor_sync(0xffffffffu, v0, 18);
-    v1 += __shfl_xor_sync(0xffffffffu, v1, 18);
-    return make_float2(v0, v1);
+    const bool lower = (lane & 4) == 0;
+    const float got = __shfl_xor_sync(0xffffffffu, lower ? v1 : v0, 4);
+    float v = (lower ? v0 : v1) + got;
+    v += __shfl_xor_sync(0xffffffffu, v, 9);
+    v += __shfl_xor_sync(0xffffffffu, v, 18);
+    return v;
 }
 
 // This warp's share of one pair's chunk: blocks q, q + WPG, ... of 32 units each, never more
@@ -139,21 +142,40 @@ __device__ __forceinline__ float2 diagonal_sum(const float (&c)[4], int g, int t
 //   registers (gate_up, where x is the same for every neuron of the item); my_full : whole
 //   blocks of this warp; tail_lanes : lanes with data in the block after them (0: no such block)
 constexpr int MMA_BLOCKS_PER_WARP = 8;
-constexpr int MMA_BATCH = 4;
-template <bool DOWN>
-__device__ __forceinline__ void block_mma(float (&acc)[4][4], int i, const uint4 &r0, const uint4 &r1, const uint4 &v,
-                                          const uint4 &w) {
-    mma_bf16(acc[(2 * i) & 3], r0.x, r1.x, r0.y, r1.y, v.x, v.y);
-    mma_bf16(acc[(2 * i + 1) & 3], r0.z, r1.z, r0.w, r1.w, v.z, v.w);
+#ifndef GRIFFIN_DEC_BATCH
+#define GRIFFIN_DEC_BATCH 4
+#endif
+#ifndef GRIFFIN_DEC_ACCS
+#define GRIFFIN_DEC_ACCS 8
+#endif
+constexpr int MMA_BATCH = GRIFFIN_DEC_BATCH;
+constexpr int MMA_ACCS = GRIFFIN_DEC_ACCS;  // independent accumulators: an MMA never waits for the one issued just before it
+// The MMAs of one batch: first every block against v, then (down) every block against w, so
+// that two MMAs into the same accumulator are MMA_ACCS instructions apart.
+template <bool DOWN, int N>
+__device__ __forceinline__ void batch_mma(float (&acc)[MMA_ACCS][4], const uint4 (&r0)[MMA_BATCH],
+                                          const uint4 (&r1)[MMA_BATCH], const uint4 (&v)[MMA_BATCH],
+                                          const uint4 (&w)[MMA_BATCH]) {
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        mma_bf16(acc[(2 * i) & (MMA_ACCS - 1)], r0[i].x, r1[i].x, r0[i].y, r1[i].y, v[i].x, v[i].y);
+        mma_bf16(acc[(2 * i + 1) & (MMA_ACCS - 1)], r0[i].z, r1[i].z, r0[i].w, r1[i].w, v[i].z, v[i].w);
+    }
     if (DOWN) {
-        mma_bf16(acc[(2 * i) & 3], r0.x, r1.x, r0.y, r1.y, w.x, w.y);
-        mma_bf16(acc[(2 * i + 1) & 3], r0.z, r1.z, r0.w, r1.w, w.z, w.w);
+#pragma unroll
+        for (int i = 0; i < N; ++i) {
+            mma_bf16(acc[(2 * i) & (MMA_ACCS - 1)], r0[i].x, r1[i].x, r0[i].y, r1[i].y, w[i].x, w[i].y);
+            mma_bf16(acc[(2 * i + 1) & (MMA_ACCS - 1)], r0[i].z, r1[i].z, r0[i].w, r1[i].w, w[i].z, w[i].w);
+        }
     }
 }
-template <bool DOWN, int WPG>
-__device__ __forceinline__ void pair_mma(float (&acc)[4][4], const uint4 *p0, const uint4 *p1, const uint4 *pv,
-                                         const uint4 *pw, const uint4 (&xr)[MMA_BLOCKS_PER_WARP], int my_full,
-                                         int tail_lanes, int lane) {
+// VREG: the vector's units come from the registers xr (and wr for down's z_lo) instead of
+// shared memory.
+template <bool DOWN, bool VREG, int WPG>
+__device__ __forceinline__ void pair_mma(float (&acc)[MMA_ACCS][4], const uint4 *p0, const uint4 *p1, const uint4 *pv,
+                                         const uint4 *pw, const uint4 (&xr)[MMA_BLOCKS_PER_WARP],
+                                         const uint4 (&wr)[MMA_BLOCKS_PER_WARP], int my_full, int tail_lanes,
+                                         int lane) {
     constexpr int BS = WPG * 32;  // units between consecutive blocks of this warp
 #pragma unroll
     for (int b0 = 0; b0 < MMA_BLOCKS_PER_WARP; b0 += MMA_BATCH) {
@@ -163,36 +185,42 @@ __device__ __forceinline__ void pair_mma(float (&acc)[4][4], const uint4 *p0, co
             for (int i = 0; i < MMA_BATCH; ++i) {
                 r0[i] = p0[(b0 + i) * BS];
                 r1[i] = p1[(b0 + i) * BS];
-                if (DOWN) {
-                    v[i] = pv[(b0 + i) * BS];
-                    w[i] = pw[(b0 + i) * BS];
-                } else {
+                if (VREG) {
                     v[i] = xr[b0 + i];
+                    if (DOWN) w[i] = wr[b0 + i];
+                } else {
+                    v[i] = pv[(b0 + i) * BS];
+                    if (DOWN) w[i] = pw[(b0 + i) * BS];
                 }
             }
-#pragma unroll
-            for (int i = 0; i < MMA_BATCH; ++i) block_mma<DOWN>(acc, i, r0[i], r1[i], v[i], DOWN ? w[i] : v[i]);
+            batch_mma<DOWN, MMA_BATCH>(acc, r0, r1, v, w);
         } else if (b0 == 0 || b0 <= my_full) {  // a shorter batch ends the warp's blocks
             const int n = my_full - b0 + (tail_lanes > 0 ? 1 : 0);  // blocks left, the cut one included
             if (n > 0) {
                 const uint4 zero = make_uint4(0, 0, 0, 0);
 #pragma unroll
                 for (int i = 0; i < MMA_BATCH; ++i) {
-                    r0[i] = zero; r1[i] = zero; v[i] = zero; w[i] = zero;
-                    if (i < n && (b0 + i < my_full || lane < tail_lanes)) {
+                    if (b0 + i >= my_full) {  // warp-uniform: only the cut block needs zeros
+                        r0[i] = zero; r1[i] = zero; v[i] = zero; w[i] = zero;
+                    }
+                    if (b0 + i < my_full || (i < n && lane < tail_lanes)) {
                         r0[i] = p0[(b0 + i) * BS];
                         r1[i] = p1[(b0 + i) * BS];
-                        if (DOWN) {
+                        if (!VREG) {
                             v[i] = pv[(b0 + i) * BS];
-                            w[i] = pw[(b0 + i) * BS];
-                        } else {
-                            v[i] = xr[b0 + i];
+                            if (DOWN) w[i] = pw[(b0 + i) * BS];
                         }
                     }
+                    if (VREG) {  // (zero past the end of the row)
+                        v[i] = xr[b0 + i];
+                        if (DOWN) w[i] = wr[b0 + i];
+                    }
                 }
-#pragma unroll
-                for (int i = 0; i < MMA_BATCH; ++i)
-                    if (i < n) block_mma<DOWN>(acc, i, r0[i], r1[i], v[i], DOWN ? w[i] : v[i]);  // warp-uniform
+                // warp-uniform
+                if (n == 1) batch_mma<DOWN, 1>(acc, r0, r1, v, w);
+                else if (n == 2) batch_mma<DOWN, (2 < MMA_BATCH ? 2 : MMA_BATCH)>(acc, r0, r1, v, w);
+                else if (n == 3) batch_mma<DOWN, (3 < MMA_BATCH ? 3 : MMA_BATCH)>(acc, r0, r1, v, w);
+                else batch_mma<DOWN, MMA_BATCH>(acc, r0, r1, v, w);
             }
         }
     }
@@ -246,7 +274,7 @@ struct FusedPlan {
     MmaPlan gu, dn;   // per-half geometry (their n_stages / stage_bytes are overridden below)
     int slot_bytes;   // ring slot = the larger of the two halves' stages
     int n_stages;
-    int vec_bytes;    // the larger of x (d * 2) and z_hi | z_lo (ldk * 4)
+    int vec_bytes;    // z_hi | z_lo (ldk * 4) when it is staged in shared memory
 };
 
 __device__ __forceinline__ MmaSmem carve_fused(uint8_t *smem, const FusedPlan &fp) {
@@ -320,7 +348,11 @@ __device__ __forceinline__ void group_barrier(int group) {
 }
 
 // Consumer side of one half (all 8 consumer warps).  Returns false after a give-up.
-template <bool DOWN, int WPG>
+// VREG: a row is one chunk, so every stage of an item meets the same units of the vector and
+// each lane keeps its units of it in registers (read straight from global memory, once per
+// item); otherwise (rows longer than MMA_CHUNK_UNITS_MAX units, down only) the vector is
+// staged in shared memory and read from there block by block.
+template <bool DOWN, bool VREG, int WPG>
 __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPlan &pl, const MmaSmem &s, int n_stages,
                                              int slot_bytes, int n_slices, RingPos &pos, uint32_t &pgc,
                                              int &item_parity, int act, int tid, int warp, int lane) {
@@ -332,7 +364,6 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
     const int group = warp / DEC_GROUP_WARPS, wig = warp - group * DEC_GROUP_WARPS;
     constexpr int wpg = WPG;  // warps of a group per pair (4 / R)
     const int ns2 = n_stages >> 1;
-    const int g = lane >> 2, t = lane & 3;
     const int my_pair = wig / wpg, q = wig - my_pair * wpg;
     // this lane's unit of this warp's first block, within a staged row and within the vector
     const int lane_unit = q * 32 + lane;
@@ -341,6 +372,7 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
     // the scratch holds, per sequence, z_hi [ldk] then z_lo [ldk] in bf16 (same bytes as fp32 [ldk])
     __nv_bfloat16 *zbits = reinterpret_cast<__nv_bfloat16 *>(p.z);
     int cur_b = -1;
+    uint4 xr[MMA_BLOCKS_PER_WARP], wr[MMA_BLOCKS_PER_WARP];  // x, or z_hi and z_lo
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, item_parity ^= 1) {
         const int b = item / n_slices, sl = item - b * n_slices;
         const int r0 = (int)((long long)sl * total_rows / n_slices);
@@ -351,29 +383,28 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
         // the groups finish an item independently; before a further item (partial-sum buffers
         // and the staged vector are about to be reused) they meet
         if (item != (int)blockIdx.x) consumer_barrier();
-        if (b != cur_b) {  // stage this sequence's vector in shared memory
-            if (!DOWN) {
-                const uint4 *src =
-                    reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(p.x) + (size_t)b * p.d);
-                for (int v = tid; v < pl.row_units; v += DEC_CONSUMERS) reinterpret_cast<uint4 *>(s.vec)[v] = src[v];
-            } else {  // z_hi [ldk] then z_lo [ldk], written by other CTAs of this grid: read through L2
-                const uint4 *src = reinterpret_cast<const uint4 *>(zbits + (size_t)b * 2 * p.ldk);
-                for (int v = tid; v < 2 * pl.row_units; v += DEC_CONSUMERS)
+        if (b != cur_b) {  // this sequence's vector: x, or z_hi [ldk] then z_lo [ldk]
+            // (x was written by earlier work on the stream, z by other CTAs of this grid: both
+            // are read through L2)
+            const uint4 *src = DOWN ? reinterpret_cast<const uint4 *>(zbits + (size_t)b * 2 * p.ldk)
+                                    : reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(p.x) +
+                                                                      (size_t)b * p.d);
+            if (VREG) {
+                const uint4 zero = make_uint4(0, 0, 0, 0);
+#pragma unroll
+                for (int i = 0; i < MMA_BLOCKS_PER_WARP; ++i) {
+                    const int u = i * (WPG * 32) + lane_unit;
+                    xr[i] = u < pl.row_units ? __ldcg(src + u) : zero;
+                    if (DOWN) wr[i] = u < pl.row_units ? __ldcg(src + pl.row_units + u) : zero;
+                }
+            } else {
+                for (int v = tid; v < (DOWN ? 2 : 1) * pl.row_units; v += DEC_CONSUMERS)
                     reinterpret_cast<uint4 *>(s.vec)[v] = __ldcg(src + v);
+                consumer_barrier();
             }
-            consumer_barrier();
             cur_b = b;
         }
         const uint4 *vec0 = reinterpret_cast<const uint4 *>(s.vec);
-        const uint4 *vec1 = vec0 + pl.row_units;  // z_lo (down only)
-        uint4 xr[MMA_BLOCKS_PER_WARP];
-        if (!DOWN) {  // x does not change within the item: this lane's units of it stay in registers
-#pragma unroll
-            for (int i = 0; i < MMA_BLOCKS_PER_WARP; ++i) {
-                const int u = (q + i * wpg) * 32 + lane;
-                xr[i] = u < pl.row_units ? vec0[u] : make_uint4(0, 0, 0, 0);
-            }
-        }
         // After a give-up anywhere in the CTA the remaining work is skipped, but every barrier is
         // still visited in the same order by both groups, so that nobody is left waiting.
         bool ok = !*s.abort;
@@ -381,7 +412,7 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
             if (!ok) continue;
             if ((int)(pgc & 1) != group) continue;  // the other group's stage(s)
             const bool have = pg + my_pair < n_pairs;
-            float acc[4][4] = {};
+            float acc[MMA_ACCS][4] = {};
             if (pl.n_chunks > 1) my_blocks<WPG>(pl.chunk_units, q, my_full, tail_lanes);
             for (int c = 0; c < pl.n_chunks; ++c, pos.advance(ns2)) {
                 const int stage = group * ns2 + pos.slot;  // this group's half of the ring
@@ -396,8 +427,8 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
                                                                       (size_t)(2 * my_pair) * chunk_bytes_max) +
                                       lane_unit;
                     const uint4 *pv = vec0 + c * pl.chunk_units + lane_unit;
-                    pair_mma<DOWN, WPG>(acc, p0, p0 + pl.chunk_units, pv, pv + pl.row_units, xr, my_full, tail_lanes,
-                                        lane);
+                    pair_mma<DOWN, VREG, WPG>(acc, p0, p0 + pl.chunk_units, pv, pv + pl.row_units, xr, wr, my_full,
+                                              tail_lanes, lane);
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&s.empty[stage]);
@@ -405,9 +436,15 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
             if (ok && have) {
                 float sum[4];
 #pragma unroll
-                for (int e = 0; e < 4; ++e) sum[e] = (acc[0][e] + acc[1][e]) + (acc[2][e] + acc[3][e]);
-                const float2 d2 = diagonal_sum(sum, g, t);
-                if (lane == 0) part[(pg + my_pair) * DEC_CONSUMER_WARPS + q] = d2;
+                for (int e = 0; e < 4; ++e) {  // a fixed order: results are reproducible
+                    float lo = (acc[0][e] + acc[1][e]) + (acc[2][e] + acc[3][e]);
+                    if (MMA_ACCS == 8) lo += (acc[4 % MMA_ACCS][e] + acc[5 % MMA_ACCS][e]) + (acc[6 % MMA_ACCS][e] + acc[7 % MMA_ACCS][e]);
+                    sum[e] = lo;
+                }
+                const float dsum = diagonal_sum(sum, lane);
+                float *slot = reinterpret_cast<float *>(&part[(pg + my_pair) * DEC_CONSUMER_WARPS + q]);
+                if (lane == 0) slot[0] = dsum;  // first row of the pair
+                if (lane == 4) slot[1] = dsum;  // second row
             }
         }
         group_barrier(group);  // this group's partial sums are in place
@@ -515,10 +552,14 @@ __global__ void __launch_bounds__(DEC_THREADS, GRIFFIN_DEC_MIN_CTAS) decode_fuse
     RingPos pos = {0, 0, 0};  // of this warp's group
     uint32_t pgc = 0;         // pair groups seen by everybody
     int item_parity = 0;
-    switch (fp.gu.R) {  // warps per pair as a compile-time constant: block offsets become immediates
-        case 4: consume_half<false, 1>(p, fp.gu, s, fp.n_stages, fp.slot_bytes, p.n_slices, pos, pgc, item_parity, act, tid, warp, lane); break;
-        case 2: consume_half<false, 2>(p, fp.gu, s, fp.n_stages, fp.slot_bytes, p.n_slices, pos, pgc, item_parity, act, tid, warp, lane); break;
-        default: consume_half<false, 4>(p, fp.gu, s, fp.n_stages, fp.slot_bytes, p.n_slices, pos, pgc, item_parity, act, tid, warp, lane); break;
+#define GRIFFIN_CONSUME(DOWN_, VREG_, WPG_, PLAN_, SLICES_) \
+    consume_half<DOWN_, VREG_, WPG_>(p, PLAN_, s, fp.n_stages, fp.slot_bytes, SLICES_, pos, pgc, item_parity, act, tid, warp, lane)
+    // warps per pair as a compile-time constant: block offsets become immediates.  A row of
+    // W_g_hat or W_1_hat (d <= GRIFFIN_MAX_D elements) is always one chunk.
+    switch (fp.gu.R) {
+        case 4: GRIFFIN_CONSUME(false, true, 1, fp.gu, p.n_slices); break;
+        case 2: GRIFFIN_CONSUME(false, true, 2, fp.gu, p.n_slices); break;
+        default: GRIFFIN_CONSUME(false, true, 4, fp.gu, p.n_slices); break;
     }
     // each group reports on its own: 2 arrivals per CTA
     const int group = warp / DEC_GROUP_WARPS;
@@ -526,11 +567,17 @@ __global__ void __launch_bounds__(DEC_THREADS, GRIFFIN_DEC_MIN_CTAS) decode_fuse
     group_barrier(group);
     if ((tid & (DEC_GROUP_WARPS * 32 - 1)) == 0) grid_meet(static_cast<WsHeader *>(p.ws), 2 * gridDim.x, s.abort, p.ws);
     consumer_barrier();  // both groups have seen everybody: the staged vector may be replaced by z
-    switch (fp.dn.R) {
-        case 4: consume_half<true, 1>(p, fp.dn, s, fp.n_stages, fp.slot_bytes, p.n_slices_dn, pos, pgc, item_parity, act, tid, warp, lane); break;
-        case 2: consume_half<true, 2>(p, fp.dn, s, fp.n_stages, fp.slot_bytes, p.n_slices_dn, pos, pgc, item_parity, act, tid, warp, lane); break;
-        default: consume_half<true, 4>(p, fp.dn, s, fp.n_stages, fp.slot_bytes, p.n_slices_dn, pos, pgc, item_parity, act, tid, warp, lane); break;
+    if (fp.dn.n_chunks == 1) {
+        switch (fp.dn.R) {
+            case 4: GRIFFIN_CONSUME(true, true, 1, fp.dn, p.n_slices_dn); break;
+            case 2: GRIFFIN_CONSUME(true, true, 2, fp.dn, p.n_slices_dn); break;
+            default: GRIFFIN_CONSUME(true, true, 4, fp.dn, p.n_slices_dn); break;
+        }
+    } else {  // chunks of 8 KB or more: at most two pairs per stage
+        if (fp.dn.R == 2) GRIFFIN_CONSUME(true, false, 2, fp.dn, p.n_slices_dn);
+        else GRIFFIN_CONSUME(true, false, 4, fp.dn, p.n_slices_dn);
     }
+#undef GRIFFIN_CONSUME
 }
 
 griffin_status decode_bf16_mma(DecodeParams &p, int act, uint32_t flags, cudaStream_t stream) {
@@ -542,7 +589,7 @@ griffin_status decode_bf16_mma(DecodeParams &p, int act, uint32_t flags, cudaStr
     fp.gu = make_plan(p.d, p.d * 2);
     fp.dn = make_plan(p.ldk, p.ldk * 4);
     fp.slot_bytes = max(fp.gu.stage_bytes, fp.dn.stage_bytes);
-    fp.vec_bytes = max(p.d * 2, p.ldk * 4);
+    fp.vec_bytes = fp.dn.n_chunks > 1 ? p.ldk * 4 : 16;  // only rows of several chunks stage z in shared memory
     int n = ((int)MMA_SMEM_TARGET - fp.vec_bytes - (int)mma_fixed_smem(8)) / fp.slot_bytes;
     fp.n_stages = (n < 2 ? 2 : (n > 8 ? 8 : n)) & ~1;  // two halves, one per consumer group
     p.n_slices = slices_for(p.k, sms);
