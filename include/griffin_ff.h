@@ -106,6 +106,12 @@ typedef struct {
  * stream WRITES the compact weights this call reads (do not set it on the first decode
  * call after griffin_compact_experts). */
 #define GRIFFIN_DECODE_OVERLAP_WEIGHT_PREFETCH 1u
+/* bf16 only: use the tcgen05 kernel (the weights go from shared memory straight into the
+ * 5th-generation tensor cores) for shapes that it takes (d and ldk multiples of 128); other
+ * shapes, and calls without the flag, run the warp-level (mma.sync) kernel.  Results agree
+ * within the documented tolerance.  On the measured workloads the warp-level kernel is the
+ * faster of the two, which is why it is the default. */
+#define GRIFFIN_DECODE_TCGEN05 2u
 
 /* Status text for a code (static string, never NULL). */
 const char *griffin_status_string(griffin_status st);

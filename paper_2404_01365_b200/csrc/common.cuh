@@ -22,8 +22,8 @@ constexpr int DEV_STATUS_BAD_INDEX = 2;  // an expert index outside [0, d_ff)
 struct WsHeader {
     int status;           // DEV_STATUS_*
     int detail;           // where it happened (kernel-specific code)
-    unsigned int arrive;  // grid barrier of the fused decode kernel: CTAs that finished the first half
-    unsigned int depart;  // ... and CTAs that have seen everybody arrive (the last one resets both)
+    unsigned int meet_warp;  // meeting-point counter of the warp-level fused decode kernel (see grid_meet)
+    unsigned int meet_tc;    // ... and of the tcgen05 one (the two have different numbers of parties)
 };
 
 __device__ __forceinline__ void raise_status(void *ws, int status, int detail) {
@@ -133,6 +133,25 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, vo
 #pragma unroll 1
         for (int i = 0; i < 4096; ++i)
             if (mbar_try_wait(bar, parity)) return true;
+        if (*abort) return false;
+        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+            *abort = 1;
+            raise_status(ws, DEV_STATUS_TIMEOUT, where);
+            return false;
+        }
+    }
+}
+
+// The same for many threads that wait long (an epilogue waiting for a whole work item): they
+// sleep between polls, so that their polling does not take issue slots and shared-memory
+// cycles from the warps that do the work.
+__device__ __forceinline__ bool wait_or_abort_relaxed(uint64_t *bar, uint32_t parity, volatile int *abort, void *ws,
+                                                      int where) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+        __nanosleep(64);
+        if (mbar_try_wait(bar, parity)) return true;
         if (*abort) return false;
         if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
             *abort = 1;

@@ -1,4 +1,4 @@
-// Pieces shared by the two families of decode kernels (fp32-FMA and warp-MMA).
+// Pieces shared by the decode kernels (fp32-FMA, warp-MMA and tcgen05).
 #pragma once
 
 #include "common.cuh"
@@ -71,6 +71,36 @@ __device__ __forceinline__ void producer_drain(const DecSmem &s, int n_stages, u
 }
 
 
+__device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int *p) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Grid-wide meeting point between the two halves, called by one thread per arriving party
+// after the party's z entries have been written and are visible to this thread (a CTA-level
+// barrier is enough for that: the fence below is cumulative).  Every call of a kernel adds
+// n arrivals to a counter that runs round modulo 2 n and is never reset: a call whose
+// arrivals find it below n is complete when it reaches n, the next one when it wraps to 0.
+// (A party of the call after next cannot arrive before every party of this call has left:
+// all CTAs of a grid must be resident to meet, one per SM.)  Bounded: gives up after
+// WAIT_LIMIT_CYCLES.
+__device__ __forceinline__ bool grid_meet(unsigned int *counter, unsigned int n, volatile int *abort, void *ws) {
+    __threadfence();
+    const bool upper = atomicInc(counter, 2 * n - 1) >= n;
+    const long long t0 = clock64();
+    for (;;) {
+        const unsigned int v = ld_acquire_u32(counter);
+        if (upper ? v < n : v >= n) return true;
+        if (*abort) return false;
+        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+            *abort = 1;
+            raise_status(ws, DEV_STATUS_TIMEOUT, 9);
+            return false;
+        }
+    }
+}
+
 // Launches `func`, optionally allowing it to start before the previous kernel on the stream
 // has completed (programmatic dependent launch).
 cudaError_t launch_maybe_overlapped(const void *func, dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
@@ -82,5 +112,11 @@ int slices_for(int rows, int grid);
 
 // bf16 decode through warp-level MMA (decode_mma.cu).
 griffin_status decode_bf16_mma(DecodeParams &p, int act, uint32_t flags, cudaStream_t stream);
+
+// bf16 decode through tcgen05 (decode_tc.cu): at most DTC_MAX_B sequences, d and ldk multiples
+// of 64, a workspace for the meeting point.
+constexpr int DTC_MAX_B = 4;
+bool decode_tc_supported(const DecodeParams &p);
+griffin_status decode_bf16_tc(DecodeParams &p, int act, uint32_t flags, cudaStream_t stream);
 
 }  // namespace griffin

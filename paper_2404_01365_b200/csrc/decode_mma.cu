@@ -149,7 +149,15 @@ constexpr int MMA_BLOCKS_PER_WARP = 8;
 #define GRIFFIN_DEC_ACCS 8
 #endif
 constexpr int MMA_BATCH = GRIFFIN_DEC_BATCH;
-constexpr int MMA_ACCS = GRIFFIN_DEC_ACCS;  // independent accumulators: an MMA never waits for the one issued just before it
+constexpr int MMA_ACCS = GRIFFIN_DEC_ACCS;
+// Whether z crosses the halves as two bf16 numbers z_hi + z_lo per entry (every block of
+// W_2_hat then meets both, at twice the MMAs) or as one, rounded to bf16 like the Z that the
+// prompt-phase kernels hand to their second GEMM.  The second half is bound by its own
+// instructions, not by HBM, and the extra bits are below the rounding of the bf16 output.
+#ifndef GRIFFIN_DEC_Z_LO
+#define GRIFFIN_DEC_Z_LO 0
+#endif
+constexpr bool Z_LO = GRIFFIN_DEC_Z_LO != 0;  // independent accumulators: an MMA never waits for the one issued just before it
 // The MMAs of one batch: first every block against v, then (down) every block against w, so
 // that two MMAs into the same accumulator are MMA_ACCS instructions apart.
 template <bool DOWN, int N>
@@ -161,7 +169,7 @@ __device__ __forceinline__ void batch_mma(float (&acc)[MMA_ACCS][4], const uint4
         mma_bf16(acc[(2 * i) & (MMA_ACCS - 1)], r0[i].x, r1[i].x, r0[i].y, r1[i].y, v[i].x, v[i].y);
         mma_bf16(acc[(2 * i + 1) & (MMA_ACCS - 1)], r0[i].z, r1[i].z, r0[i].w, r1[i].w, v[i].z, v[i].w);
     }
-    if (DOWN) {
+    if (DOWN && Z_LO) {
 #pragma unroll
         for (int i = 0; i < N; ++i) {
             mma_bf16(acc[(2 * i) & (MMA_ACCS - 1)], r0[i].x, r1[i].x, r0[i].y, r1[i].y, w[i].x, w[i].y);
@@ -187,10 +195,10 @@ __device__ __forceinline__ void pair_mma(float (&acc)[MMA_ACCS][4], const uint4 
                 r1[i] = p1[(b0 + i) * BS];
                 if (VREG) {
                     v[i] = xr[b0 + i];
-                    if (DOWN) w[i] = wr[b0 + i];
+                    if (DOWN && Z_LO) w[i] = wr[b0 + i];
                 } else {
                     v[i] = pv[(b0 + i) * BS];
-                    if (DOWN) w[i] = pw[(b0 + i) * BS];
+                    if (DOWN && Z_LO) w[i] = pw[(b0 + i) * BS];
                 }
             }
             batch_mma<DOWN, MMA_BATCH>(acc, r0, r1, v, w);
@@ -208,12 +216,12 @@ __device__ __forceinline__ void pair_mma(float (&acc)[MMA_ACCS][4], const uint4 
                         r1[i] = p1[(b0 + i) * BS];
                         if (!VREG) {
                             v[i] = pv[(b0 + i) * BS];
-                            if (DOWN) w[i] = pw[(b0 + i) * BS];
+                            if (DOWN && Z_LO) w[i] = pw[(b0 + i) * BS];
                         }
                     }
                     if (VREG) {  // (zero past the end of the row)
                         v[i] = xr[b0 + i];
-                        if (DOWN) w[i] = wr[b0 + i];
+                        if (DOWN && Z_LO) w[i] = wr[b0 + i];
                     }
                 }
                 // warp-uniform
@@ -395,10 +403,10 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
                 for (int i = 0; i < MMA_BLOCKS_PER_WARP; ++i) {
                     const int u = i * (WPG * 32) + lane_unit;
                     xr[i] = u < pl.row_units ? __ldcg(src + u) : zero;
-                    if (DOWN) wr[i] = u < pl.row_units ? __ldcg(src + pl.row_units + u) : zero;
+                    if (DOWN && Z_LO) wr[i] = u < pl.row_units ? __ldcg(src + pl.row_units + u) : zero;
                 }
             } else {
-                for (int v = tid; v < (DOWN ? 2 : 1) * pl.row_units; v += DEC_CONSUMERS)
+                for (int v = tid; v < (DOWN && Z_LO ? 2 : 1) * pl.row_units; v += DEC_CONSUMERS)
                     reinterpret_cast<uint4 *>(s.vec)[v] = __ldcg(src + v);
                 consumer_barrier();
             }
@@ -465,11 +473,11 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
                 const int j = r0 + my_row;
                 if (p.seq[b].b_gate) a0 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[b].b_gate)[j]);
                 if (p.seq[b].b_up) a1 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[b].b_up)[j]);
-                // z leaves as two bf16 numbers, z_hi + z_lo, ready to be the down half's vector
+                // z leaves in bf16 (Z_LO: as two bf16 numbers, z_hi + z_lo), ready to be the down half's vector
                 const float zv = sigma_rt(act, a0) * a1;
                 const __nv_bfloat16 h = __float2bfloat16_rn(zv);
                 zbits[(size_t)b * 2 * p.ldk + j] = h;
-                zbits[(size_t)b * 2 * p.ldk + p.ldk + j] = __float2bfloat16_rn(zv - __bfloat162float(h));
+                if (Z_LO) zbits[(size_t)b * 2 * p.ldk + p.ldk + j] = __float2bfloat16_rn(zv - __bfloat162float(h));
             } else {
                 const int c = r0 + my_row;
                 float acc = (my_row & 1) ? a1 : a0;
@@ -477,42 +485,13 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
                 static_cast<__nv_bfloat16 *>(p.y)[(size_t)b * p.d + c] = __float2bfloat16_rn(acc);
             }
         }
-        if (!DOWN) {  // the last slice also clears the padding of z (at most 7 entries)
-            const int pad = tid - (DEC_CONSUMERS - 8);
-            if (sl == n_slices - 1 && pad >= 0 && p.k + pad < p.ldk) {
-                zbits[(size_t)b * 2 * p.ldk + p.k + pad] = __float2bfloat16_rn(0.f);
-                zbits[(size_t)b * 2 * p.ldk + p.ldk + p.k + pad] = __float2bfloat16_rn(0.f);
+        if (!DOWN && sl == n_slices - 1)  // the last slice also clears the padding of z
+            for (int j = p.k + tid; j < p.ldk; j += DEC_CONSUMERS) {
+                zbits[(size_t)b * 2 * p.ldk + j] = __float2bfloat16_rn(0.f);
+                if (Z_LO) zbits[(size_t)b * 2 * p.ldk + p.ldk + j] = __float2bfloat16_rn(0.f);
             }
-        }
     }
     return !*s.abort;
-}
-
-__device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int *p) {
-    unsigned int v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
-
-// Grid-wide meeting point between the two halves, called by one thread per CTA after the
-// CTA's z entries have been written and fenced.  Bounded: gives up after WAIT_LIMIT_CYCLES.
-// The counters clean up after themselves: the last CTA to leave resets both.
-__device__ __forceinline__ bool grid_meet(WsHeader *h, unsigned int n_ctas, volatile int *abort, void *ws) {
-    atomicAdd(&h->arrive, 1u);
-    const long long t0 = clock64();
-    while (!*abort && ld_acquire_u32(&h->arrive) < n_ctas) {
-        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
-            *abort = 1;
-            raise_status(ws, DEV_STATUS_TIMEOUT, 9);
-            return false;
-        }
-    }
-    if (atomicAdd(&h->depart, 1u) == n_ctas - 1) {  // everybody has seen the full count
-        h->depart = 0;
-        h->arrive = 0;
-        __threadfence();
-    }
-    return true;
 }
 
 #ifndef GRIFFIN_DEC_MIN_CTAS
@@ -563,10 +542,10 @@ __global__ void __launch_bounds__(DEC_THREADS, GRIFFIN_DEC_MIN_CTAS) decode_fuse
     }
     // each group reports on its own: 2 arrivals per CTA
     const int group = warp / DEC_GROUP_WARPS;
-    __threadfence();  // this group's z entries are visible device-wide before it reports in
-    group_barrier(group);
-    if ((tid & (DEC_GROUP_WARPS * 32 - 1)) == 0) grid_meet(static_cast<WsHeader *>(p.ws), 2 * gridDim.x, s.abort, p.ws);
-    consumer_barrier();  // both groups have seen everybody: the staged vector may be replaced by z
+    group_barrier(group);  // this group's z entries are written (the thread that reports in makes them visible device-wide)
+    if ((tid & (DEC_GROUP_WARPS * 32 - 1)) == 0)
+        grid_meet(&static_cast<WsHeader *>(p.ws)->meet_warp, 2 * gridDim.x, s.abort, p.ws);
+    group_barrier(group);  // the group has seen everybody: z is complete
     if (fp.dn.n_chunks == 1) {
         switch (fp.dn.R) {
             case 4: GRIFFIN_CONSUME(true, true, 1, fp.dn, p.n_slices_dn); break;
@@ -589,7 +568,7 @@ griffin_status decode_bf16_mma(DecodeParams &p, int act, uint32_t flags, cudaStr
     fp.gu = make_plan(p.d, p.d * 2);
     fp.dn = make_plan(p.ldk, p.ldk * 4);
     fp.slot_bytes = max(fp.gu.stage_bytes, fp.dn.stage_bytes);
-    fp.vec_bytes = fp.dn.n_chunks > 1 ? p.ldk * 4 : 16;  // only rows of several chunks stage z in shared memory
+    fp.vec_bytes = fp.dn.n_chunks > 1 ? p.ldk * (Z_LO ? 4 : 2) : 16;  // only rows of several chunks stage z in shared memory
     int n = ((int)MMA_SMEM_TARGET - fp.vec_bytes - (int)mma_fixed_smem(8)) / fp.slot_bytes;
     fp.n_stages = (n < 2 ? 2 : (n > 8 ? 8 : n)) & ~1;  // two halves, one per consumer group
     p.n_slices = slices_for(p.k, sms);
