@@ -298,8 +298,9 @@ __device__ __forceinline__ MmaSmem carve_fused(uint8_t *smem, const FusedPlan &f
 
 // Producer side of one half.  Lane l < 2R copies row (l & 1) of pair (l >> 1).  Weights only.
 template <bool DOWN>
-__device__ __forceinline__ bool produce_half(const DecodeParams &p, const MmaPlan &pl, const MmaSmem &s, int n_stages,
+__device__ __forceinline__ bool produce_half(const DecodeParams &p, const MmaPlan &plan, const MmaSmem &s, int n_stages,
                                              int slot_bytes, int n_slices, RingPos (&pos)[2], uint32_t &pgc, int lane) {
+    const MmaPlan pl = plan;  // in registers: the asm statements in the loops clobber memory, and a reload costs a round trip
     const int n_items = p.B * n_slices;
     const int total_rows = DOWN ? p.d : p.k;
     const int ns2 = n_stages >> 1;
@@ -361,9 +362,10 @@ __device__ __forceinline__ void group_barrier(int group) {
 // item); otherwise (rows longer than MMA_CHUNK_UNITS_MAX units, down only) the vector is
 // staged in shared memory and read from there block by block.
 template <bool DOWN, bool VREG, int WPG>
-__device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPlan &pl, const MmaSmem &s, int n_stages,
+__device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPlan &plan, const MmaSmem &s, int n_stages,
                                              int slot_bytes, int n_slices, RingPos &pos, uint32_t &pgc,
                                              int &item_parity, int act, int tid, int warp, int lane) {
+    const MmaPlan pl = plan;  // in registers: the asm statements in the loops clobber memory, and a reload costs a round trip
     const int n_items = p.B * n_slices;
     const int total_rows = DOWN ? p.d : p.k;
     const int chunk_bytes_max = pl.chunk_units * 16;
