@@ -301,6 +301,7 @@ template <bool DOWN>
 __device__ __forceinline__ bool produce_half(const DecodeParams &p, const MmaPlan &plan, const MmaSmem &s, int n_stages,
                                              int slot_bytes, int n_slices, RingPos (&pos)[2], uint32_t &pgc, int lane) {
     const MmaPlan pl = plan;  // in registers: the asm statements in the loops clobber memory, and a reload costs a round trip
+    void *const ws = p.ws;
     const int n_items = p.B * n_slices;
     const int total_rows = DOWN ? p.d : p.k;
     const int ns2 = n_stages >> 1;
@@ -332,7 +333,7 @@ __device__ __forceinline__ bool produce_half(const DecodeParams &p, const MmaPla
                 const uint32_t use = cur.round;
                 int go = 1;
                 if (lane == 0) {
-                    if (use > 0 && !wait_or_abort(&s.empty[stage], (use - 1) & 1, s.abort, p.ws, DOWN ? 7 : 5)) go = 0;
+                    if (use > 0 && !wait_or_abort(&s.empty[stage], (use - 1) & 1, s.abort, ws, DOWN ? 7 : 5)) go = 0;
                     if (go) mbar_arrive_expect_tx(&s.full[stage], (uint32_t)(rows_in_stage * units * 16));
                 }
                 go = __shfl_sync(0xffffffffu, go, 0);
@@ -366,6 +367,7 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
                                              int slot_bytes, int n_slices, RingPos &pos, uint32_t &pgc,
                                              int &item_parity, int act, int tid, int warp, int lane) {
     const MmaPlan pl = plan;  // in registers: the asm statements in the loops clobber memory, and a reload costs a round trip
+    void *const ws = p.ws;
     const int n_items = p.B * n_slices;
     const int total_rows = DOWN ? p.d : p.k;
     const int chunk_bytes_max = pl.chunk_units * 16;
@@ -426,7 +428,7 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
             if (pl.n_chunks > 1) my_blocks<WPG>(pl.chunk_units, q, my_full, tail_lanes);
             for (int c = 0; c < pl.n_chunks; ++c, pos.advance(ns2)) {
                 const int stage = group * ns2 + pos.slot;  // this group's half of the ring
-                if (!wait_or_abort(&s.full[stage], pos.round & 1, s.abort, p.ws, DOWN ? 8 : 6)) {
+                if (!wait_or_abort(&s.full[stage], pos.round & 1, s.abort, ws, DOWN ? 8 : 6)) {
                     ok = false;
                     break;
                 }
