@@ -17,7 +17,7 @@ from . import build as _build
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(7)
 ACT_SWIGLU, ACT_GEGLU_TANH, ACT_REGLU = 0, 1, 2
 DT_F32, DT_BF16 = 0, 1
-DECODE_DEFAULT, DECODE_OVERLAP_WEIGHT_PREFETCH = 0, 1
+DECODE_DEFAULT, DECODE_OVERLAP_WEIGHT_PREFETCH, DECODE_TCGEN05 = 0, 1, 2
 MAX_BATCH = 32
 
 ACT_BY_NAME = {"swiglu": ACT_SWIGLU, "geglu_tanh": ACT_GEGLU_TANH, "reglu": ACT_REGLU}

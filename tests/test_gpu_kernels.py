@@ -138,6 +138,44 @@ def test_decode_matches_oracle(dtype, d, d_ff, k, B):
     assert torch.equal(y, y2) and torch.equal(y, y3)   # deterministic, launch mode does not matter
 
 
+# Shapes that the opt-in tcgen05 kernel takes (d and ldk multiples of 128) and two that it hands
+# back to the warp-level kernel (ldk = 344; d = 1000).
+TCGEN05_SHAPES = [
+    # d, d_ff, k, B
+    (128, 256, 128, 1),      # a single 256-byte window per row of W_g_hat; fewer rows than CTAs
+    (2048, 5632, 2816, 1),
+    (3072, 4096, 4096, 1),   # k = d_ff, GEGLU
+    (4096, 11008, 5504, 1),  # Llama-2-7B shape: rows of W_2_hat end in a short piece
+    (5120, 2048, 1024, 8),   # batch 8: several work items per CTA, the vector changes between them
+    (8192, 1024, 512, 3),    # largest supported d; rows of W_2_hat shorter than a batch of windows
+    (1024, 3000, 1500, 2),   # k not a multiple of 8: ldk = 1504 is not a multiple of 128 either -> warp-level kernel
+    (256, 688, 344, 1),      # falls back as well
+]
+
+
+@pytest.mark.parametrize("d,d_ff,k,B", TCGEN05_SHAPES)
+def test_decode_tcgen05_kernel_matches_oracle_and_default_kernel(d, d_ff, k, B):
+    act = "geglu_tanh" if d == 3072 else "swiglu"
+    L, host = make_layer(d, d_ff, "bf16", act=act, bias=(d_ff < 2500), seed=3 * d + k, n_seq=B)
+    rs = np.random.default_rng(d + k)
+    x = rand((B, d), torch.bfloat16, 98)
+    sets, refs = [], []
+    for b in range(B):
+        e_np = np.sort(rs.choice(d_ff, size=k, replace=False)).astype(np.int32)
+        sets.append(L.compact(torch.from_numpy(e_np).to(dev())))
+        c = O.compact_experts(e_np, h64(host, "wg"), h64(host, "wu"), h64(host, "wd"), h64(host, "bg"), h64(host, "bu"))
+        refs.append(O.ff_pruned(np64(x[b]), c, act, h64(host, "bd")))
+    y_tc = L.decode(sets, x, G.DECODE_TCGEN05)
+    y_tc2 = L.decode(sets, x, G.DECODE_TCGEN05 | G.DECODE_OVERLAP_WEIGHT_PREFETCH)
+    y_warp = L.decode(sets, x)
+    y_tc3 = L.decode(sets, x, G.DECODE_TCGEN05 | G.DECODE_OVERLAP_WEIGHT_PREFETCH)   # after the other kernel used the workspace
+    assert L.status() == G.OK
+    for b in range(B):
+        assert rel_l2(np64(y_tc[b]), refs[b]) < TOL_OUT["bf16"], b
+        assert rel_l2(np64(y_tc[b]), np64(y_warp[b])) < TOL_OUT["bf16"], b
+    assert torch.equal(y_tc, y_tc2) and torch.equal(y_tc, y_tc3)   # deterministic, launch mode does not matter
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_decode_with_all_neurons_is_the_dense_ff(dtype):
     d, d_ff = 512, 1536
