@@ -34,8 +34,8 @@
 //   * C[m][n] pairs virtual row m with virtual vector n; only the diagonal m = n belongs to
 //     the dot product.  Lane (g, t = g / 2) holds it; three shuffles add the 8 diagonal
 //     entries.  The tensor core does 8x the needed multiplies, which is free here.
-//   * second half: z crosses as two bf16 numbers z_hi + z_lo per entry and each block runs
-//     the MMAs once against each, into the same accumulators, so 16 bits of z survive.
+//   * second half: z crosses in bf16 (with GRIFFIN_DEC_Z_LO as two bf16 numbers z_hi + z_lo
+//     per entry; each block then runs the MMAs once against each, into the same accumulators).
 //   * The 4 / R warps of a group share a pair; their partial sums meet in shared memory at
 //     the end of a work item, in a fixed order, so results are bitwise reproducible.
 #include "decode_common.cuh"
