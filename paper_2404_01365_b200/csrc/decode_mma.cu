@@ -84,13 +84,16 @@ static size_t mma_fixed_smem(int n_stages) {
     return 2 * n_stages * sizeof(uint64_t) + 2 * DEC_MAX_ROWS * DEC_CONSUMER_WARPS * sizeof(float2) + 16;
 }
 
-static MmaPlan make_plan(int row_elems, int vec_bytes) {
+static MmaPlan make_plan(int row_elems, int vec_bytes, int stage_target, int blocks_per_warp) {
     MmaPlan pl;
     pl.row_units = row_elems / 8;
     pl.n_chunks = (pl.row_units + MMA_CHUNK_UNITS_MAX - 1) / MMA_CHUNK_UNITS_MAX;
     pl.chunk_units = (pl.row_units + pl.n_chunks - 1) / pl.n_chunks;
     const int pair_bytes = 2 * pl.chunk_units * 16;
-    pl.R = pair_bytes * 4 <= MMA_STAGE_TARGET ? 4 : (pair_bytes * 2 <= MMA_STAGE_TARGET ? 2 : 1);
+    pl.R = pair_bytes * 4 <= stage_target ? 4 : (pair_bytes * 2 <= stage_target ? 2 : 1);
+    // the DEC_GROUP_WARPS / R warps that share a pair must not get more blocks than they have registers for
+    const int row_blocks = (pl.chunk_units + 31) / 32;
+    while (pl.R > 1 && (row_blocks + DEC_GROUP_WARPS / pl.R - 1) / (DEC_GROUP_WARPS / pl.R) > blocks_per_warp) pl.R >>= 1;
     pl.stage_bytes = pl.R * pair_bytes;
     pl.vec_bytes = vec_bytes;
     int n = ((int)MMA_SMEM_TARGET - vec_bytes - (int)mma_fixed_smem(8)) / pl.stage_bytes;
@@ -142,6 +145,14 @@ __device__ __forceinline__ float diagonal_sum(const float (&c)[4], int lane) {
 //   registers (gate_up, where x is the same for every neuron of the item); my_full : whole
 //   blocks of this warp; tail_lanes : lanes with data in the block after them (0: no such block)
 constexpr int MMA_BLOCKS_PER_WARP = 8;
+// The second half takes larger stages (two pairs of rows of W_2_hat where one pair is more than
+// half a first-half stage): every stage costs its consumers a fixed round of waiting, reducing
+// and handing back, and this half runs at their pace.  A warp then has up to 12 blocks.
+#ifndef GRIFFIN_DEC_DOWN_STAGE_KB
+#define GRIFFIN_DEC_DOWN_STAGE_KB 48
+#endif
+constexpr int MMA_BLOCKS_PER_WARP_DOWN = 12;
+template <bool DOWN> struct BlocksPerWarp { static constexpr int N = DOWN ? MMA_BLOCKS_PER_WARP_DOWN : MMA_BLOCKS_PER_WARP; };
 #ifndef GRIFFIN_DEC_BATCH
 #define GRIFFIN_DEC_BATCH 4
 #endif
@@ -181,12 +192,12 @@ __device__ __forceinline__ void batch_mma(float (&acc)[MMA_ACCS][4], const uint4
 // shared memory.
 template <bool DOWN, bool VREG, int WPG>
 __device__ __forceinline__ void pair_mma(float (&acc)[MMA_ACCS][4], const uint4 *p0, const uint4 *p1, const uint4 *pv,
-                                         const uint4 *pw, const uint4 (&xr)[MMA_BLOCKS_PER_WARP],
-                                         const uint4 (&wr)[MMA_BLOCKS_PER_WARP], int my_full, int tail_lanes,
+                                         const uint4 *pw, const uint4 (&xr)[BlocksPerWarp<DOWN>::N],
+                                         const uint4 (&wr)[BlocksPerWarp<DOWN>::N], int my_full, int tail_lanes,
                                          int lane) {
     constexpr int BS = WPG * 32;  // units between consecutive blocks of this warp
 #pragma unroll
-    for (int b0 = 0; b0 < MMA_BLOCKS_PER_WARP; b0 += MMA_BATCH) {
+    for (int b0 = 0; b0 < BlocksPerWarp<DOWN>::N; b0 += MMA_BATCH) {
         uint4 r0[MMA_BATCH], r1[MMA_BATCH], v[MMA_BATCH], w[MMA_BATCH];
         if (b0 + MMA_BATCH <= my_full) {  // warp-uniform: four whole blocks
 #pragma unroll
@@ -384,7 +395,7 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
     // the scratch holds, per sequence, z_hi [ldk] then z_lo [ldk] in bf16 (same bytes as fp32 [ldk])
     __nv_bfloat16 *zbits = reinterpret_cast<__nv_bfloat16 *>(p.z);
     int cur_b = -1;
-    uint4 xr[MMA_BLOCKS_PER_WARP], wr[MMA_BLOCKS_PER_WARP];  // x, or z_hi and z_lo
+    uint4 xr[BlocksPerWarp<DOWN>::N], wr[BlocksPerWarp<DOWN>::N];  // x, or z_hi and z_lo
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, item_parity ^= 1) {
         const int b = item / n_slices, sl = item - b * n_slices;
         const int r0 = (int)((long long)sl * total_rows / n_slices);
@@ -404,7 +415,7 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
             if (VREG) {
                 const uint4 zero = make_uint4(0, 0, 0, 0);
 #pragma unroll
-                for (int i = 0; i < MMA_BLOCKS_PER_WARP; ++i) {
+                for (int i = 0; i < BlocksPerWarp<DOWN>::N; ++i) {
                     const int u = i * (WPG * 32) + lane_unit;
                     xr[i] = u < pl.row_units ? __ldcg(src + u) : zero;
                     if (DOWN && Z_LO) wr[i] = u < pl.row_units ? __ldcg(src + pl.row_units + u) : zero;
@@ -569,8 +580,8 @@ griffin_status decode_bf16_mma(DecodeParams &p, int act, uint32_t flags, cudaStr
     if (p.ws == nullptr) return GRIFFIN_ERR_WORKSPACE;  // the meeting point's counters live in the header
     const bool overlap = (flags & GRIFFIN_DECODE_OVERLAP_WEIGHT_PREFETCH) != 0;
     FusedPlan fp;
-    fp.gu = make_plan(p.d, p.d * 2);
-    fp.dn = make_plan(p.ldk, p.ldk * 4);
+    fp.gu = make_plan(p.d, p.d * 2, MMA_STAGE_TARGET, MMA_BLOCKS_PER_WARP);
+    fp.dn = make_plan(p.ldk, p.ldk * 4, GRIFFIN_DEC_DOWN_STAGE_KB * 1024, MMA_BLOCKS_PER_WARP_DOWN);
     fp.slot_bytes = max(fp.gu.stage_bytes, fp.dn.stage_bytes);
     fp.vec_bytes = fp.dn.n_chunks > 1 ? p.ldk * (Z_LO ? 4 : 2) : 16;  // only rows of several chunks stage z in shared memory
     int n = ((int)MMA_SMEM_TARGET - fp.vec_bytes - (int)mma_fixed_smem(8)) / fp.slot_bytes;
