@@ -235,6 +235,31 @@ __global__ void score_finish_kernel(const float *__restrict__ colpart, int n_row
     score[j] = sqrtf(acc);
 }
 
+// The statistic only needs Z, the down projection only Z as well: with the tensor-core path the
+// statistic kernels run on a stream of the library's own beside the second GEMM (whose
+// persistent CTAs leave room for them on every SM) and join the caller's stream at the end.
+// One lane per host thread and device, created at first use and kept.
+struct SideLane {
+    cudaStream_t stream;
+    cudaEvent_t fork, join;
+};
+static SideLane *side_lane_of_current_device() {
+    constexpr int MAX_DEV = 64;
+    static thread_local SideLane lanes[MAX_DEV];
+    static thread_local int state[MAX_DEV];  // 0 untried, 1 ready, -1 unavailable
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEV) return nullptr;
+    if (state[dev] == 0) {
+        SideLane &l = lanes[dev];
+        state[dev] = (cudaStreamCreateWithFlags(&l.stream, cudaStreamNonBlocking) == cudaSuccess &&
+                      cudaEventCreateWithFlags(&l.fork, cudaEventDisableTiming) == cudaSuccess &&
+                      cudaEventCreateWithFlags(&l.join, cudaEventDisableTiming) == cudaSuccess)
+                         ? 1
+                         : -1;
+    }
+    return state[dev] == 1 ? &lanes[dev] : nullptr;
+}
+
 template <typename T>
 static griffin_status prefill_typed(const griffin_ff_desc *desc, const griffin_ff_weights *w, const void *x, int S,
                                     void *y, float *score, uint8_t *scratch, void *ws, cudaStream_t stream) {
@@ -251,11 +276,18 @@ static griffin_status prefill_typed(const griffin_ff_desc *desc, const griffin_f
     bool ff2_done = false;
     bool use_tc = false;
     if constexpr (kBf16) use_tc = prefill_tc_supported(desc, S);
+    cudaStream_t stat_stream = stream;  // where the statistic kernels go
+    SideLane *lane = nullptr;
     if (use_tc) {
         if constexpr (kBf16) {
+            if (y != nullptr) lane = side_lane_of_current_device();
             griffin_status st = launch_prefill_tc(desc, w, x, S, y, z, zf, rowsq, reinterpret_cast<float *>(scratch + ps.ypart_off),
-                                                  &n_col_tiles, ws, stream);
+                                                  &n_col_tiles, ws, stream, lane ? lane->fork : nullptr);
             if (st != GRIFFIN_OK) return st;
+            if (lane != nullptr) {
+                if (cudaStreamWaitEvent(lane->stream, lane->fork, 0) != cudaSuccess) return GRIFFIN_ERR_CUDA;
+                stat_stream = lane->stream;
+            }
         }
         ff2_done = true;
     } else {
@@ -274,14 +306,17 @@ static griffin_status prefill_typed(const griffin_ff_desc *desc, const griffin_f
                                                           d_ff);
         if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
     }
-    row_inv_kernel<<<(S + 7) / 8, 256, 0, stream>>>(rowsq, S, n_col_tiles, inv);
+    row_inv_kernel<<<(S + 7) / 8, 256, 0, stat_stream>>>(rowsq, S, n_col_tiles, inv);
     if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
     const float *z32 = kBf16 ? zf : reinterpret_cast<const float *>(z);
     const dim3 g4((d_ff + 127) / 128, ps.n_row_chunks);
-    col_partial_kernel<<<g4, 256, 0, stream>>>(z32, inv, S, d_ff, colpart);
+    col_partial_kernel<<<g4, 256, 0, stat_stream>>>(z32, inv, S, d_ff, colpart);
     if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
-    score_finish_kernel<<<(d_ff + 255) / 256, 256, 0, stream>>>(colpart, ps.n_row_chunks, d_ff, score);
+    score_finish_kernel<<<(d_ff + 255) / 256, 256, 0, stat_stream>>>(colpart, ps.n_row_chunks, d_ff, score);
     if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
+    if (lane != nullptr &&
+        (cudaEventRecord(lane->join, lane->stream) != cudaSuccess || cudaStreamWaitEvent(stream, lane->join, 0) != cudaSuccess))
+        return GRIFFIN_ERR_CUDA;
     return GRIFFIN_OK;
 }
 

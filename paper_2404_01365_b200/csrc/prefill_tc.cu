@@ -320,7 +320,7 @@ static griffin_status launch_tc(const CUtensorMap &ma, const CUtensorMap &mb0, c
 
 griffin_status launch_prefill_tc(const griffin_ff_desc *desc, const griffin_ff_weights *w, const void *x, int S,
                                  void *y, __nv_bfloat16 *z, float *zf, float *rowsq, float *ypart, int *n_col_tiles,
-                                 void *ws, cudaStream_t stream) {
+                                 void *ws, cudaStream_t stream, cudaEvent_t after_ff1) {
     const int d = desc->d, d_ff = desc->d_ff;
     const int sms = device_sm_count();
     if (sms <= 0) return GRIFFIN_ERR_CUDA;
@@ -345,6 +345,7 @@ griffin_status launch_prefill_tc(const griffin_ff_desc *desc, const griffin_ff_w
     p.splits = 1;
     *n_col_tiles = p.n_tiles;
     griffin_status st = launch_tc<true, 128>(mx, mg, mu, p, sms, stream);
+    if (st == GRIFFIN_OK && after_ff1 != nullptr && cudaEventRecord(after_ff1, stream) != cudaSuccess) return GRIFFIN_ERR_CUDA;
     if (st != GRIFFIN_OK || y == nullptr) return st;
 
     // Y = Z W_2^T + b_2
