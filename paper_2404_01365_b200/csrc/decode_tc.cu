@@ -50,7 +50,6 @@ constexpr int DTC_EPI_THREADS = 128;
 constexpr int DTC_WINDOW = 256;            // bytes of a row that one MMA takes (two K steps of 8 units)
 constexpr int DTC_SLOT_BYTES = 32 * 1024;  // one stage of the ring
 constexpr int DTC_MAX_STAGES = 7;
-constexpr int DTC_MAX_WPC = DTC_SLOT_BYTES / 8 / DTC_WINDOW;  // windows per piece with sets of 8 rows
 constexpr int DTC_MAX_SETS = 16;           // sets per work item (128 rows of 8)
 constexpr int DTC_TMEM_COLS = 512;         // 32 accumulators of 16 columns
 #ifndef GRIFFIN_DTC_SET_ROWS_0
