@@ -170,8 +170,10 @@ griffin_status griffin_compact_experts(const griffin_ff_desc *desc, const griffi
 
 /* Generation phase (Eqs. 4, 5): for each of B sequences, with its own compact set,
  *   y[b] = W_2_hat (sigma(W_g_hat x[b] + b_g_hat) * (W_1_hat x[b] + b_1_hat)) + b_2.
- * sets: HOST array of B structs (entries may repeat to share a set); every set must have
- * the same k and ldk.  b_down [d] or NULL is shared by all sequences.  x [B, d] in,
+ * sets: HOST array of B structs; every set must have the same k and ldk.  Entries may repeat
+ * to share a set: when 2..8 sequences of a bf16 call all name the same buffers (one expert
+ * set for the batch, Eq. 7) and d and ldk are multiples of 128, the weights are streamed
+ * once and every row meets all B vectors (otherwise each sequence is a pass of its own).  b_down [d] or NULL is shared by all sequences.  x [B, d] in,
  * y [B, d] out.  1 <= B <= GRIFFIN_MAX_BATCH, d <= GRIFFIN_MAX_D.  flags: GRIFFIN_DECODE_*.
  * The activations z_hat [B, ldk] pass through the workspace (4 bytes per entry).  With bf16
  * storage the call is one kernel whose CTAs (one per SM) meet half-way through a counter in

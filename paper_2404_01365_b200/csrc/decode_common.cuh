@@ -113,10 +113,10 @@ int slices_for(int rows, int grid);
 // bf16 decode through warp-level MMA (decode_mma.cu).
 griffin_status decode_bf16_mma(DecodeParams &p, int act, uint32_t flags, cudaStream_t stream);
 
-// bf16 decode through tcgen05 (decode_tc.cu): at most DTC_MAX_B sequences, d and ldk multiples
-// of 64, a workspace for the meeting point.
-constexpr int DTC_MAX_B = 4;
+// bf16 decode through tcgen05 (decode_tc.cu): d and ldk multiples of 128, a workspace for the
+// meeting point.
 bool decode_tc_supported(const DecodeParams &p);
+bool decode_tc_shared(const DecodeParams &p);  // 2..8 sequences that all use one expert set: streamed once for all
 griffin_status decode_bf16_tc(DecodeParams &p, int act, uint32_t flags, cudaStream_t stream);
 
 }  // namespace griffin

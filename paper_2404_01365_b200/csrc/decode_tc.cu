@@ -52,6 +52,7 @@ constexpr int DTC_SLOT_BYTES = 32 * 1024;  // one stage of the ring
 constexpr int DTC_MAX_STAGES = 7;
 constexpr int DTC_MAX_SETS = 16;           // sets per work item (128 rows of 8)
 constexpr int DTC_TMEM_COLS = 512;         // 32 accumulators of 16 columns
+constexpr int DTC_MAX_VEC = 8;             // vectors that may share one expert set in a call
 #ifndef GRIFFIN_DTC_SET_ROWS_0
 #define GRIFFIN_DTC_SET_ROWS_0 16
 #endif
@@ -68,16 +69,19 @@ struct DtcHalf {
     int wpc;       // windows per piece (the last may be shorter)
     int sbo_b;     // bytes from the vector to its second copy (z_lo), 0 if there is none
     int n_acc;     // accumulators per set (a power of two), taken in turn by the windows of a row
+    int acc_cols;  // columns of one accumulator = N of the MMA: 8 per group of B rows, at least 16
 };
 struct DtcPlan {
     DtcHalf h[2];
     int n_stages;
-    int vec_bytes;  // shared memory set aside for the vector
+    int vec_bytes;   // shared memory set aside for the vector(s)
+    int n_vec;       // 1: every sequence has its own expert set; B: one set for the B vectors of the call
+    int vec_stride;  // bytes between the vectors in shared memory (n_vec > 1)
 };
 
 struct DtcSmem {
     uint8_t *ring, *vec;
-    float *part;  // [DTC_MAX_SETS * 16]
+    float *part;  // [DTC_MAX_VEC][DTC_MAX_SETS * 16]
     uint64_t *full, *empty, *vec_full, *acc_full;
     uint32_t *tmem_slot;
     volatile int *abort;
@@ -85,7 +89,7 @@ struct DtcSmem {
 // An MMA always reads 16 staged rows: with sets of 8 rows the other 8 lie beyond the stage, so
 // what follows the ring must be at least that long (what is read there is never used).
 static size_t dtc_smem_bytes(const DtcPlan &pl) {
-    size_t tail = pl.vec_bytes + DTC_MAX_SETS * 16 * sizeof(float) + (2 * DTC_MAX_STAGES + 2) * sizeof(uint64_t) + 16;
+    size_t tail = pl.vec_bytes + DTC_MAX_VEC * DTC_MAX_SETS * 16 * sizeof(float) + (2 * DTC_MAX_STAGES + 2) * sizeof(uint64_t) + 16;
     for (int i = 0; i < 2; ++i) {
         const size_t beyond = (size_t)(16 - pl.h[i].set_rows) * pl.h[i].wpc * DTC_WINDOW;
         if (beyond > tail) tail = beyond;
@@ -152,10 +156,11 @@ __device__ __forceinline__ void dtc_item_rows(const DtcHalf &h, int sl, int &r0,
 // row, so this is also the window's number in the row modulo NACC.
 //   first : these are the first windows of the row (accumulators 0 .. NACC-1 are overwritten)
 template <int NACC>
-__device__ __forceinline__ void mma_batch8(uint32_t d_set, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool first) {
+__device__ __forceinline__ void mma_batch8(const uint32_t (&dacc)[NACC], uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                           bool first) {
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-        const uint32_t d = d_set + (uint32_t)(j % NACC) * 16u;
+        const uint32_t d = dacc[j % NACC];
         const uint64_t a = a_desc + (uint64_t)(j * (DTC_WINDOW >> 4)), b = b_desc + (uint64_t)(j * (DTC_WINDOW >> 4));
         if (j < NACC)
             umma_bf16(d, a, b, idesc, first ? 0u : 1u);
@@ -168,10 +173,10 @@ __device__ __forceinline__ void mma_batch8(uint32_t d_set, uint64_t a_desc, uint
 template <int NACC>
 __device__ __forceinline__ bool dtc_issue_half(const DecodeParams &p, const DtcPlan &pl, const DtcSmem &s, int half,
                                                uint32_t tmem_base, uint32_t &it, uint32_t &n_item) {
-    constexpr uint32_t IDESC = umma_idesc(128, 16);
     const DtcHalf h = half ? pl.h[1] : pl.h[0];  // (a copy in registers: the asm statements below clobber memory)
+    const uint32_t IDESC = umma_idesc(128, h.acc_cols);
     const int n_stages = pl.n_stages;
-    const int n_items = p.B * h.n_slices;
+    const int n_items = (pl.n_vec > 1 ? 1 : p.B) * h.n_slices;
     const uint32_t piece_max = (uint32_t)h.wpc * DTC_WINDOW;
     const uint64_t a_desc0 = smem_desc_plain(smem_u32(s.ring), 128u, piece_max);
     const uint64_t b_desc0 = smem_desc_plain(smem_u32(s.vec), 128u, (uint32_t)h.sbo_b);
@@ -186,7 +191,10 @@ __device__ __forceinline__ bool dtc_issue_half(const DecodeParams &p, const DtcP
         if (!wait_or_abort(s.vec_full, n_item & 1, s.abort, p.ws, 32 + half)) return false;
         tc_fence_after_sync();
         uint32_t d_set = tmem_base;
-        for (int row_s = 0; row_s < n_rows_item; row_s += h.set_rows, d_set += NACC * 16u) {
+        for (int row_s = 0; row_s < n_rows_item; row_s += h.set_rows, d_set += NACC * (uint32_t)h.acc_cols) {
+            uint32_t dacc[NACC];
+#pragma unroll
+            for (int a = 0; a < NACC; ++a) dacc[a] = d_set + (uint32_t)(a * h.acc_cols);
             for (int c = 0; c < h.n_chunks; ++c, ++it) {
                 if (!wait_or_abort(&s.full[stage], round & 1, s.abort, p.ws, 34 + half)) return false;
                 tc_fence_after_sync();
@@ -196,12 +204,12 @@ __device__ __forceinline__ bool dtc_issue_half(const DecodeParams &p, const DtcP
                 uint64_t b_desc = b_desc0 + (uint64_t)((uint32_t)(c * h.wpc) * (DTC_WINDOW >> 4));
                 int w = 0;
                 for (; w + 8 <= nw; w += 8) {
-                    mma_batch8<NACC>(d_set, a_desc, b_desc, IDESC, c == 0 && w == 0);
+                    mma_batch8<NACC>(dacc, a_desc, b_desc, IDESC, c == 0 && w == 0);
                     a_desc += 8 * (DTC_WINDOW >> 4);
                     b_desc += 8 * (DTC_WINDOW >> 4);
                 }
                 for (int j = 0; w < nw; ++w, ++j)  // what is left of the row's last piece
-                    umma_bf16(d_set + (uint32_t)(j % NACC) * 16u, a_desc + (uint64_t)(j * (DTC_WINDOW >> 4)),
+                    umma_bf16(d_set + (uint32_t)((j % NACC) * h.acc_cols), a_desc + (uint64_t)(j * (DTC_WINDOW >> 4)),
                               b_desc + (uint64_t)(j * (DTC_WINDOW >> 4)), IDESC, (c * h.wpc + w) >= NACC ? 1u : 0u);
                 umma_commit(&s.empty[stage]);  // the stage may be refilled once these MMAs have read it
                 if (++stage == n_stages) {
@@ -222,7 +230,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
     s.ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     s.vec = s.ring + (size_t)pl.n_stages * DTC_SLOT_BYTES;
     s.part = reinterpret_cast<float *>(s.vec + pl.vec_bytes);
-    s.full = reinterpret_cast<uint64_t *>(s.part + DTC_MAX_SETS * 16);
+    s.full = reinterpret_cast<uint64_t *>(s.part + DTC_MAX_VEC * DTC_MAX_SETS * 16);
     s.empty = s.full + DTC_MAX_STAGES;
     s.vec_full = s.empty + DTC_MAX_STAGES;
     s.acc_full = s.vec_full + 1;
@@ -253,7 +261,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
         bool ok = true;
         for (int half = 0; ok && half < 2; ++half) {
             const DtcHalf h = half ? pl.h[1] : pl.h[0];  // (a copy in registers: the asm statements below clobber memory)
-            const int n_items = p.B * h.n_slices;
+            const int n_items = (pl.n_vec > 1 ? 1 : p.B) * h.n_slices;  // (one shared set: the slices of that one set)
             const size_t row_bytes = (size_t)h.windows * DTC_WINDOW;
             const uint32_t piece_max = (uint32_t)h.wpc * DTC_WINDOW;
             for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
@@ -329,7 +337,9 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
         bool stop = false;
         for (int half = 0; !stop && half < 2; ++half) {
             const DtcHalf h = half ? pl.h[1] : pl.h[0];  // (a copy in registers: the asm statements below clobber memory)
-            const int n_items = p.B * h.n_slices;
+            const int n_vec = pl.n_vec;                    // vectors that meet every staged row
+            const int n_groups = n_vec > 1 ? n_vec : (half ? 2 : 1);  // groups of 8 B rows with data: vectors, or z_hi and z_lo
+            const int n_items = (n_vec > 1 ? 1 : p.B) * h.n_slices;
             int cur_b = -1;
             for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n_item) {
                 const int b = item / h.n_slices, sl = item - b * h.n_slices;
@@ -339,24 +349,29 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                 const int n_rows_item = half ? R : 2 * R;
                 const int n_sets = (n_rows_item + h.set_rows - 1) / h.set_rows;
                 if (b != cur_b) {
-                    // the vector, read through L2 (x comes from earlier work on the stream, z from
-                    // other CTAs of this grid): x, or z_hi then z_lo, as they lie in memory
-                    const int n_units = h.windows * (DTC_WINDOW / 16) * (half ? 2 : 1);
-                    const uint4 *src = half ? reinterpret_cast<const uint4 *>(zbits + (size_t)b * 2 * p.ldk)
-                                            : reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(p.x) +
-                                                                              (size_t)b * p.d);
-                    uint4 *dst = reinterpret_cast<uint4 *>(s.vec);
-                    for (int u0 = et; u0 < n_units; u0 += 4 * DTC_EPI_THREADS) {
-                        uint4 v[4];
+                    // the vector(s), read through L2 (x comes from earlier work on the stream, z from
+                    // other CTAs of this grid).  One vector: x, or z_hi then z_lo, as they lie in
+                    // memory.  A shared set: x (or z_hi) of every sequence, vec_stride bytes apart.
+                    const int row_units = h.windows * (DTC_WINDOW / 16);
+                    const int n_units = n_vec > 1 ? row_units : row_units * (half ? 2 : 1);
+                    for (int v = 0; v < n_vec; ++v) {
+                        const int seq = n_vec > 1 ? v : b;
+                        const uint4 *src = half ? reinterpret_cast<const uint4 *>(zbits + (size_t)seq * 2 * p.ldk)
+                                                : reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(p.x) +
+                                                                                  (size_t)seq * p.d);
+                        uint4 *dst = reinterpret_cast<uint4 *>(s.vec + (size_t)v * pl.vec_stride);
+                        for (int u0 = et; u0 < n_units; u0 += 4 * DTC_EPI_THREADS) {
+                            uint4 t[4];
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {  // all loads of a round are in flight together
-                            const int u = u0 + j * DTC_EPI_THREADS;
-                            v[j] = u < n_units ? __ldcg(src + u) : make_uint4(0, 0, 0, 0);
-                        }
+                            for (int j = 0; j < 4; ++j) {  // all loads of a round are in flight together
+                                const int u = u0 + j * DTC_EPI_THREADS;
+                                t[j] = u < n_units ? __ldcg(src + u) : make_uint4(0, 0, 0, 0);
+                            }
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const int u = u0 + j * DTC_EPI_THREADS;
-                            if (u < n_units) dst[u] = v[j];
+                            for (int j = 0; j < 4; ++j) {
+                                const int u = u0 + j * DTC_EPI_THREADS;
+                                if (u < n_units) dst[u] = t[j];
+                            }
                         }
                     }
                     fence_proxy_async_smem();  // the MMA reads shared memory through the async proxy
@@ -375,19 +390,35 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     const uint32_t taddr = tmem_base + ((uint32_t)(wq * 32) << 16);
 #pragma unroll 1
                     for (int set = 0; set < n_sets; ++set) {
-                        float val = 0.f;
-                        for (int a = 0; a < h.n_acc; ++a) {  // (a fixed order: results are reproducible)
-                            float v[16];
-                            tmem_ld16(taddr + (uint32_t)(set * h.n_acc + a) * 16u, v);
+                        float val[DTC_MAX_VEC];  // per group of B rows: this lane's diagonal entry
 #pragma unroll
-                            for (int c = 0; c < 8; ++c)
-                                if (c == unit) val += half ? v[c] + v[8 + c] : v[c];
+                        for (int g = 0; g < DTC_MAX_VEC; ++g) val[g] = 0.f;
+                        for (int a = 0; a < h.n_acc; ++a) {  // (a fixed order: results are reproducible)
+                            const uint32_t acc_addr = taddr + (uint32_t)((set * h.n_acc + a) * h.acc_cols);
+#pragma unroll
+                            for (int g2 = 0; g2 < DTC_MAX_VEC / 2; ++g2) {  // 16 columns = two groups at a time
+                                if (2 * g2 < n_groups) {               // warp-uniform
+                                    float t[16];
+                                    tmem_ld16(acc_addr + (uint32_t)g2 * 16u, t);
+#pragma unroll
+                                    for (int c = 0; c < 8; ++c)
+                                        if (c == unit) {
+                                            val[2 * g2] += t[c];
+                                            if (2 * g2 + 1 < n_groups) val[2 * g2 + 1] += t[8 + c];
+                                        }
+                                }
+                            }
                         }
-                        // the 8 units of a weight row sit in 8 consecutive lanes
-                        val += __shfl_xor_sync(0xffffffffu, val, 1);
-                        val += __shfl_xor_sync(0xffffffffu, val, 2);
-                        val += __shfl_xor_sync(0xffffffffu, val, 4);
-                        if (unit == 0) s.part[set * 16 + row_in_set] = val;
+                        if (n_vec == 1 && half) val[0] += val[1];  // z_hi and z_lo belong to the same output
+#pragma unroll
+                        for (int g = 0; g < DTC_MAX_VEC; ++g)
+                            if (g < n_vec) {  // the 8 units of a weight row sit in 8 consecutive lanes
+                                float t = val[g];
+                                t += __shfl_xor_sync(0xffffffffu, t, 1);
+                                t += __shfl_xor_sync(0xffffffffu, t, 2);
+                                t += __shfl_xor_sync(0xffffffffu, t, 4);
+                                if (unit == 0) s.part[g * (DTC_MAX_SETS * 16) + set * 16 + row_in_set] = t;
+                            }
                     }
                 }
                 tc_fence_before_sync();
@@ -395,29 +426,37 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     stop = true;
                     break;
                 }
-                // thread t finishes row r0 + t of the item
+                // thread t finishes row r0 + t of the item, for every vector
                 if (et < R) {
                     const int row = r0 + et;
-                    if (!half) {
-                        const int iu = R + et;  // the up row's place in the item
-                        float a0 = s.part[(et / h.set_rows) * 16 + et % h.set_rows];
-                        float a1 = s.part[(iu / h.set_rows) * 16 + iu % h.set_rows];
-                        if (p.seq[b].b_gate) a0 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[b].b_gate)[row]);
-                        if (p.seq[b].b_up) a1 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[b].b_up)[row]);
-                        const float zv = sigma_rt(act, a0) * a1;
-                        const __nv_bfloat16 hi = __float2bfloat16_rn(zv);
-                        zbits[(size_t)b * 2 * p.ldk + row] = hi;
-                        zbits[(size_t)b * 2 * p.ldk + p.ldk + row] = __float2bfloat16_rn(zv - __bfloat162float(hi));
-                    } else {
-                        float acc = s.part[(et / h.set_rows) * 16 + et % h.set_rows];
-                        if (p.b_down) acc += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.b_down)[row]);
-                        static_cast<__nv_bfloat16 *>(p.y)[(size_t)b * p.d + row] = __float2bfloat16_rn(acc);
+                    const int ig = (et / h.set_rows) * 16 + et % h.set_rows;  // where the (gate) row's result is
+                    for (int v = 0; v < n_vec; ++v) {
+                        const int seq = n_vec > 1 ? v : b;
+                        const float *part = s.part + v * (DTC_MAX_SETS * 16);
+                        if (!half) {
+                            const int iu = R + et;  // the up row's place in the item
+                            float a0 = part[ig];
+                            float a1 = part[(iu / h.set_rows) * 16 + iu % h.set_rows];
+                            if (p.seq[b].b_gate) a0 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[b].b_gate)[row]);
+                            if (p.seq[b].b_up) a1 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[b].b_up)[row]);
+                            const float zv = sigma_rt(act, a0) * a1;
+                            const __nv_bfloat16 hi = __float2bfloat16_rn(zv);
+                            zbits[(size_t)seq * 2 * p.ldk + row] = hi;
+                            if (n_vec == 1) zbits[(size_t)seq * 2 * p.ldk + p.ldk + row] = __float2bfloat16_rn(zv - __bfloat162float(hi));
+                        } else {
+                            float acc = part[ig];
+                            if (p.b_down) acc += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.b_down)[row]);
+                            static_cast<__nv_bfloat16 *>(p.y)[(size_t)seq * p.d + row] = __float2bfloat16_rn(acc);
+                        }
                     }
                 }
                 if (!half && sl == h.n_slices - 1)  // the last slice also clears the padding of z
-                    for (int j = p.k + et; j < p.ldk; j += DTC_EPI_THREADS) {
-                        zbits[(size_t)b * 2 * p.ldk + j] = __float2bfloat16_rn(0.f);
-                        zbits[(size_t)b * 2 * p.ldk + p.ldk + j] = __float2bfloat16_rn(0.f);
+                    for (int v = 0; v < n_vec; ++v) {
+                        const int seq = n_vec > 1 ? v : b;
+                        for (int j = p.k + et; j < p.ldk; j += DTC_EPI_THREADS) {
+                            zbits[(size_t)seq * 2 * p.ldk + j] = __float2bfloat16_rn(0.f);
+                            zbits[(size_t)seq * 2 * p.ldk + p.ldk + j] = __float2bfloat16_rn(0.f);
+                        }
                     }
             }
             if (!stop && half == 0) {
@@ -448,7 +487,20 @@ bool decode_tc_supported(const DecodeParams &p) {
     return true;
 }
 
-static void dtc_plan_half(DtcHalf &h, int n_rows, int mats, int row_elems, int set_rows, int sms) {
+// One expert set for all the sequences of the call (entries of `sets` that all name the same
+// buffers): the weights are streamed once and every staged row meets all B vectors in one MMA.
+bool decode_tc_shared(const DecodeParams &p) {
+    if (p.B < 2 || p.B > DTC_MAX_VEC || !decode_tc_supported(p)) return false;
+    for (int b = 1; b < p.B; ++b)
+        if (p.seq[b].w_gate != p.seq[0].w_gate || p.seq[b].w_up != p.seq[0].w_up || p.seq[b].w_down != p.seq[0].w_down ||
+            p.seq[b].b_gate != p.seq[0].b_gate || p.seq[b].b_up != p.seq[0].b_up)
+            return false;
+    const int groups = ((8 * p.B + 15) / 16) * 2;
+    const size_t stride = ((size_t)max(p.d, p.ldk) * 2 + 255) & ~(size_t)255;
+    return groups * stride <= 112 * 1024;  // the vectors must leave room for a ring of three stages
+}
+
+static void dtc_plan_half(DtcHalf &h, int n_rows, int mats, int row_elems, int set_rows, int acc_cols, int sms) {
     h.n_rows = n_rows;
     h.n_slices = slices_for(n_rows, sms);
     h.set_rows = set_rows;
@@ -459,8 +511,9 @@ static void dtc_plan_half(DtcHalf &h, int n_rows, int mats, int row_elems, int s
     // all sets of the largest item keep their accumulators until its epilogue
     const int rows_max = (n_rows + h.n_slices - 1) / h.n_slices;
     const int sets_max = (rows_max * mats + set_rows - 1) / set_rows;
+    h.acc_cols = acc_cols;
     h.n_acc = 8;
-    while (h.n_acc > 1 && (sets_max * h.n_acc * 16 > DTC_TMEM_COLS || h.n_acc > h.windows)) h.n_acc >>= 1;  // (each is written at least once)
+    while (h.n_acc > 1 && (sets_max * h.n_acc * acc_cols > DTC_TMEM_COLS || h.n_acc > h.windows)) h.n_acc >>= 1;  // (each is written at least once)
 }
 
 griffin_status decode_bf16_tc(DecodeParams &p, int act, uint32_t flags, cudaStream_t stream) {
@@ -469,11 +522,24 @@ griffin_status decode_bf16_tc(DecodeParams &p, int act, uint32_t flags, cudaStre
     if (!decode_tc_supported(p)) return GRIFFIN_ERR_UNSUPPORTED;
     const bool overlap = (flags & GRIFFIN_DECODE_OVERLAP_WEIGHT_PREFETCH) != 0;
     DtcPlan pl;
-    dtc_plan_half(pl.h[0], p.k, 2, p.d, GRIFFIN_DTC_SET_ROWS_0, sms);
-    dtc_plan_half(pl.h[1], p.d, 1, p.ldk, GRIFFIN_DTC_SET_ROWS_1, sms);
-    pl.h[1].sbo_b = p.ldk * 2;  // z_lo lies behind z_hi
-    const int vec_need = max(p.d * 2, p.ldk * 4);
-    pl.vec_bytes = (vec_need + 127) & ~127;
+    const bool shared = decode_tc_shared(p);
+    pl.n_vec = shared ? p.B : 1;
+    pl.vec_stride = (max(p.d, p.ldk) * 2 + 255) & ~255;
+    const int acc_cols = shared ? ((8 * p.B + 15) / 16) * 16 : 16;
+    dtc_plan_half(pl.h[0], p.k, 2, p.d, GRIFFIN_DTC_SET_ROWS_0, acc_cols, sms);
+    dtc_plan_half(pl.h[1], p.d, 1, p.ldk, GRIFFIN_DTC_SET_ROWS_1, acc_cols, sms);
+    if (shared) {
+        pl.h[0].sbo_b = pl.h[1].sbo_b = pl.vec_stride;  // the next 8 rows of B are the next vector
+        pl.vec_bytes = (acc_cols / 8) * pl.vec_stride;   // (an odd number of vectors: the MMA reads one more, unused)
+    } else {
+        pl.h[1].sbo_b = p.ldk * 2;  // z_lo lies behind z_hi
+        pl.vec_bytes = (max(p.d * 2, p.ldk * 4) + 127) & ~127;
+    }
+    // every set of the largest item keeps its accumulators until the item's epilogue
+    for (int i = 0; i < 2; ++i)
+        if (((pl.h[i].n_rows + pl.h[i].n_slices - 1) / pl.h[i].n_slices * (i ? 1 : 2) + pl.h[i].set_rows - 1) / pl.h[i].set_rows *
+                pl.h[i].n_acc * acc_cols > DTC_TMEM_COLS)
+            return GRIFFIN_ERR_UNSUPPORTED;
     pl.n_stages = 0;
     for (int n = DTC_MAX_STAGES; n >= 2; --n) {
         pl.n_stages = n;

@@ -176,6 +176,36 @@ def test_decode_tcgen05_kernel_matches_oracle_and_default_kernel(d, d_ff, k, B):
     assert torch.equal(y_tc, y_tc2) and torch.equal(y_tc, y_tc3)   # deterministic, launch mode does not matter
 
 
+# One expert set for all sequences of a call (Eq. 7): d, d_ff, k, B, activation, biases
+SHARED_SET_SHAPES = [
+    (512, 1536, 768, 2, "geglu_tanh", True),
+    (4096, 11008, 5504, 3, "swiglu", False),   # an odd number of vectors
+    (4096, 11008, 5504, 8, "swiglu", False),   # the most that one call streams together
+    (2048, 5632, 2816, 5, "reglu", True),
+    (8192, 1024, 512, 8, "swiglu", False),     # the vectors would not leave room for the ring: one pass per sequence
+    (1000, 1504, 751, 4, "swiglu", False),     # shapes that only the warp-level kernel takes
+]
+
+
+@pytest.mark.parametrize("d,d_ff,k,B,act,bias", SHARED_SET_SHAPES)
+def test_decode_with_one_shared_set_matches_oracle_and_separate_calls(d, d_ff, k, B, act, bias):
+    L, host = make_layer(d, d_ff, "bf16", act=act, bias=bias, seed=7 * d + k, n_seq=B)
+    rs = np.random.default_rng(d + k + B)
+    x = rand((B, d), torch.bfloat16, 97)
+    e_np = np.sort(rs.choice(d_ff, size=k, replace=False)).astype(np.int32)
+    cs = L.compact(torch.from_numpy(e_np).to(dev()))
+    c = O.compact_experts(e_np, h64(host, "wg"), h64(host, "wu"), h64(host, "wd"), h64(host, "bg"), h64(host, "bu"))
+    ref = O.ff_pruned(np64(x), c, act, h64(host, "bd"))
+    y = L.decode([cs] * B, x)
+    y2 = L.decode([cs] * B, x, G.DECODE_OVERLAP_WEIGHT_PREFETCH)
+    assert L.status() == G.OK
+    assert torch.equal(y, y2)
+    for b in range(B):
+        assert rel_l2(np64(y[b]), ref[b]) < TOL_OUT["bf16"], b
+        y1 = L.decode([cs], x[b:b + 1])   # the same sequence on its own
+        assert rel_l2(np64(y[b]), np64(y1[0])) < TOL_OUT["bf16"], b
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_decode_with_all_neurons_is_the_dense_ff(dtype):
     d, d_ff = 512, 1536
