@@ -52,6 +52,7 @@ constexpr int DTC_SLOT_BYTES = 32 * 1024;  // one stage of the ring
 constexpr int DTC_MAX_STAGES = 7;
 constexpr int DTC_MAX_SETS = 16;           // sets per work item (128 rows of 8)
 constexpr int DTC_TMEM_COLS = 512;         // 32 accumulators of 16 columns
+constexpr int DTC_STAGING_DEPTH = 12;      // 16-byte loads that a thread keeps in flight while it stages a vector
 constexpr int DTC_MAX_VEC = 8;             // vectors that may share one expert set in a call
 #ifndef GRIFFIN_DTC_SET_ROWS_0
 #define GRIFFIN_DTC_SET_ROWS_0 16
@@ -223,6 +224,9 @@ __device__ __forceinline__ bool dtc_issue_half(const DecodeParams &p, const DtcP
     return true;
 }
 
+// SHARED: one expert set for all the vectors of the call (see decode_tc_shared); otherwise one
+// vector per work item.
+template <bool SHARED>
 __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_constant__ DecodeParams p,
                                                                 const __grid_constant__ DtcPlan pl, int act) {
     extern __shared__ uint8_t smem_raw[];
@@ -348,30 +352,116 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                 const int R = r1 - r0;
                 const int n_rows_item = half ? R : 2 * R;
                 const int n_sets = (n_rows_item + h.set_rows - 1) / h.set_rows;
+                if constexpr (!SHARED) {
+                if (b != cur_b) {
+                    // the vector, read through L2 (x comes from earlier work on the stream, z from
+                    // other CTAs of this grid): x, or z_hi then z_lo, as they lie in memory
+                    const int n_units = h.windows * (DTC_WINDOW / 16) * (half ? 2 : 1);
+                    const uint4 *src = half ? reinterpret_cast<const uint4 *>(zbits + (size_t)b * 2 * p.ldk)
+                                            : reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(p.x) +
+                                                                              (size_t)b * p.d);
+                    uint4 *dst = reinterpret_cast<uint4 *>(s.vec);
+                    for (int u0 = et; u0 < n_units; u0 += 4 * DTC_EPI_THREADS) {
+                        uint4 v[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {  // all loads of a round are in flight together
+                            const int u = u0 + j * DTC_EPI_THREADS;
+                            v[j] = u < n_units ? __ldcg(src + u) : make_uint4(0, 0, 0, 0);
+                        }
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int u = u0 + j * DTC_EPI_THREADS;
+                            if (u < n_units) dst[u] = v[j];
+                        }
+                    }
+                    fence_proxy_async_smem();  // the MMA reads shared memory through the async proxy
+                    cur_b = b;
+                }
+                tc_fence_before_sync();
+                if (epi_barrier_or(*s.abort != 0)) {
+                    stop = true;
+                    break;
+                }
+                if (et == 0) mbar_arrive(s.vec_full);
+                const bool got = __all_sync(
+                    0xffffffffu, wait_or_abort_relaxed(s.acc_full, n_item & 1, s.abort, p.ws, 36 + half));  // (tcgen05.ld is warp-wide)
+                tc_fence_after_sync();
+                if (got) {
+                    const uint32_t taddr = tmem_base + ((uint32_t)(wq * 32) << 16);
+#pragma unroll 1
+                    for (int set = 0; set < n_sets; ++set) {
+                        float val = 0.f;
+                        for (int a = 0; a < h.n_acc; ++a) {  // (a fixed order: results are reproducible)
+                            float v[16];
+                            tmem_ld16(taddr + (uint32_t)(set * h.n_acc + a) * 16u, v);
+#pragma unroll
+                            for (int c = 0; c < 8; ++c)
+                                if (c == unit) val += half ? v[c] + v[8 + c] : v[c];
+                        }
+                        // the 8 units of a weight row sit in 8 consecutive lanes
+                        val += __shfl_xor_sync(0xffffffffu, val, 1);
+                        val += __shfl_xor_sync(0xffffffffu, val, 2);
+                        val += __shfl_xor_sync(0xffffffffu, val, 4);
+                        if (unit == 0) s.part[set * 16 + row_in_set] = val;
+                    }
+                }
+                tc_fence_before_sync();
+                if (epi_barrier_or(!got)) {
+                    stop = true;
+                    break;
+                }
+                // thread t finishes row r0 + t of the item
+                if (et < R) {
+                    const int row = r0 + et;
+                    if (!half) {
+                        const int iu = R + et;  // the up row's place in the item
+                        float a0 = s.part[(et / h.set_rows) * 16 + et % h.set_rows];
+                        float a1 = s.part[(iu / h.set_rows) * 16 + iu % h.set_rows];
+                        if (p.seq[b].b_gate) a0 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[b].b_gate)[row]);
+                        if (p.seq[b].b_up) a1 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[b].b_up)[row]);
+                        const float zv = sigma_rt(act, a0) * a1;
+                        const __nv_bfloat16 hi = __float2bfloat16_rn(zv);
+                        zbits[(size_t)b * 2 * p.ldk + row] = hi;
+                        zbits[(size_t)b * 2 * p.ldk + p.ldk + row] = __float2bfloat16_rn(zv - __bfloat162float(hi));
+                    } else {
+                        float acc = s.part[(et / h.set_rows) * 16 + et % h.set_rows];
+                        if (p.b_down) acc += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.b_down)[row]);
+                        static_cast<__nv_bfloat16 *>(p.y)[(size_t)b * p.d + row] = __float2bfloat16_rn(acc);
+                    }
+                }
+                if (!half && sl == h.n_slices - 1)  // the last slice also clears the padding of z
+                    for (int j = p.k + et; j < p.ldk; j += DTC_EPI_THREADS) {
+                        zbits[(size_t)b * 2 * p.ldk + j] = __float2bfloat16_rn(0.f);
+                        zbits[(size_t)b * 2 * p.ldk + p.ldk + j] = __float2bfloat16_rn(0.f);
+                    }
+                } else {
                 if (b != cur_b) {
                     // the vector(s), read through L2 (x comes from earlier work on the stream, z from
                     // other CTAs of this grid).  One vector: x, or z_hi then z_lo, as they lie in
                     // memory.  A shared set: x (or z_hi) of every sequence, vec_stride bytes apart.
                     const int row_units = h.windows * (DTC_WINDOW / 16);
                     const int n_units = n_vec > 1 ? row_units : row_units * (half ? 2 : 1);
-                    for (int v = 0; v < n_vec; ++v) {
-                        const int seq = n_vec > 1 ? v : b;
-                        const uint4 *src = half ? reinterpret_cast<const uint4 *>(zbits + (size_t)seq * 2 * p.ldk)
-                                                : reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(p.x) +
-                                                                                  (size_t)seq * p.d);
-                        uint4 *dst = reinterpret_cast<uint4 *>(s.vec + (size_t)v * pl.vec_stride);
-                        for (int u0 = et; u0 < n_units; u0 += 4 * DTC_EPI_THREADS) {
-                            uint4 t[4];
+                    // (plain loads: a bulk copy would queue behind the producer's weight copies; the
+                    // units of all vectors are shared out together so that many loads are in flight)
+                    const size_t src_stride = half ? (size_t)2 * p.ldk * 2 : (size_t)p.d * 2;  // bytes between sequences
+                    const uint8_t *src0 = half ? reinterpret_cast<const uint8_t *>(zbits) : static_cast<const uint8_t *>(p.x);
+                    const int total = n_vec * n_units;
+                    for (int e0 = et; e0 < total; e0 += DTC_STAGING_DEPTH * DTC_EPI_THREADS) {
+                        uint4 t[DTC_STAGING_DEPTH];
+                        int v = e0 / n_units, u = e0 - v * n_units;  // (vector, unit) of this thread's first load of the round
+                        const int v0 = v, u0 = u;
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) {  // all loads of a round are in flight together
-                                const int u = u0 + j * DTC_EPI_THREADS;
-                                t[j] = u < n_units ? __ldcg(src + u) : make_uint4(0, 0, 0, 0);
-                            }
+                        for (int j = 0; j < DTC_STAGING_DEPTH; ++j) {  // all loads of a round are in flight together
+                            t[j] = e0 + j * DTC_EPI_THREADS < total
+                                       ? __ldcg(reinterpret_cast<const uint4 *>(src0 + (size_t)v * src_stride) + u)
+                                       : make_uint4(0, 0, 0, 0);
+                            for (u += DTC_EPI_THREADS; u >= n_units; u -= n_units) ++v;
+                        }
+                        v = v0, u = u0;
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                const int u = u0 + j * DTC_EPI_THREADS;
-                                if (u < n_units) dst[u] = t[j];
-                            }
+                        for (int j = 0; j < DTC_STAGING_DEPTH; ++j) {
+                            if (e0 + j * DTC_EPI_THREADS < total) reinterpret_cast<uint4 *>(s.vec + (size_t)v * pl.vec_stride)[u] = t[j];
+                            for (u += DTC_EPI_THREADS; u >= n_units; u -= n_units) ++v;
                         }
                     }
                     fence_proxy_async_smem();  // the MMA reads shared memory through the async proxy
@@ -458,6 +548,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                             zbits[(size_t)seq * 2 * p.ldk + p.ldk + j] = __float2bfloat16_rn(0.f);
                         }
                     }
+                }
             }
             if (!stop && half == 0) {
                 // ---- the meeting point: this CTA's z entries are written; the thread that reports in makes them visible
@@ -548,7 +639,7 @@ griffin_status decode_bf16_tc(DecodeParams &p, int act, uint32_t flags, cudaStre
     const size_t smem = dtc_smem_bytes(pl);
     if (smem > 227 * 1024) return GRIFFIN_ERR_UNSUPPORTED;
     // every CTA of the grid must be able to run at the same time (they meet half-way): one per SM
-    const void *fn = (const void *)decode_tc_kernel;
+    const void *fn = shared ? (const void *)decode_tc_kernel<true> : (const void *)decode_tc_kernel<false>;
     if (ensure_dynamic_smem(fn, smem) != cudaSuccess) return GRIFFIN_ERR_CUDA;
     void *args[] = {&p, &pl, &act};
     if (launch_maybe_overlapped(fn, dim3(sms), dim3(DTC_THREADS), smem, stream, overlap, args) != cudaSuccess)
