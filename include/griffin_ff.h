@@ -59,7 +59,8 @@ typedef enum {
 typedef enum {
     GRIFFIN_ACT_SWIGLU = 0,       /* sigma(t) = t / (1 + exp(-t))                                   */
     GRIFFIN_ACT_GEGLU_TANH = 1,   /* sigma(t) = t/2 (1 + tanh(sqrt(2/pi) (t + 0.044715 t^3)))       */
-    GRIFFIN_ACT_REGLU = 2         /* sigma(t) = max(t, 0)                                           */
+    GRIFFIN_ACT_REGLU = 2,        /* sigma(t) = max(t, 0)                                           */
+    GRIFFIN_ACT_GEGLU_ERF = 3     /* sigma(t) = t/2 (1 + erf(t / sqrt(2)))                          */
 } griffin_act;
 
 typedef enum { GRIFFIN_DT_F32 = 0, GRIFFIN_DT_BF16 = 1 } griffin_dtype;

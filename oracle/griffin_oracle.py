@@ -39,7 +39,10 @@ import numpy as np
 SWIGLU = "swiglu"
 GEGLU_TANH = "geglu_tanh"
 REGLU = "reglu"
-ACTIVATIONS = (SWIGLU, GEGLU_TANH, REGLU)
+GEGLU_ERF = "geglu_erf"
+ACTIVATIONS = (SWIGLU, GEGLU_TANH, REGLU, GEGLU_ERF)
+
+_erf = np.vectorize(math.erf, otypes=[np.float64])
 
 
 def _f64(a):
@@ -54,6 +57,7 @@ def sigma(t, act):
       swiglu      sigma(t) = t / (1 + exp(-t))                       (SiLU)
       geglu_tanh  sigma(t) = t/2 * (1 + tanh(sqrt(2/pi) (t + 0.044715 t^3)))
       reglu       sigma(t) = max(t, 0)
+      geglu_erf   sigma(t) = t/2 * (1 + erf(t / sqrt(2)))            (exact GELU)
     """
     t = _f64(t)
     if act == SWIGLU:
@@ -63,6 +67,8 @@ def sigma(t, act):
         return 0.5 * t * (1.0 + np.tanh(math.sqrt(2.0 / math.pi) * (t + 0.044715 * t ** 3)))
     if act == REGLU:
         return np.maximum(t, 0.0)
+    if act == GEGLU_ERF:
+        return 0.5 * t * (1.0 + _erf(t / math.sqrt(2.0)))
     raise ValueError(f"unknown activation {act!r}")
 
 

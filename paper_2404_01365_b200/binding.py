@@ -15,12 +15,12 @@ import torch
 from . import build as _build
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(7)
-ACT_SWIGLU, ACT_GEGLU_TANH, ACT_REGLU = 0, 1, 2
+ACT_SWIGLU, ACT_GEGLU_TANH, ACT_REGLU, ACT_GEGLU_ERF = 0, 1, 2, 3
 DT_F32, DT_BF16 = 0, 1
 DECODE_DEFAULT, DECODE_OVERLAP_WEIGHT_PREFETCH, DECODE_TCGEN05 = 0, 1, 2
 MAX_BATCH = 32
 
-ACT_BY_NAME = {"swiglu": ACT_SWIGLU, "geglu_tanh": ACT_GEGLU_TANH, "reglu": ACT_REGLU}
+ACT_BY_NAME = {"swiglu": ACT_SWIGLU, "geglu_tanh": ACT_GEGLU_TANH, "reglu": ACT_REGLU, "geglu_erf": ACT_GEGLU_ERF}
 DTYPE_BY_NAME = {"f32": DT_F32, "bf16": DT_BF16}
 
 EXPORTS = (

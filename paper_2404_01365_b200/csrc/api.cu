@@ -53,7 +53,8 @@ static griffin_status check_desc(const griffin_ff_desc *desc) {
     if (desc->d < 8 || desc->d_ff < 8) return GRIFFIN_ERR_INVALID_ARG;
     if (desc->d % 8 != 0 || desc->d_ff % 8 != 0) return GRIFFIN_ERR_ALIGNMENT;
     if (desc->dtype != GRIFFIN_DT_F32 && desc->dtype != GRIFFIN_DT_BF16) return GRIFFIN_ERR_UNSUPPORTED;
-    if (desc->act != GRIFFIN_ACT_SWIGLU && desc->act != GRIFFIN_ACT_GEGLU_TANH && desc->act != GRIFFIN_ACT_REGLU)
+    if (desc->act != GRIFFIN_ACT_SWIGLU && desc->act != GRIFFIN_ACT_GEGLU_TANH && desc->act != GRIFFIN_ACT_REGLU &&
+        desc->act != GRIFFIN_ACT_GEGLU_ERF)
         return GRIFFIN_ERR_UNSUPPORTED;
     return GRIFFIN_OK;
 }

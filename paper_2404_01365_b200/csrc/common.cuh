@@ -71,6 +71,8 @@ template <int ACT> __device__ __forceinline__ float sigma(float t) {
         // tanh(a) = 1 - 2 / (exp(2a) + 1); an overflowing exp still gives the right limit
         const float th = 1.0f - 2.0f / (__expf(2.0f * inner) + 1.0f);
         return 0.5f * t * (1.0f + th);
+    } else if constexpr (ACT == GRIFFIN_ACT_GEGLU_ERF) {
+        return 0.5f * t * (1.0f + erff(t * 0.70710678118654752f));
     } else {
         return fmaxf(t, 0.0f);
     }
@@ -80,6 +82,7 @@ __device__ __forceinline__ float sigma_rt(int act, float t) {
     switch (act) {
         case GRIFFIN_ACT_SWIGLU: return sigma<GRIFFIN_ACT_SWIGLU>(t);
         case GRIFFIN_ACT_GEGLU_TANH: return sigma<GRIFFIN_ACT_GEGLU_TANH>(t);
+        case GRIFFIN_ACT_GEGLU_ERF: return sigma<GRIFFIN_ACT_GEGLU_ERF>(t);
         default: return sigma<GRIFFIN_ACT_REGLU>(t);
     }
 }

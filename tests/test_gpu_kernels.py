@@ -119,7 +119,7 @@ DECODE_SHAPES = [
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("d,d_ff,k,B", DECODE_SHAPES)
 def test_decode_matches_oracle(dtype, d, d_ff, k, B):
-    act = "geglu_tanh" if d == 3072 else "swiglu"
+    act = {3072: "geglu_tanh", 2048: "geglu_erf", 1000: "reglu"}.get(d, "swiglu")
     L, host = make_layer(d, d_ff, dtype, act=act, bias=(d_ff < 2000), seed=d + k, n_seq=B)
     rs = np.random.default_rng(d + k)
     x = rand((B, d), TD[dtype], 99)
@@ -182,6 +182,7 @@ SHARED_SET_SHAPES = [
     (4096, 11008, 5504, 3, "swiglu", False),   # an odd number of vectors
     (4096, 11008, 5504, 8, "swiglu", False),   # the most that one call streams together
     (2048, 5632, 2816, 5, "reglu", True),
+    (1024, 2816, 1408, 2, "geglu_erf", True),
     (8192, 1024, 512, 8, "swiglu", False),     # the vectors would not leave room for the ring: one pass per sequence
     (1000, 1504, 751, 4, "swiglu", False),     # shapes that only the warp-level kernel takes
 ]
@@ -243,7 +244,7 @@ PREFILL_SHAPES = [(64, 256, 688), (1, 64, 96), (37, 72, 200), (130, 512, 1032), 
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-@pytest.mark.parametrize("act", ["swiglu", "geglu_tanh", "reglu"])
+@pytest.mark.parametrize("act", ["swiglu", "geglu_tanh", "reglu", "geglu_erf"])
 @pytest.mark.parametrize("S,d,d_ff", PREFILL_SHAPES)
 def test_prefill_score_matches_oracle(dtype, act, S, d, d_ff):
     L, host = make_layer(d, d_ff, dtype, act=act, bias=(S == 37), seed=S + d, S_max=S)

@@ -44,6 +44,15 @@ def test_sigma_closed_form_values():
     assert O.sigma(np.array([1.0]), O.SWIGLU)[0] == pytest.approx(0.7310585786300049, abs=1e-15)
     assert O.sigma(np.array([1.0]), O.GEGLU_TANH)[0] == pytest.approx(0.8411919906082768, abs=1e-12)
     assert O.sigma(np.array([-3.0, 2.5]), O.REGLU).tolist() == [0.0, 2.5]
+    # exact GELU: t * Phi(t) with Phi the standard normal distribution function; Phi(1) = 0.8413447460685429,
+    # Phi(-1.96) = 0.024997895148220435; g(t) - g(-t) = t; close to, but not the same as, the tanh form.
+    ge = O.sigma(t, O.GEGLU_ERF)
+    assert ge - ge[::-1] == pytest.approx(t, abs=1e-14)
+    assert O.sigma(np.array([1.0]), O.GEGLU_ERF)[0] == pytest.approx(0.8413447460685429, abs=1e-15)
+    assert O.sigma(np.array([-1.96]), O.GEGLU_ERF)[0] == pytest.approx(-1.96 * 0.024997895148220435, abs=1e-15)
+    assert O.sigma(np.array([0.0, 40.0]), O.GEGLU_ERF).tolist() == [0.0, 40.0]
+    assert 1e-4 < abs(O.sigma(np.array([1.0]), O.GEGLU_ERF)[0] - O.sigma(np.array([1.0]), O.GEGLU_TANH)[0]) < 3e-4
+    assert np.max(np.abs(ge - g)) < 1e-3
 
 
 def test_sigma_swiglu_is_t_times_logistic_and_stable():
@@ -58,7 +67,8 @@ def test_sigma_swiglu_is_t_times_logistic_and_stable():
 # ------------------------------------------------------- dense FF (Eq.1,3) ---
 
 def _brute_ff(x, wg, wu, wd, act, bg=None, bu=None, bd=None):
-    f = {"swiglu": _silu, "geglu_tanh": _gelu_tanh, "reglu": lambda t: max(t, 0.0)}[act]
+    f = {"swiglu": _silu, "geglu_tanh": _gelu_tanh, "reglu": lambda t: max(t, 0.0),
+         "geglu_erf": lambda t: 0.5 * t * math.erfc(-t / math.sqrt(2.0))}[act]
     S, d = len(x), len(x[0])
     n = len(wg)
     Z = [[0.0] * n for _ in range(S)]
