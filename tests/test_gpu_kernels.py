@@ -238,6 +238,37 @@ def test_decode_many_steps_back_to_back_with_overlap():
     assert rel_l2(np64(ys), ref) < TOL_OUT["bf16"]
 
 
+def test_decode_calls_replayed_from_a_cuda_graph_give_the_same_bits():
+    """bench.py captures the decode calls of a step once and replays them: same kernels, same
+    launch attributes (the overlapped-launch edges included), so the same bits."""
+    d, d_ff, k, n = 1024, 2816, 1408, 6
+    L, host = make_layer(d, d_ff, "bf16", seed=5)
+    cs = L.compact(torch.arange(0, d_ff, 2, dtype=torch.int32, device=dev()))
+    arr = G.compact_array([cs])
+    xs = rand((n, d), torch.bfloat16, 12).to(dev())
+    y_direct, y_graph = torch.empty_like(xs), torch.zeros_like(xs)
+
+    def calls(out):
+        for t in range(n):
+            G.griffin_ff_decode(L.desc, arr, None, xs[t:t + 1], out[t:t + 1], L.ws,
+                                G.DECODE_OVERLAP_WEIGHT_PREFETCH if t > 0 else G.DECODE_DEFAULT)
+
+    calls(y_direct)
+    torch.cuda.synchronize()
+    g, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            calls(y_graph)
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(3):
+        y_graph.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(y_graph, y_direct)
+    assert L.status() == G.OK
+
+
 # ---------------------------------------------------------------- prefill ---
 
 PREFILL_SHAPES = [(64, 256, 688), (1, 64, 96), (37, 72, 200), (130, 512, 1032), (256, 1024, 2816)]
