@@ -49,7 +49,10 @@ PrefillScratch prefill_scratch(const griffin_ff_desc *desc, int S) {
     if (desc->dtype != GRIFFIN_DT_F32) {
         int bn = 0, splits = 1;
         gemm2_plan(S, desc->d, &bn, &splits);
-        if (splits > 1) off = align_up(off + (size_t)splits * S * desc->d * sizeof(float), 256);
+        size_t need = splits > 1 ? (size_t)splits * S * desc->d * sizeof(float) : 0;
+        const size_t tail = gemm1_tail_bytes(S, desc->d, desc->d_ff);  // (used up before the down projection starts)
+        if (tail > need) need = tail;
+        if (need > 0) off = align_up(off + need, 256);
     }
     ps.total = off;
     return ps;

@@ -47,7 +47,43 @@ struct TcParams {
     float *part;                         // splits > 1: fp32 partial outputs [splits, S, n_total]
     int act;
     void *ws;
+    // DUAL only: tiles from tail_first on are cut along K into tail_ks parts (tail_ks = 1: none is),
+    // whose raw accumulators (gate | up, fp32) go to tail_part [part][128 rows][256 columns]
+    int tail_first, tail_ks;
+    float *tail_part;
 };
+
+// Work item -> (row block m, column block n, K blocks [kb0, kb1), index of the cut tile's part or -1).
+// Uniform K splits (the down projection) number the items split-major; the cut tiles of the first GEMM
+// follow the whole ones.
+struct TcItem {
+    int m, n, sp, kb0, kb1, part;
+};
+__device__ __forceinline__ TcItem tc_item(const TcParams &p, int item, int kb_total) {
+    TcItem t;
+    const int tiles = p.m_tiles * p.n_tiles;
+    int tile = item, ks = p.splits;
+    t.sp = 0;
+    t.part = -1;
+    if (p.tail_ks > 1) {
+        ks = 1;
+        if (item >= p.tail_first) {
+            const int j = item - p.tail_first;
+            ks = p.tail_ks;
+            tile = p.tail_first + j / ks;
+            t.sp = j - (j / ks) * ks;
+            t.part = j;
+        }
+    } else if (ks > 1) {
+        t.sp = item / tiles;
+        tile = item - t.sp * tiles;
+    }
+    t.m = tile % p.m_tiles;  // tiles sharing weights are neighbours
+    t.n = tile / p.m_tiles;
+    t.kb0 = t.sp * kb_total / ks;
+    t.kb1 = (t.sp + 1) * kb_total / ks;
+    return t;
+}
 
 struct TcSmem {
     uint8_t *stages;
@@ -97,7 +133,9 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
     tc_fence_after_sync();
     const uint32_t tmem_base = *s.tmem_slot;
 
-    const int n_tiles_total = p.m_tiles * p.n_tiles * p.splits;  // work items: (m, n, K split)
+    // work items: (m, n, K split), or whole tiles followed by the parts of the cut ones
+    const int n_tiles_total = p.tail_ks > 1 ? p.tail_first + (p.m_tiles * p.n_tiles - p.tail_first) * p.tail_ks
+                                            : p.m_tiles * p.n_tiles * p.splits;
     const int kb_total = p.K / TC_BK;
 
     if (warp == 0) {
@@ -106,9 +144,8 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
             uint32_t it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < n_tiles_total; tile += gridDim.x) {
-                const int m = tile % p.m_tiles, rest = tile / p.m_tiles;  // tiles sharing weights are neighbours
-                const int n = rest % p.n_tiles, sp = rest / p.n_tiles;
-                const int kb0 = sp * kb_total / p.splits, kb1 = (sp + 1) * kb_total / p.splits;
+                const TcItem ti = tc_item(p, tile, kb_total);
+                const int m = ti.m, n = ti.n, kb0 = ti.kb0, kb1 = ti.kb1;
                 for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const int stage = it % TC_STAGES;
                     const uint32_t use = it / TC_STAGES;
@@ -142,8 +179,8 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
                 if (acc_use > 0 && !wait_or_abort(&s.acc_empty[acc], (acc_use - 1) & 1, s.abort, p.ws, 21)) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * NT);
-                const int sp = tile / (p.m_tiles * p.n_tiles);
-                const int kb0 = sp * kb_total / p.splits, kb1 = (sp + 1) * kb_total / p.splits;
+                const TcItem ti = tc_item(p, tile, kb_total);
+                const int kb0 = ti.kb0, kb1 = ti.kb1;
                 for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const int stage = it % TC_STAGES;
                     if (!wait_or_abort(&s.full[stage], (it / TC_STAGES) & 1, s.abort, p.ws, 22)) {
@@ -167,15 +204,27 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
         const int row_in_tile = wq * 32 + lane;  // one output row per thread
         uint32_t tcount = 0;
         for (int tile = blockIdx.x; tile < n_tiles_total; tile += gridDim.x, ++tcount) {
-            const int m = tile % p.m_tiles, rest = tile / p.m_tiles;
-            const int n = rest % p.n_tiles, sp = rest / p.n_tiles;
+            const TcItem ti = tc_item(p, tile, kb_total);
+            const int m = ti.m, n = ti.n, sp = ti.sp;
             const int acc = tcount & 1;
             if (!wait_or_abort(&s.acc_full[acc], (tcount >> 1) & 1, s.abort, p.ws, 23)) break;
             tc_fence_after_sync();
             const int row = m * TC_BM + row_in_tile;
             const bool live = row < p.S;
             const uint32_t taddr = tmem_base + ((uint32_t)(wq * 32) << 16) + (uint32_t)(acc * NT);
-            if (DUAL) {
+            if (DUAL && ti.part >= 0) {
+                // a part of a cut tile: the raw accumulators leave in fp32 (gate | up); the finishing
+                // kernel adds the parts and does what the epilogue below does
+                float *dst = p.tail_part + ((size_t)ti.part * TC_BM + row_in_tile) * 256;
+#pragma unroll 1
+                for (int c = 0; c < 256; c += 32) {
+                    float a[32];
+                    tmem_ld32(taddr + c, a);
+#pragma unroll
+                    for (int v = 0; v < 8; ++v)
+                        reinterpret_cast<float4 *>(dst + c)[v] = make_float4(a[4 * v], a[4 * v + 1], a[4 * v + 2], a[4 * v + 3]);
+                }
+            } else if (DUAL) {
                 float sq = 0.f;
 #pragma unroll 1
                 for (int c = 0; c < 128; c += 32) {
@@ -253,6 +302,40 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
     }
 }
 
+// Finishes the cut tiles of the first GEMM: one warp per (cut tile, row), four neurons of the tile per
+// lane.  The parts are added in order, then bias, activation and gating as in the epilogue above:
+// Z in bf16 and fp32, and the row's sum of squares over the tile's 128 columns (fixed order).
+__global__ void __launch_bounds__(128) dual_tail_finish_kernel(TcParams p) {
+    const int w = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    const int tile = p.tail_first + w / TC_BM, r = w % TC_BM, c = lane * 4;
+    const int m = tile % p.m_tiles, n = tile / p.m_tiles;
+    const int row = m * TC_BM + r, col = n * 128 + c;
+    float4 g = make_float4(0.f, 0.f, 0.f, 0.f), u = g;
+    for (int sp = 0; sp < p.tail_ks; ++sp) {
+        const float *src = p.tail_part + ((size_t)((tile - p.tail_first) * p.tail_ks + sp) * TC_BM + r) * 256;
+        const float4 a = *reinterpret_cast<const float4 *>(src + c), b = *reinterpret_cast<const float4 *>(src + 128 + c);
+        g.x += a.x; g.y += a.y; g.z += a.z; g.w += a.w;
+        u.x += b.x; u.y += b.y; u.z += b.z; u.w += b.w;
+    }
+    float gv[4] = {g.x, g.y, g.z, g.w}, uv[4] = {u.x, u.y, u.z, u.w}, z[4];
+    float sq = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if (p.bias0) gv[i] += __bfloat162float(p.bias0[col + i]);
+        if (p.bias1) uv[i] += __bfloat162float(p.bias1[col + i]);
+        z[i] = sigma_rt(p.act, gv[i]) * uv[i];
+        sq = fmaf(z[i], z[i], sq);
+    }
+    if (row < p.S) {
+        const __nv_bfloat162 h0 = __floats2bfloat162_rn(z[0], z[1]), h1 = __floats2bfloat162_rn(z[2], z[3]);
+        *reinterpret_cast<uint2 *>(p.out + (size_t)row * p.n_total + col) =
+            make_uint2(*reinterpret_cast<const uint32_t *>(&h0), *reinterpret_cast<const uint32_t *>(&h1));
+        *reinterpret_cast<float4 *>(p.zf + (size_t)row * p.n_total + col) = make_float4(z[0], z[1], z[2], z[3]);
+    }
+    sq = warp_sum(sq);
+    if (lane == 0 && row < p.S) p.rowsq[(size_t)row * p.n_tiles + n] = sq;
+}
+
 // y = bf16(sum over K splits of part + bias), four columns per thread, splits added in order.
 __global__ void splitk_reduce_kernel(const float *__restrict__ part, const __nv_bfloat16 *__restrict__ bias,
                                      __nv_bfloat16 *__restrict__ y, int splits, size_t n_elems, int n_total) {
@@ -277,6 +360,27 @@ __global__ void splitk_reduce_kernel(const float *__restrict__ part, const __nv_
 // Host side
 // ---------------------------------------------------------------------------------------
 constexpr int TC_TARGET_CTAS = 148;  // SMs of a B200: what a grid should fill
+
+void gemm1_tail_plan(int S, int d, int d_ff, int *tail_first, int *ks) {
+    const int tiles = ((S + TC_BM - 1) / TC_BM) * (d_ff / 128);
+    const int rem = tiles % TC_TARGET_CTAS;
+    *tail_first = tiles;
+    *ks = 1;
+    // (only where the last round is a large part of the whole: with many rounds the parts cost more than they save)
+    if (tiles > TC_TARGET_CTAS && tiles <= 4 * TC_TARGET_CTAS && rem > 0 && 2 * rem <= TC_TARGET_CTAS && d / TC_BK >= 16) {
+        const int k = TC_TARGET_CTAS / rem;
+        *ks = k > 4 ? 4 : k;
+        *tail_first = tiles - rem;
+    }
+}
+
+size_t gemm1_tail_bytes(int S, int d, int d_ff) {
+    int first = 0, ks = 1;
+    gemm1_tail_plan(S, d, d_ff, &first, &ks);
+    if (ks <= 1) return 0;
+    const int tiles = ((S + TC_BM - 1) / TC_BM) * (d_ff / 128);
+    return (size_t)(tiles - first) * ks * TC_BM * 256 * sizeof(float);
+}
 
 void gemm2_plan(int S, int d, int *bn, int *splits) {
     const int m_tiles = (S + TC_BM - 1) / TC_BM;
@@ -313,7 +417,8 @@ static griffin_status launch_tc(const CUtensorMap &ma, const CUtensorMap &mb0, c
     const size_t smem = 1024 + (size_t)TC_STAGES * (TC_BM * TC_BK * 2 + NT * TC_BK * 2) + TC_TAIL_BYTES;
     const void *fn = (const void *)ff_tc_kernel<DUAL, BN>;
     if (ensure_dynamic_smem(fn, smem) != cudaSuccess) return GRIFFIN_ERR_CUDA;
-    const int tiles = p.m_tiles * p.n_tiles * p.splits;
+    const int tiles = p.tail_ks > 1 ? p.tail_first + (p.m_tiles * p.n_tiles - p.tail_first) * p.tail_ks
+                                    : p.m_tiles * p.n_tiles * p.splits;
     ff_tc_kernel<DUAL, BN><<<tiles < sms ? tiles : sms, TC_THREADS, smem, stream>>>(ma, mb0, mb1, p);
     return cudaGetLastError() == cudaSuccess ? GRIFFIN_OK : GRIFFIN_ERR_CUDA;
 }
@@ -343,8 +448,14 @@ griffin_status launch_prefill_tc(const griffin_ff_desc *desc, const griffin_ff_w
     p.act = desc->act;
     p.ws = ws;
     p.splits = 1;
+    gemm1_tail_plan(S, d, d_ff, &p.tail_first, &p.tail_ks);
+    p.tail_part = ypart;  // (the down projection's partials use the same scratch, later)
     *n_col_tiles = p.n_tiles;
     griffin_status st = launch_tc<true, 128>(mx, mg, mu, p, sms, stream);
+    if (st == GRIFFIN_OK && p.tail_ks > 1) {
+        dual_tail_finish_kernel<<<(p.m_tiles * p.n_tiles - p.tail_first) * (TC_BM / 4), 128, 0, stream>>>(p);
+        if (cudaGetLastError() != cudaSuccess) st = GRIFFIN_ERR_CUDA;
+    }
     if (st == GRIFFIN_OK && after_ff1 != nullptr && cudaEventRecord(after_ff1, stream) != cudaSuccess) return GRIFFIN_ERR_CUDA;
     if (st != GRIFFIN_OK || y == nullptr) return st;
 
@@ -365,6 +476,7 @@ griffin_status launch_prefill_tc(const griffin_ff_desc *desc, const griffin_ff_w
     q.ws = ws;
     q.splits = splits;
     q.part = splits > 1 ? ypart : nullptr;
+    q.tail_ks = 1;
     st = bn == 256 ? launch_tc<false, 256>(mz, md, md, q, sms, stream) : launch_tc<false, 128>(mz, md, md, q, sms, stream);
     if (st != GRIFFIN_OK || splits == 1) return st;
     const size_t n_elems = (size_t)S * d;

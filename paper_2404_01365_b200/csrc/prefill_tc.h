@@ -13,6 +13,14 @@ namespace griffin {
 // arithmetic on the shape, so that workspace sizing and launch agree.
 void gemm2_plan(int S, int d, int *bn, int *splits);
 
+// The first GEMM has m_tiles x (d_ff / 128) tiles for one CTA per SM.  When the last round of
+// tiles would leave more than half of the SMs idle, those tiles are cut along K into *ks parts
+// (2..4) whose fp32 partial accumulators meet in a small finishing kernel: *tail_first is the
+// first tile that is cut (= the number of tiles when none is).  Pure arithmetic on the shape.
+void gemm1_tail_plan(int S, int d, int d_ff, int *tail_first, int *ks);
+// Bytes of fp32 scratch that the parts of the cut tiles need (0 when none is cut).
+size_t gemm1_tail_bytes(int S, int d, int d_ff);
+
 // Whether the tensor-core kernels take this shape (bf16, d and d_ff multiples of 64, ...).
 bool prefill_tc_supported(const griffin_ff_desc *desc, int S);
 

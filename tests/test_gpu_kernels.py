@@ -292,6 +292,25 @@ def test_prefill_score_matches_oracle(dtype, act, S, d, d_ff):
     assert np.array_equal(np64(s2), s)                   # deterministic; y is optional
 
 
+@pytest.mark.parametrize("S,d,d_ff", [(256, 1024, 10240), (200, 2048, 9728)])
+def test_prefill_with_a_cut_last_round_of_tiles(S, d, d_ff):
+    """160 (152) tiles of the first GEMM on 148 SMs: the last 12 (4) are cut along K into parts
+    whose partial accumulators meet in the finishing kernel."""
+    L, host = make_layer(d, d_ff, "bf16", act="geglu_tanh", bias=True, seed=S + d_ff, S_max=S)
+    x = rand((S, d), torch.bfloat16, 15) + rand((1, d), torch.bfloat16, 16, 4.0 / d ** 0.5)
+    y, s = L.prefill(x)
+    ref_y, ref_z = O.ff_dense(np64(x), h64(host, "wg"), h64(host, "wu"), h64(host, "wd"), "geglu_tanh",
+                              h64(host, "bg"), h64(host, "bu"), h64(host, "bd"))
+    ref_s = O.flock_score(ref_z)
+    assert L.status() == G.OK
+    assert rel_l2(np64(y), ref_y) < TOL_OUT["bf16"]
+    s = np64(s)
+    assert np.all(np.abs(s - ref_s) <= score_tol("bf16") * ref_s + 1e-6 * np.sqrt(S / d_ff))
+    assert abs(float(np.sum(s * s)) - S) < 1e-5 * S
+    _, s2 = L.prefill(x, want_y=False)
+    assert np.array_equal(np64(s2), s)
+
+
 def test_prefill_zero_row_contributes_nothing():
     S, d, d_ff = 16, 64, 96
     L, host = make_layer(d, d_ff, "f32", S_max=S)
