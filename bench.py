@@ -354,7 +354,11 @@ def run_ours(args, w, keep):
         # one top-k launch for all blocks; 2 compaction kernels; one fused kernel per decode call
         # (two for fp32 storage)
         split = w.dtype == "bf16" and ((S + 127) // 128) * (w.d // 256 if w.d % 256 == 0 else w.d // 128) <= 74
-        launches = L * B * (5 + (1 if split else 0)) + 1 + L * B * 2 + T * L * (1 if w.dtype == "bf16" else 2)
+        # ... and the finishing kernel of the first GEMM when its last round of 128x128 tiles is cut along K
+        g1_tiles = ((S + 127) // 128) * (w.d_ff // 128)
+        cut = (w.dtype == "bf16" and w.d % 128 == 0 and w.d_ff % 128 == 0 and 148 < g1_tiles <= 4 * 148
+               and 0 < g1_tiles % 148 <= 74 and w.d // 64 >= 16)
+        launches = L * B * (5 + (1 if split else 0) + (1 if cut else 0)) + 1 + L * B * 2 + T * L * (1 if w.dtype == "bf16" else 2)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
