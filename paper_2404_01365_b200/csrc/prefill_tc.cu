@@ -310,12 +310,20 @@ __global__ void __launch_bounds__(128) dual_tail_finish_kernel(TcParams p) {
     const int tile = p.tail_first + w / TC_BM, r = w % TC_BM, c = lane * 4;
     const int m = tile % p.m_tiles, n = tile / p.m_tiles;
     const int row = m * TC_BM + r, col = n * 128 + c;
-    float4 g = make_float4(0.f, 0.f, 0.f, 0.f), u = g;
-    for (int sp = 0; sp < p.tail_ks; ++sp) {
-        const float *src = p.tail_part + ((size_t)((tile - p.tail_first) * p.tail_ks + sp) * TC_BM + r) * 256;
-        const float4 a = *reinterpret_cast<const float4 *>(src + c), b = *reinterpret_cast<const float4 *>(src + 128 + c);
-        g.x += a.x; g.y += a.y; g.z += a.z; g.w += a.w;
-        u.x += b.x; u.y += b.y; u.z += b.z; u.w += b.w;
+    float4 g = make_float4(0.f, 0.f, 0.f, 0.f), u = g, a[4], b[4];
+#pragma unroll
+    for (int sp = 0; sp < 4; ++sp) {  // at most four parts; all loads in flight together
+        a[sp] = b[sp] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (sp < p.tail_ks) {
+            const float *src = p.tail_part + ((size_t)((tile - p.tail_first) * p.tail_ks + sp) * TC_BM + r) * 256;
+            a[sp] = __ldcs(reinterpret_cast<const float4 *>(src + c));
+            b[sp] = __ldcs(reinterpret_cast<const float4 *>(src + 128 + c));
+        }
+    }
+#pragma unroll
+    for (int sp = 0; sp < 4; ++sp) {  // added in order (absent parts are zeros)
+        g.x += a[sp].x; g.y += a[sp].y; g.z += a[sp].z; g.w += a[sp].w;
+        u.x += b[sp].x; u.y += b[sp].y; u.z += b[sp].z; u.w += b[sp].w;
     }
     float gv[4] = {g.x, g.y, g.z, g.w}, uv[4] = {u.x, u.y, u.z, u.w}, z[4];
     float sq = 0.f;
