@@ -401,8 +401,11 @@ griffin_status launch_decode(const griffin_ff_desc *desc, int B, const griffin_f
     p.B = B;
     if (desc->dtype == GRIFFIN_DT_F32) return decode_simt<float>(p, desc->act, flags, stream);
     // one expert set for several sequences (Eq. 7): only the tcgen05 kernel streams it once for all of them
-    if (decode_tc_shared(p)) return decode_bf16_tc(p, desc->act, flags, stream);
-    if ((flags & GRIFFIN_DECODE_TCGEN05) && decode_tc_supported(p)) return decode_bf16_tc(p, desc->act, flags, stream);
+    // (a shape that its plan cannot place in shared memory or TMEM after all goes to the warp-level kernel)
+    if (decode_tc_shared(p) || ((flags & GRIFFIN_DECODE_TCGEN05) && decode_tc_supported(p))) {
+        const griffin_status st = decode_bf16_tc(p, desc->act, flags, stream);
+        if (st != GRIFFIN_ERR_UNSUPPORTED) return st;
+    }
     return decode_bf16_mma(p, desc->act, flags, stream);
 }
 
