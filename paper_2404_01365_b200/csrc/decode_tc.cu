@@ -52,7 +52,7 @@ constexpr int DTC_SLOT_BYTES = 32 * 1024;  // one stage of the ring
 constexpr int DTC_MAX_STAGES = 7;
 constexpr int DTC_MAX_SETS = 16;           // sets per work item (128 rows of 8)
 constexpr int DTC_TMEM_COLS = 512;         // 32 accumulators of 16 columns
-constexpr int DTC_STAGING_DEPTH = 12;      // 16-byte loads that a thread keeps in flight while it stages a vector
+constexpr int DTC_STAGING_DEPTH_SHARED = 32;  // 16-byte loads a thread keeps in flight while it stages the up to 8 vectors that share a set
 constexpr int DTC_MAX_VEC = 8;             // vectors that may share one expert set in a call
 #ifndef GRIFFIN_DTC_SET_ROWS_0
 #define GRIFFIN_DTC_SET_ROWS_0 16
@@ -446,12 +446,12 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     const size_t src_stride = half ? (size_t)2 * p.ldk * 2 : (size_t)p.d * 2;  // bytes between sequences
                     const uint8_t *src0 = half ? reinterpret_cast<const uint8_t *>(zbits) : static_cast<const uint8_t *>(p.x);
                     const int total = n_vec * n_units;
-                    for (int e0 = et; e0 < total; e0 += DTC_STAGING_DEPTH * DTC_EPI_THREADS) {
-                        uint4 t[DTC_STAGING_DEPTH];
+                    for (int e0 = et; e0 < total; e0 += DTC_STAGING_DEPTH_SHARED * DTC_EPI_THREADS) {
+                        uint4 t[DTC_STAGING_DEPTH_SHARED];
                         int v = e0 / n_units, u = e0 - v * n_units;  // (vector, unit) of this thread's first load of the round
                         const int v0 = v, u0 = u;
 #pragma unroll
-                        for (int j = 0; j < DTC_STAGING_DEPTH; ++j) {  // all loads of a round are in flight together
+                        for (int j = 0; j < DTC_STAGING_DEPTH_SHARED; ++j) {  // all loads of a round are in flight together
                             t[j] = e0 + j * DTC_EPI_THREADS < total
                                        ? __ldcg(reinterpret_cast<const uint4 *>(src0 + (size_t)v * src_stride) + u)
                                        : make_uint4(0, 0, 0, 0);
@@ -459,7 +459,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                         }
                         v = v0, u = u0;
 #pragma unroll
-                        for (int j = 0; j < DTC_STAGING_DEPTH; ++j) {
+                        for (int j = 0; j < DTC_STAGING_DEPTH_SHARED; ++j) {
                             if (e0 + j * DTC_EPI_THREADS < total) reinterpret_cast<uint4 *>(s.vec + (size_t)v * pl.vec_stride)[u] = t[j];
                             for (u += DTC_EPI_THREADS; u >= n_units; u -= n_units) ++v;
                         }
@@ -516,15 +516,16 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     stop = true;
                     break;
                 }
-                // thread t finishes row r0 + t of the item, for every vector
-                if (et < R) {
-                    const int row = r0 + et;
-                    const int ig = (et / h.set_rows) * 16 + et % h.set_rows;  // where the (gate) row's result is
-                    for (int v = 0; v < n_vec; ++v) {
+                // the (vector, row) results of the item are shared out among the threads
+                for (int task = et; task < n_vec * R; task += DTC_EPI_THREADS) {
+                    const int v = task / R, rr = task - v * R;
+                    const int row = r0 + rr;
+                    const int ig = (rr / h.set_rows) * 16 + rr % h.set_rows;  // where the (gate) row's result is
+                    {
                         const int seq = n_vec > 1 ? v : b;
                         const float *part = s.part + v * (DTC_MAX_SETS * 16);
                         if (!half) {
-                            const int iu = R + et;  // the up row's place in the item
+                            const int iu = R + rr;  // the up row's place in the item
                             float a0 = part[ig];
                             float a1 = part[(iu / h.set_rows) * 16 + iu % h.set_rows];
                             if (p.seq[b].b_gate) a0 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[b].b_gate)[row]);
