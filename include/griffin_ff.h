@@ -98,6 +98,18 @@ typedef struct {
     int32_t ldk;                  /* leading dimension of w_down_c, >= k, multiple of 8 */
 } griffin_ff_compact;
 
+/* Full weights of one FF block in neuron-major form: neuron j owns row j of all three
+ * matrices, so w_down_t is the TRANSPOSE of W_2 (made once, when the model is loaded).  Used
+ * by griffin_ff_decode_indexed.  Biases may be NULL (= absent). */
+typedef struct {
+    const void *w_gate;           /* [d_ff, d]  W_g                                     */
+    const void *w_up;             /* [d_ff, d]  W_1                                     */
+    const void *w_down_t;         /* [d_ff, d]  W_2 transposed                          */
+    const void *b_gate;           /* [d_ff] or NULL                                     */
+    const void *b_up;             /* [d_ff] or NULL                                     */
+    const void *b_down;           /* [d]    or NULL                                     */
+} griffin_ff_weights_nm;
+
 /* Flags of griffin_ff_decode. */
 #define GRIFFIN_DECODE_DEFAULT 0u
 /* Launch the decode kernels with programmatic dependent launch: each kernel may begin
@@ -183,6 +195,26 @@ griffin_status griffin_ff_decode(const griffin_ff_desc *desc, int32_t B,
                                  const griffin_ff_compact *sets /*host*/, const void *b_down,
                                  const void *x, void *y, void *workspace, size_t ws_bytes,
                                  uint32_t flags, void *stream);
+
+/* Generation phase (Eqs. 4, 5) without a compact copy: the pruned block
+ *   y[b] = W_2[:, E_b] (sigma(W_g[E_b, :] x[b] + b_g[E_b]) * (W_1[E_b, :] x[b] + b_1[E_b])) + b_2
+ * is evaluated by reading the rows idx[b, 0..k) of the neuron-major full weights in place, so
+ * griffin_compact_experts and its k x d copies per sequence are not needed.  The result is
+ * that of griffin_ff_decode on the compact set of the same indices, up to rounding (z stays
+ * in fp32 here).  bf16 storage only (GRIFFIN_ERR_UNSUPPORTED otherwise), d <= GRIFFIN_MAX_D,
+ * 1 <= B <= GRIFFIN_MAX_BATCH, 1 <= k <= d_ff.
+ * idx [B, k] int32 on the DEVICE; the order of a sequence's indices does not matter and
+ * sequences may share or differ in their lists.  An entry outside [0, d_ff) is not
+ * dereferenced: that neuron contributes nothing and the device status word is raised.
+ * x [B, d] in, y [B, d] out.  The workspace holds one fp32 partial y per SM and sequence
+ * (griffin_workspace_bytes covers it).  flags: GRIFFIN_DECODE_DEFAULT or
+ * GRIFFIN_DECODE_OVERLAP_WEIGHT_PREFETCH (the promise then covers idx as well as the
+ * weights).  One kernel whose CTAs (one per SM) meet at the end through a counter in the
+ * workspace header: run it on a GPU whose SMs it can all occupy. */
+griffin_status griffin_ff_decode_indexed(const griffin_ff_desc *desc, int32_t B,
+                                         const griffin_ff_weights_nm *w, const int32_t *idx, int32_t k,
+                                         const void *x, void *y, void *workspace, size_t ws_bytes,
+                                         uint32_t flags, void *stream);
 
 /* The paper has no counterpart to this call: it is griffin_ff_decode for callers that have
  * no device memory to give as a workspace and may not allocate any.  That is the situation

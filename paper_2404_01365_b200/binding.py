@@ -27,7 +27,7 @@ EXPORTS = (
     "griffin_status_string", "griffin_version", "griffin_k_from_keep_ratio", "griffin_compact_ldk",
     "griffin_workspace_bytes", "griffin_workspace_init", "griffin_ff_prefill_score", "griffin_select_topk",
     "griffin_combine_scores", "griffin_compact_experts", "griffin_ff_decode", "griffin_check_device_status",
-    "griffin_ff_decode_static",
+    "griffin_ff_decode_static", "griffin_ff_decode_indexed",
 )
 
 
@@ -43,6 +43,10 @@ class FFDesc(C.Structure):
 
 class FFWeights(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("w_gate", "w_up", "w_down", "b_gate", "b_up", "b_down")]
+
+
+class FFWeightsNM(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("w_gate", "w_up", "w_down_t", "b_gate", "b_up", "b_down")]
 
 
 class FFCompact(C.Structure):
@@ -86,6 +90,8 @@ def load(path=None):
     lib.griffin_compact_experts.argtypes = [C.POINTER(FFDesc), C.POINTER(FFWeights), vp, C.POINTER(FFCompact), vp, vp]
     lib.griffin_ff_decode.restype = C.c_int
     lib.griffin_ff_decode.argtypes = [C.POINTER(FFDesc), i32, C.POINTER(FFCompact), vp, vp, vp, vp, sz, u32, vp]
+    lib.griffin_ff_decode_indexed.restype = C.c_int
+    lib.griffin_ff_decode_indexed.argtypes = [C.POINTER(FFDesc), i32, C.POINTER(FFWeightsNM), vp, i32, vp, vp, vp, sz, u32, vp]
     lib.griffin_ff_decode_static.restype = C.c_int
     lib.griffin_ff_decode_static.argtypes = [C.POINTER(FFDesc), i32, C.POINTER(FFCompact), vp, vp, vp, u32, vp]
     lib.griffin_check_device_status.restype = C.c_int
@@ -134,6 +140,13 @@ def make_desc(d, d_ff, act, dtype):
 def make_weights(w_gate, w_up, w_down, b_gate=None, b_up=None, b_down=None):
     w = FFWeights(_ptr(w_gate), _ptr(w_up), _ptr(w_down), _ptr(b_gate), _ptr(b_up), _ptr(b_down))
     w._keep = (w_gate, w_up, w_down, b_gate, b_up, b_down)  # keep the tensors alive
+    return w
+
+
+def make_weights_nm(w_gate, w_up, w_down_t, b_gate=None, b_up=None, b_down=None):
+    """Neuron-major full weights for griffin_ff_decode_indexed: w_down_t is W_2 transposed, [d_ff, d]."""
+    w = FFWeightsNM(_ptr(w_gate), _ptr(w_up), _ptr(w_down_t), _ptr(b_gate), _ptr(b_up), _ptr(b_down))
+    w._keep = (w_gate, w_up, w_down_t, b_gate, b_up, b_down)
     return w
 
 
@@ -209,6 +222,14 @@ def griffin_ff_decode(desc, sets, b_down, x, y, ws, flags=DECODE_DEFAULT, stream
     arr = sets if isinstance(sets, C.Array) else compact_array(sets)
     _check(load().griffin_ff_decode(C.byref(desc), len(arr), arr, _ptr(b_down), _ptr(x), _ptr(y), _ptr(ws),
                                     ws.numel(), int(flags), _stream(stream)), "griffin_ff_decode")
+
+
+def griffin_ff_decode_indexed(desc, weights_nm, idx, x, y, ws, flags=DECODE_DEFAULT, stream=None):
+    """Pruned FF straight from the full neuron-major weights; idx [B, k] int32 on the device."""
+    B, k = (1, idx.shape[0]) if idx.dim() == 1 else idx.shape
+    _check(load().griffin_ff_decode_indexed(C.byref(desc), int(B), C.byref(weights_nm), _ptr(idx), int(k), _ptr(x),
+                                            _ptr(y), _ptr(ws), ws.numel(), int(flags), _stream(stream)),
+           "griffin_ff_decode_indexed")
 
 
 STATIC_SCRATCH_BYTES = 1 << 20

@@ -96,6 +96,10 @@ size_t griffin_workspace_bytes(const griffin_ff_desc *desc, int32_t S_max, int32
     if (S_max > 0) need = prefill_scratch(desc, S_max).total;
     const size_t dec = decode_scratch_bytes(desc, n_seq_max);
     if (dec > need) need = dec;
+    if (desc->dtype == GRIFFIN_DT_BF16 && desc->d <= GRIFFIN_MAX_D) {
+        const size_t di = decode_indexed_scratch_bytes(desc->d, n_seq_max);
+        if (di > need) need = di;
+    }
     return WS_HEADER_BYTES + need;
 }
 
@@ -185,6 +189,26 @@ griffin_status griffin_ff_decode(const griffin_ff_desc *desc, int32_t B, const g
     if (ws_bytes < WS_HEADER_BYTES + (size_t)B * sets[0].ldk * sizeof(float)) return GRIFFIN_ERR_WORKSPACE;
     float *z = reinterpret_cast<float *>(static_cast<uint8_t *>(workspace) + WS_HEADER_BYTES);
     return launch_decode(desc, B, sets, b_down, x, y, z, workspace, flags, static_cast<cudaStream_t>(stream));
+}
+
+griffin_status griffin_ff_decode_indexed(const griffin_ff_desc *desc, int32_t B, const griffin_ff_weights_nm *w,
+                                         const int32_t *idx, int32_t k, const void *x, void *y, void *workspace,
+                                         size_t ws_bytes, uint32_t flags, void *stream) {
+    griffin_status st = check_desc(desc);
+    if (st != GRIFFIN_OK) return st;
+    if (w == nullptr || idx == nullptr || x == nullptr || y == nullptr) return GRIFFIN_ERR_INVALID_ARG;
+    if (w->w_gate == nullptr || w->w_up == nullptr || w->w_down_t == nullptr) return GRIFFIN_ERR_INVALID_ARG;
+    if (B < 1 || k < 1 || k > desc->d_ff) return GRIFFIN_ERR_INVALID_ARG;
+    if (flags & ~GRIFFIN_DECODE_OVERLAP_WEIGHT_PREFETCH) return GRIFFIN_ERR_INVALID_ARG;
+    if (desc->dtype != GRIFFIN_DT_BF16 || B > GRIFFIN_MAX_BATCH || desc->d > GRIFFIN_MAX_D) return GRIFFIN_ERR_UNSUPPORTED;
+    if (!aligned16(w->w_gate) || !aligned16(w->w_up) || !aligned16(w->w_down_t) || !aligned16(x) || !aligned16(y) ||
+        (reinterpret_cast<uintptr_t>(idx) & 3u) != 0)
+        return GRIFFIN_ERR_ALIGNMENT;
+    if (workspace == nullptr) return GRIFFIN_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return GRIFFIN_ERR_ALIGNMENT;
+    if (ws_bytes < WS_HEADER_BYTES + decode_indexed_scratch_bytes(desc->d, B)) return GRIFFIN_ERR_WORKSPACE;
+    float *ypart = reinterpret_cast<float *>(static_cast<uint8_t *>(workspace) + WS_HEADER_BYTES);
+    return launch_decode_indexed(desc, B, w, idx, k, x, y, ypart, workspace, flags, static_cast<cudaStream_t>(stream));
 }
 
 griffin_status griffin_ff_decode_static(const griffin_ff_desc *desc, int32_t B, const griffin_ff_compact *sets,

@@ -24,6 +24,7 @@ struct WsHeader {
     int detail;           // where it happened (kernel-specific code)
     unsigned int meet_warp;  // meeting-point counter of the warp-level fused decode kernel (see grid_meet)
     unsigned int meet_tc;    // ... and of the tcgen05 one (the two have different numbers of parties)
+    unsigned int meet_idx;   // ... and of the index-direct one
 };
 
 __device__ __forceinline__ void raise_status(void *ws, int status, int detail) {

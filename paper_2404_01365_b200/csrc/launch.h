@@ -23,6 +23,13 @@ griffin_status launch_decode(const griffin_ff_desc *desc, int B, const griffin_f
 griffin_status launch_decode_static(const griffin_ff_desc *desc, int B, const griffin_ff_compact *sets,
                                     const void *b_down, const void *x, void *y, uint32_t flags, cudaStream_t stream);
 
+// Index-direct decode (decode_indexed.cu): expert rows read in place from neuron-major weights.
+constexpr int IDX_MAX_GRID = 148;  // CTAs (= partial-sum rows per sequence in the workspace) at most
+size_t decode_indexed_scratch_bytes(int d, int n_seq);
+griffin_status launch_decode_indexed(const griffin_ff_desc *desc, int B, const griffin_ff_weights_nm *w,
+                                     const int32_t *idx, int k, const void *x, void *y, float *ypart, void *ws,
+                                     uint32_t flags, cudaStream_t stream);
+
 griffin_status launch_select_topk(const float *score, int n_seq, int d_ff, int k, int32_t *idx, cudaStream_t stream);
 
 griffin_status launch_combine_scores(const float *score, const int32_t *prompt_len_host, int n_seq, int d_ff,

@@ -89,5 +89,16 @@ class GpuLayer:
         G.griffin_ff_decode(self.desc, sets, self.t["bd"], x, y, self.ws, flags)
         return y
 
+    def decode_indexed(self, idx, x, flags=0):
+        """Pruned FF straight from the full weights (W_2 transposed once, as at model load)."""
+        if not hasattr(self, "weights_nm"):
+            self.t["wd_t"] = self.t["wd"].t().contiguous()
+            self.weights_nm = G.make_weights_nm(self.t["wg"], self.t["wu"], self.t["wd_t"], self.t["bg"], self.t["bu"],
+                                                self.t["bd"])
+        x = x.to(dev()).contiguous()
+        y = torch.empty_like(x)
+        G.griffin_ff_decode_indexed(self.desc, self.weights_nm, idx, x, y, self.ws, flags)
+        return y
+
     def status(self):
         return G.griffin_check_device_status(self.ws)

@@ -93,6 +93,24 @@ def test_host_validation_rejects_before_any_launch(lib):
     assert dcd(C.byref(desc), 2, mixed, None, fake, fake, fake, 1 << 30, 0, None) == G.ERR_INVALID_ARG
     wide = G.make_desc(8200, 688, "swiglu", "f32")
     assert dcd(C.byref(wide), 1, sets, None, fake, fake, fake, 1 << 30, 0, None) == G.ERR_UNSUPPORTED
+    # decode through the index list
+    dix = lib.griffin_ff_decode_indexed
+    bdesc = G.make_desc(256, 688, "swiglu", "bf16")
+    wn = G.FFWeightsNM(fake, fake, fake, None, None, None)
+    big = 1 << 30
+    assert dix(C.byref(bdesc), 1, None, fake, 344, fake, fake, fake, big, 0, None) == G.ERR_INVALID_ARG
+    assert dix(C.byref(bdesc), 1, C.byref(wn), None, 344, fake, fake, fake, big, 0, None) == G.ERR_INVALID_ARG
+    assert dix(C.byref(bdesc), 1, C.byref(wn), fake, 0, fake, fake, fake, big, 0, None) == G.ERR_INVALID_ARG
+    assert dix(C.byref(bdesc), 1, C.byref(wn), fake, 689, fake, fake, fake, big, 0, None) == G.ERR_INVALID_ARG
+    assert dix(C.byref(bdesc), 1, C.byref(wn), fake, 344, fake, fake, fake, big, 2, None) == G.ERR_INVALID_ARG
+    assert dix(C.byref(desc), 1, C.byref(wn), fake, 344, fake, fake, fake, big, 0, None) == G.ERR_UNSUPPORTED  # fp32
+    assert dix(C.byref(bdesc), 33, C.byref(wn), fake, 344, fake, fake, fake, big, 0, None) == G.ERR_UNSUPPORTED
+    assert dix(C.byref(bdesc), 1, C.byref(wn), fake, 344, odd, fake, fake, big, 0, None) == G.ERR_ALIGNMENT
+    assert dix(C.byref(bdesc), 1, C.byref(wn), fake, 344, fake, fake, None, 0, 0, None) == G.ERR_WORKSPACE
+    assert dix(C.byref(bdesc), 2, C.byref(wn), fake, 344, fake, fake, fake,
+               G.griffin_workspace_bytes(bdesc, 0, 1), 0, None) == G.ERR_WORKSPACE   # sized for one sequence
+    no_down = G.FFWeightsNM(fake, fake, None, None, None, None)
+    assert dix(C.byref(bdesc), 1, C.byref(no_down), fake, 344, fake, fake, fake, big, 0, None) == G.ERR_INVALID_ARG
     # combine
     cmb = lib.griffin_combine_scores
     lens = (C.c_int32 * 2)(4, 0)

@@ -207,6 +207,71 @@ def test_decode_with_one_shared_set_matches_oracle_and_separate_calls(d, d_ff, k
         assert rel_l2(np64(y[b]), np64(y1[0])) < TOL_OUT["bf16"], b
 
 
+# Decode straight from the full weights through the index list: d, d_ff, k, B, activation, biases
+INDEXED_SHAPES = [
+    (256, 688, 344, 1, "swiglu", True),        # the tiny workload's shape
+    (64, 96, 37, 3, "reglu", True),            # fewer experts than CTAs: most slices are empty
+    (1000, 1504, 751, 2, "geglu_erf", True),   # rows that end inside a block of 32 units
+    (2048, 5632, 2816, 1, "swiglu", False),
+    (256, 20000, 16400, 2, "geglu_tanh", False),   # two work items per CTA and sequence
+    (4096, 11008, 5504, 1, "swiglu", False),   # Llama-2-7B shape
+    (4096, 11008, 5504, 4, "swiglu", False),   # the final sum takes four columns per lane
+    (5120, 2048, 1024, 8, "swiglu", True),     # one pair per stage, batch 8
+    (8192, 1024, 512, 2, "swiglu", False),     # largest supported d
+    (512, 1536, 1536, 2, "geglu_tanh", True),  # every neuron, in a shuffled order
+]
+
+
+@pytest.mark.parametrize("d,d_ff,k,B,act,bias", INDEXED_SHAPES)
+def test_decode_indexed_matches_oracle_and_compact_path(d, d_ff, k, B, act, bias):
+    L, host = make_layer(d, d_ff, "bf16", act=act, bias=bias, seed=5 * d + k, n_seq=B)
+    rs = np.random.default_rng(d + k + B)
+    x = rand((B, d), torch.bfloat16, 96)
+    idx = np.empty((B, k), dtype=np.int32)
+    refs = []
+    for b in range(B):
+        e_np = rs.choice(d_ff, size=k, replace=False).astype(np.int32)
+        idx[b] = e_np if b % 2 else np.sort(e_np)       # the order of the list must not matter
+        c = O.compact_experts(idx[b], h64(host, "wg"), h64(host, "wu"), h64(host, "wd"), h64(host, "bg"), h64(host, "bu"))
+        refs.append(O.ff_pruned(np64(x[b]), c, act, h64(host, "bd")))
+    e = torch.from_numpy(idx).to(dev())
+    y = L.decode_indexed(e, x)
+    y2 = L.decode_indexed(e, x, G.DECODE_OVERLAP_WEIGHT_PREFETCH)
+    y3 = L.decode_indexed(e, x, G.DECODE_OVERLAP_WEIGHT_PREFETCH)
+    assert L.status() == G.OK
+    assert torch.equal(y, y2) and torch.equal(y, y3)    # deterministic, launch mode does not matter
+    for b in range(B):
+        assert rel_l2(np64(y[b]), refs[b]) < TOL_OUT["bf16"], b
+    if B <= 2:   # the compact-set kernels on the same indices
+        y_c = L.decode([L.compact(e[b]) for b in range(B)], x)
+        assert rel_l2(np64(y), np64(y_c)) < TOL_OUT["bf16"]
+
+
+def test_decode_indexed_out_of_range_index_is_reported_not_read():
+    d, d_ff = 256, 688
+    L, host = make_layer(d, d_ff, "bf16", seed=77)
+    good = np.arange(0, 600, 2, dtype=np.int32)
+    bad = good.copy()
+    bad[7], bad[100] = d_ff, -3
+    x = rand((1, d), torch.bfloat16, 95)
+    y = L.decode_indexed(torch.from_numpy(bad).to(dev()), x)
+    assert L.status() == G.ERR_INVALID_ARG
+    G.griffin_workspace_init(L.ws)
+    # the two bad entries contribute nothing: the result is that of the list without them
+    keep = np.delete(good, [7, 100])
+    c = O.compact_experts(keep, h64(host, "wg"), h64(host, "wu"), h64(host, "wd"))
+    assert rel_l2(np64(y[0]), O.ff_pruned(np64(x[0]), c, "swiglu")) < TOL_OUT["bf16"]
+    assert L.status() == G.OK
+
+
+def test_decode_indexed_rejects_fp32_storage():
+    L, _ = make_layer(64, 96, "f32")
+    e = torch.arange(8, dtype=torch.int32, device=dev())
+    with pytest.raises(G.GriffinError) as err:
+        L.decode_indexed(e, rand((1, 64), torch.float32, 1))
+    assert err.value.status == G.ERR_UNSUPPORTED
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_decode_with_all_neurons_is_the_dense_ff(dtype):
     d, d_ff = 512, 1536
