@@ -20,9 +20,10 @@
 //                u = t, t + 128, ...: no reduction across lanes is needed, so plain FMAs on
 //                the unpacked bf16 pairs are far below the issue limit.
 // After every item the two groups' shares of y are added through shared memory and join the
-// CTA's partial y of that sequence in the workspace; after the last item all CTAs meet (bounded wait) and each
-// sums a share of the columns over all CTAs' partials in a fixed order, adds b_2 and writes
-// bf16.  Results are bitwise reproducible.
+// CTA's partial y of that sequence in the workspace.  After its last item a CTA reports in; the
+// last few to do so wait (bounded) for the rest and sum the columns over all CTAs' partials in
+// a fixed order, add b_2 and write bf16, while the others have already left their SMs to the
+// next kernel on the stream.  Results are bitwise reproducible.
 #include "decode_mma.cuh"
 
 namespace griffin {
@@ -39,6 +40,7 @@ struct IndexedParams {
     int n_slices;   // work items per sequence (a multiple of the grid)
     int n_stages;   // ring slots (even: one half per consumer group)
     int red_vec;    // columns per lane in the final reduction: 1 or 4
+    int n_red;      // CTAs that share the final reduction (the last ones to finish their items)
 };
 
 struct IdxSmem {
@@ -339,17 +341,45 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) decode_indexed_kernel(const __
         }
     }
 
-    // ---- every CTA's partial sums are written: meet, then add them up column by column
+    // ---- this CTA's partial sums are written.  The CTAs report in on a counter that runs round
+    //      modulo 2 n and is never reset (as at the meeting point of the compact-set kernel); the
+    //      order of arrival decides who adds the partial sums up: the last n_red CTAs to arrive
+    //      wait (bounded) until everybody has reported and take the column blocks between them,
+    //      the earlier ones are done and leave their SM to the next kernel on the stream.
     consumer_barrier();
-    if (tid == 0) grid_meet(&static_cast<WsHeader *>(ws)->meet_idx, gridDim.x, s.abort, ws);
+    volatile int *role = reinterpret_cast<volatile int *>(s.zs);  // (z is not needed any more)
+    const int n_red = p.n_red;
+    if (tid == 0) {
+        unsigned int *counter = &static_cast<WsHeader *>(ws)->meet_idx;
+        const unsigned int n = gridDim.x;
+        __threadfence();
+        const unsigned int old = atomicInc(counter, 2 * n - 1);
+        const bool upper = old >= n;
+        int mine = (int)(upper ? old - n : old) - ((int)n - n_red);  // >= 0: this CTA's first column block
+        if (mine >= 0) {
+            const long long t0 = clock64();
+            for (;;) {
+                const unsigned int v = ld_acquire_u32(counter);
+                if (upper ? v < n : v >= n) break;
+                if (*s.abort || clock64() - t0 > WAIT_LIMIT_CYCLES) {
+                    *s.abort = 1;
+                    raise_status(ws, DEV_STATUS_TIMEOUT, 25);
+                    mine = -1;
+                    break;
+                }
+            }
+        }
+        *role = mine;
+    }
     consumer_barrier();
-    if (*s.abort) return;
+    const int first_blk = *role;
+    if (first_blk < 0) return;
     const int V = p.red_vec;            // columns per lane: 1 or 4
     const int total = B * d;            // columns of all sequences
     const int blk_cols = 32 * V;
     const int n_blocks = (total + blk_cols - 1) / blk_cols;
     const int grid = (int)gridDim.x;
-    for (int blk = blockIdx.x; blk < n_blocks; blk += grid) {
+    for (int blk = first_blk; blk < n_blocks; blk += n_red) {
         const int col = blk * blk_cols + lane * V;  // V divides d: the lane's columns lie in one sequence
         float4 acc4 = make_float4(0.f, 0.f, 0.f, 0.f);
         if (col < total) {
@@ -429,7 +459,11 @@ griffin_status launch_decode_indexed(const griffin_ff_desc *desc, int B, const g
     p.n_stages = (n > 8 ? 8 : n) & ~1;
     if (p.n_stages < 2) return GRIFFIN_ERR_UNSUPPORTED;
     const long long total = (long long)B * p.d;
-    p.red_vec = total >= 4ll * 32 * grid ? 4 : 1;
+    p.red_vec = total > 32ll * grid ? 4 : 1;  // narrow column blocks while every CTA gets at most one of them
+    {
+        const long long n_blocks = (total + 32 * p.red_vec - 1) / (32 * p.red_vec);
+        p.n_red = n_blocks < grid ? (int)n_blocks : grid;
+    }
     const int wpg = DEC_GROUP_WARPS / pl.R;
     const int nu = (pl.row_units + 127) / 128;
     const void *fn = nullptr;
