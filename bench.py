@@ -43,6 +43,8 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=None, help="override the number of blocks (smaller footprint)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch every decode call from the host instead of replaying a CUDA graph")
+    ap.add_argument("--decode", default="compact", choices=["compact", "indexed"],
+                    help="indexed: no compaction step, the decode calls read the expert rows in place from the full weights")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
 
@@ -216,7 +218,8 @@ def run_ours(args, w, keep):
     L = args.layers or w.L
     B, T, S = w.B, w.T, w.S
     k = G.griffin_k_from_keep_ratio(w.d_ff, keep)
-    stack = FFStack(w.d, w.d_ff, w.act, w.dtype, L, B, S, k, dev)
+    indexed = args.decode == "indexed"
+    stack = FFStack(w.d, w.d_ff, w.act, w.dtype, L, B, S, k, dev, indexed=indexed)
     for l in range(L):
         stack.add_block(*synth.make_weights(w, l, device=dev))
     seq0 = rank * B  # every rank has its own sequences
@@ -237,7 +240,7 @@ def run_ours(args, w, keep):
         if record: ev[1].record(stream)
         stack.select_all()
         if record: ev[2].record(stream)
-        for l in range(L):
+        for l in range(0 if indexed else L):
             for q in range(B):
                 stack.compact(l, q)
         if record: ev[3].record(stream)
@@ -250,8 +253,12 @@ def run_ours(args, w, keep):
     def decode_loop():
         for t in range(T):
             for l in range(L):
-                # the very first decode calls follow the compaction kernels: launch them fully ordered
-                stack.decode(l, XD[t, l], YD[t, l], overlap=t > 0)
+                # the very first decode calls follow the kernels that write what they read (the compact
+                # sets, or the index lists): launch them fully ordered
+                if indexed:
+                    stack.decode_indexed(l, XD[t, l], YD[t, l], overlap=t > 0)
+                else:
+                    stack.decode(l, XD[t, l], YD[t, l], overlap=t > 0)
 
     # The T x L decode calls of a step always touch the same buffers: after the first warm-up step
     # they are captured once, through the same public API calls, into a CUDA graph that the
@@ -358,7 +365,8 @@ def run_ours(args, w, keep):
         g1_tiles = ((S + 127) // 128) * (w.d_ff // 128)
         cut = (w.dtype == "bf16" and w.d % 128 == 0 and w.d_ff % 128 == 0 and 148 < g1_tiles <= 4 * 148
                and 0 < g1_tiles % 148 <= 74 and w.d // 64 >= 16)
-        launches = L * B * (5 + (1 if split else 0) + (1 if cut else 0)) + 1 + L * B * 2 + T * L * (1 if w.dtype == "bf16" else 2)
+        launches = (L * B * (5 + (1 if split else 0) + (1 if cut else 0)) + 1 + (0 if indexed else L * B * 2) +
+                    T * L * (1 if w.dtype == "bf16" else 2))
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -368,6 +376,8 @@ def run_ours(args, w, keep):
                        "parallelism": f"{world} independent replica(s), no collective",
                        "l2": f"inputs larger than L2: {L} blocks of weights ({L * 3 * w.d * w.d_ff * w.elem_bytes / 1e9:.1f} GB dense, "
                              f"{L * B * 3 * k * w.d * w.elem_bytes / 1e9:.1f} GB compact) are visited in turn",
+                       "decode": ("index-direct: no compaction step, expert rows read in place from neuron-major full weights"
+                                  if indexed else "compact expert sets"),
                        "decode_launch": ("the T x L decode calls of a step, captured once from the public API calls, are replayed as a CUDA graph"
                                          if dec_graph[0] is not None else "one host launch per decode call")},
             "phases": {
@@ -375,15 +385,17 @@ def run_ours(args, w, keep):
                                   "frac_of_bf16_burst": stack.prefill_flops(S) / (pf_ms * 1e-3) / 1e12 / tensor_peaks[0],
                                   "frac_of_bf16_sustained": stack.prefill_flops(S) / (pf_ms * 1e-3) / 1e12 / tensor_peaks[1]},
                 "select_topk": {"ms_all_blocks": phase_ms[1] / K},
-                "compact": {"ms_per_block": phase_ms[2] / K / (L * B),
-                            "gbs": stack.compact_bytes() / (phase_ms[2] / K / (L * B) * 1e-3) / 1e9},
+                "compact": (None if indexed else
+                            {"ms_per_block": phase_ms[2] / K / (L * B),
+                             "gbs": stack.compact_bytes() / (phase_ms[2] / K / (L * B) * 1e-3) / 1e9}),
                 "decode": {"us_per_call": dec_ms_per_call * 1e3, "tokens_per_s_per_layer": B / (dec_ms_per_call * 1e-3),
                            "gbs": achieved},
             },
-            "roofline": {"bound": "hbm", "kernel": "decode_fused_kernel (one launch per decode call)", "achieved": achieved,
+            "roofline": {"bound": "hbm", "kernel": ("decode_indexed_kernel" if indexed else "decode_fused_kernel") +
+                         " (one launch per decode call)", "achieved": achieved,
                          "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
                          "algorithmic_bytes_per_launch": dec_bytes,
-                         "traffic": traffic["dram_bytes_per_decode_call"] if traffic else None},
+                         "traffic": traffic["dram_bytes_per_decode_call"] if traffic and not indexed else None},
             "clocks": clocks,
             "gpu_launches": launches,
             "host_issue_s": host_s,

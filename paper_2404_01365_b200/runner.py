@@ -8,7 +8,9 @@ library's CUDA kernels (binding.py).  One FFStack holds, for one process / one G
     weight set, all allocated once.
 The phases mirror the GRIFFIN algorithm (Section 4.2 of the paper): prompt phase with the
 full FF and the statistic, top-k selection, slicing of the weights, then the generation
-phase on the compact weights.
+phase on the compact weights.  With indexed=True the slicing is left out: the generation phase
+reads the expert rows in place from neuron-major full weights (W_2 is transposed once, when a
+block is added), and no compact sets are allocated.
 """
 from __future__ import annotations
 
@@ -18,25 +20,29 @@ from . import binding as G
 
 
 class FFStack:
-    def __init__(self, d, d_ff, act, dtype, L, n_seq, S_max, k, device):
+    def __init__(self, d, d_ff, act, dtype, L, n_seq, S_max, k, device, indexed=False):
         self.d, self.d_ff, self.L, self.n_seq, self.S_max, self.k = d, d_ff, L, n_seq, S_max, k
         self.device = device
         self.tdtype = torch.float32 if dtype == "f32" else torch.bfloat16
         self.desc = G.make_desc(d, d_ff, act, dtype)
         self.ldk = G.griffin_compact_ldk(k)
         self.ws = G.alloc_workspace(self.desc, S_max, n_seq, device)
+        self.indexed = indexed
         self.weights = []      # per block: binding.FFWeights
+        self.weights_nm = []   # per block (indexed only): binding.FFWeightsNM
         self.score = torch.empty((L, n_seq, d_ff), device=device, dtype=torch.float32)
         self.idx = torch.empty((L, n_seq, k), device=device, dtype=torch.int32)
         self.sets = []         # per block: list of n_seq compact sets
         self.set_arrays = []   # per block: C array of the n_seq sets, ready for decode
-        for _ in range(L):
+        for _ in range(0 if indexed else L):
             sets = [G.alloc_compact(self.desc, k, device, self.tdtype) for _ in range(n_seq)]
             self.sets.append(sets)
             self.set_arrays.append(G.compact_array(sets))
 
     def add_block(self, w_gate, w_up, w_down):
         self.weights.append(G.make_weights(w_gate, w_up, w_down))
+        if self.indexed:  # a layout step at model-load time, not a step of the path
+            self.weights_nm.append(G.make_weights_nm(w_gate, w_up, w_down.t().contiguous()))
 
     # ---- prompt phase -------------------------------------------------------------------
     def prefill_score(self, layer, seq, x, y):
@@ -56,6 +62,11 @@ class FFStack:
         """Pruned FF for one token of each of the n_seq sequences: x, y are [n_seq, d]."""
         G.griffin_ff_decode(self.desc, self.set_arrays[layer], None, x, y, self.ws,
                             G.DECODE_OVERLAP_WEIGHT_PREFETCH if overlap else G.DECODE_DEFAULT)
+
+    def decode_indexed(self, layer, x, y, overlap):
+        """The same without compact sets: the rows idx[layer] are read from the full weights."""
+        G.griffin_ff_decode_indexed(self.desc, self.weights_nm[layer], self.idx[layer], x, y, self.ws,
+                                    G.DECODE_OVERLAP_WEIGHT_PREFETCH if overlap else G.DECODE_DEFAULT)
 
     def status(self):
         return G.griffin_check_device_status(self.ws)

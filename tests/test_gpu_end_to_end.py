@@ -25,7 +25,8 @@ def run_block(w, layer, keep, n_seq, oracle_seqs, steps):
     assert k == O.k_from_keep_ratio(w.d_ff, keep)
     wg, wu, wd = synth.make_weights(w, layer)
     stack = FFStack(w.d, w.d_ff, w.act, w.dtype, 1, n_seq, w.S, k, dev())
-    stack.add_block(wg.to(dev()), wu.to(dev()), wd.to(dev()))
+    wg_d, wu_d, wd_d = wg.to(dev()), wu.to(dev()), wd.to(dev())
+    stack.add_block(wg_d, wu_d, wd_d)
     X = [synth.make_prompt(w, layer, q) for q in range(n_seq)]
     XD = torch.stack([synth.make_decode_inputs(w, layer, q) for q in range(n_seq)], 1)  # [T, n_seq, d]
     Y = torch.empty((n_seq, w.S, w.d), device=dev(), dtype=w.torch_dtype)
@@ -38,6 +39,13 @@ def run_block(w, layer, keep, n_seq, oracle_seqs, steps):
     yd = torch.empty_like(xd_dev)
     for t in range(w.T):
         stack.decode(0, xd_dev[t], yd[t], overlap=t > 0)
+    yd_ix = None
+    if w.dtype == "bf16":   # the same steps without the compact sets: rows read in place through the index lists
+        wn = G.make_weights_nm(wg_d, wu_d, wd_d.t().contiguous())
+        yd_ix = torch.empty_like(xd_dev)
+        for t in range(w.T):
+            G.griffin_ff_decode_indexed(stack.desc, wn, stack.idx[0], xd_dev[t], yd_ix[t], stack.ws,
+                                        G.DECODE_OVERLAP_WEIGHT_PREFETCH if t > 0 else G.DECODE_DEFAULT)
     assert stack.status() == G.OK
     E = stack.idx[0].cpu().numpy()
     S_gpu = np64(stack.score[0])
@@ -58,6 +66,8 @@ def run_block(w, layer, keep, n_seq, oracle_seqs, steps):
         for t in steps:
             ref = O.ff_pruned(np64(XD[t, q]), c, w.act)
             assert rel_l2(np64(yd[t, q]), ref) < TOL_OUT[w.dtype], ("decode", q, t)
+            if yd_ix is not None:
+                assert rel_l2(np64(yd_ix[t, q]), ref) < TOL_OUT[w.dtype], ("index-direct decode", q, t)
     if n_seq > 1 and k < w.d_ff:   # each sequence picked its own experts
         assert any(not np.array_equal(E[0], E[q]) for q in range(1, n_seq))
     return swaps
@@ -84,6 +94,32 @@ def test_small_versions_of_every_workload(name):
     for keep in base.keeps:
         for layer in (0, base.L - 1):
             run_block(w, layer, keep, base.B, range(base.B), range(w.T))
+
+
+def test_stack_without_compact_sets():
+    """The runner's index-direct mode: prompt phase, top-k, then decode straight from the full weights."""
+    base = synth.WORKLOADS["llama2_7b"]
+    w = synth.scaled(base, **SMALL["llama2_7b"])
+    k = G.griffin_k_from_keep_ratio(w.d_ff, 0.5)
+    wg, wu, wd = synth.make_weights(w, 0)
+    stack = FFStack(w.d, w.d_ff, w.act, w.dtype, 1, 2, w.S, k, dev(), indexed=True)
+    stack.add_block(wg.to(dev()), wu.to(dev()), wd.to(dev()))
+    assert stack.sets == []
+    X = [synth.make_prompt(w, 0, q) for q in range(2)]
+    XD = torch.stack([synth.make_decode_inputs(w, 0, q) for q in range(2)], 1).to(dev())
+    Y = torch.empty((2, w.S, w.d), device=dev(), dtype=w.torch_dtype)
+    for q in range(2):
+        stack.prefill_score(0, q, X[q].to(dev()), Y[q])
+    stack.select_all()
+    yd = torch.empty_like(XD)
+    for t in range(w.T):
+        stack.decode_indexed(0, XD[t], yd[t], overlap=t > 0)
+    assert stack.status() == G.OK
+    E = stack.idx[0].cpu().numpy()
+    for q in range(2):
+        c = O.compact_experts(E[q], np64(wg), np64(wu), np64(wd))
+        for t in range(w.T):
+            assert rel_l2(np64(yd[t, q]), O.ff_pruned(np64(XD[t, q]), c, w.act)) < TOL_OUT[w.dtype], (q, t)
 
 
 def _steps(T):
@@ -123,7 +159,8 @@ def test_shared_expert_set_for_a_batch():
     n_seq, k = len(lengths), G.griffin_k_from_keep_ratio(w.d_ff, 0.5)
     wg, wu, wd = synth.make_weights(w, 0)
     stack = FFStack(w.d, w.d_ff, w.act, w.dtype, 1, n_seq, max(lengths), k, dev())
-    stack.add_block(wg.to(dev()), wu.to(dev()), wd.to(dev()))
+    wg_d, wu_d, wd_d = wg.to(dev()), wu.to(dev()), wd.to(dev())
+    stack.add_block(wg_d, wu_d, wd_d)
     wg64, wu64, wd64 = np64(wg), np64(wu), np64(wd)
     s_ref = []
     for q, S in enumerate(lengths):
