@@ -158,6 +158,19 @@ griffin_status griffin_ff_prefill_score(const griffin_ff_desc *desc, const griff
                                         const void *x, int32_t S, void *y, float *score,
                                         void *workspace, size_t ws_bytes, void *stream);
 
+/* The prompt phase for a prompt that is fed piece by piece (long prompts: the workspace only
+ * has to hold the activations of one piece).  Each call is griffin_ff_prefill_score on the S
+ * tokens of one piece -- y[S, d] = FF(X) for them -- but the statistic is carried across the
+ * calls: s_j^2 is a sum over the tokens of the prompt (Eq. 6: every token normalises its own
+ * activation row, nothing couples two tokens), so
+ *   sumsq[d_ff] (fp32, in/out) = (first ? 0 : sumsq) + sum over this piece's tokens of Zbar_ij^2,
+ *   score[d_ff] (fp32, out, may be NULL) = sqrt(sumsq): after the last piece this is s of the
+ *   whole prompt, equal to that of one call up to the order of the fp32 additions.
+ * The pieces may have any lengths >= 1.  Calls on one prompt must be ordered on one stream. */
+griffin_status griffin_ff_prefill_score_chunk(const griffin_ff_desc *desc, const griffin_ff_weights *w,
+                                              const void *x, int32_t S, void *y, float *sumsq, float *score,
+                                              int32_t first, void *workspace, size_t ws_bytes, void *stream);
+
 /* Expert selection (Section 4.2): for each of n_seq score vectors, the indices of its k
  * largest entries, written in ascending index order; equal scores go to the lower index.
  * score [n_seq, d_ff] fp32 in, idx [n_seq, k] int32 out.  Scores must not be NaN. */

@@ -27,7 +27,7 @@ EXPORTS = (
     "griffin_status_string", "griffin_version", "griffin_k_from_keep_ratio", "griffin_compact_ldk",
     "griffin_workspace_bytes", "griffin_workspace_init", "griffin_ff_prefill_score", "griffin_select_topk",
     "griffin_combine_scores", "griffin_compact_experts", "griffin_ff_decode", "griffin_check_device_status",
-    "griffin_ff_decode_static", "griffin_ff_decode_indexed",
+    "griffin_ff_decode_static", "griffin_ff_decode_indexed", "griffin_ff_prefill_score_chunk",
 )
 
 
@@ -82,6 +82,9 @@ def load(path=None):
     lib.griffin_workspace_init.argtypes = [vp, sz, vp]
     lib.griffin_ff_prefill_score.restype = C.c_int
     lib.griffin_ff_prefill_score.argtypes = [C.POINTER(FFDesc), C.POINTER(FFWeights), vp, i32, vp, vp, vp, sz, vp]
+    lib.griffin_ff_prefill_score_chunk.restype = C.c_int
+    lib.griffin_ff_prefill_score_chunk.argtypes = [C.POINTER(FFDesc), C.POINTER(FFWeights), vp, i32, vp, vp, vp, i32, vp,
+                                                   sz, vp]
     lib.griffin_select_topk.restype = C.c_int
     lib.griffin_select_topk.argtypes = [vp, i32, i32, i32, vp, vp]
     lib.griffin_combine_scores.restype = C.c_int
@@ -189,6 +192,14 @@ def griffin_ff_prefill_score(desc, weights, x, y, score, ws, stream=None):
     S = x.shape[0]
     _check(load().griffin_ff_prefill_score(C.byref(desc), C.byref(weights), _ptr(x), S, _ptr(y), _ptr(score),
                                            _ptr(ws), ws.numel(), _stream(stream)), "griffin_ff_prefill_score")
+
+
+def griffin_ff_prefill_score_chunk(desc, weights, x, y, sumsq, score, first, ws, stream=None):
+    """One piece of a prompt that is fed piece by piece: sumsq carries the statistic's squares."""
+    S = x.shape[0]
+    _check(load().griffin_ff_prefill_score_chunk(C.byref(desc), C.byref(weights), _ptr(x), S, _ptr(y), _ptr(sumsq),
+                                                 _ptr(score), 1 if first else 0, _ptr(ws), ws.numel(), _stream(stream)),
+           "griffin_ff_prefill_score_chunk")
 
 
 def griffin_select_topk(score, k, idx, stream=None):

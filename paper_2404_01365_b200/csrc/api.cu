@@ -126,8 +126,29 @@ griffin_status griffin_ff_prefill_score(const griffin_ff_desc *desc, const griff
     if (!aligned16(workspace)) return GRIFFIN_ERR_ALIGNMENT;
     const PrefillScratch ps = prefill_scratch(desc, S);
     if (ws_bytes < WS_HEADER_BYTES + ps.total) return GRIFFIN_ERR_WORKSPACE;
-    return launch_prefill_score(desc, w, x, S, y, score, static_cast<uint8_t *>(workspace) + WS_HEADER_BYTES,
-                                workspace, static_cast<cudaStream_t>(stream));
+    return launch_prefill_score(desc, w, x, S, y, score, nullptr, 1,
+                                static_cast<uint8_t *>(workspace) + WS_HEADER_BYTES, workspace,
+                                static_cast<cudaStream_t>(stream));
+}
+
+griffin_status griffin_ff_prefill_score_chunk(const griffin_ff_desc *desc, const griffin_ff_weights *w, const void *x,
+                                              int32_t S, void *y, float *sumsq, float *score, int32_t first,
+                                              void *workspace, size_t ws_bytes, void *stream) {
+    griffin_status st = check_desc(desc);
+    if (st != GRIFFIN_OK) return st;
+    if (w == nullptr || w->w_gate == nullptr || w->w_up == nullptr || x == nullptr || sumsq == nullptr || S < 1)
+        return GRIFFIN_ERR_INVALID_ARG;
+    if (y != nullptr && w->w_down == nullptr) return GRIFFIN_ERR_INVALID_ARG;
+    if (!aligned16(w->w_gate) || !aligned16(w->w_up) || !aligned16(w->w_down) || !aligned16(x) || !aligned16(y) ||
+        !aligned16(sumsq) || !aligned16(score))
+        return GRIFFIN_ERR_ALIGNMENT;
+    if (workspace == nullptr) return GRIFFIN_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return GRIFFIN_ERR_ALIGNMENT;
+    const PrefillScratch ps = prefill_scratch(desc, S);
+    if (ws_bytes < WS_HEADER_BYTES + ps.total) return GRIFFIN_ERR_WORKSPACE;
+    return launch_prefill_score(desc, w, x, S, y, score, sumsq, first != 0,
+                                static_cast<uint8_t *>(workspace) + WS_HEADER_BYTES, workspace,
+                                static_cast<cudaStream_t>(stream));
 }
 
 griffin_status griffin_select_topk(const float *score, int32_t n_seq, int32_t d_ff, int32_t k, int32_t *idx,

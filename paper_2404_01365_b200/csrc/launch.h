@@ -46,7 +46,10 @@ struct PrefillScratch {
 };
 PrefillScratch prefill_scratch(const griffin_ff_desc *desc, int S);
 
+// sumsq (may be NULL): running sum of squares of the statistic over the pieces of a prompt; `first`
+// starts it afresh.  score may be NULL when sumsq is given.
 griffin_status launch_prefill_score(const griffin_ff_desc *desc, const griffin_ff_weights *w, const void *x, int S,
-                                    void *y, float *score, uint8_t *scratch, void *ws, cudaStream_t stream);
+                                    void *y, float *score, float *sumsq, int first, uint8_t *scratch, void *ws,
+                                    cudaStream_t stream);
 
 }  // namespace griffin

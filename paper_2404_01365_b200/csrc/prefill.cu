@@ -229,13 +229,19 @@ __global__ void __launch_bounds__(256) col_partial_kernel(const float *__restric
 }
 
 // Step 5.
+// sumsq (may be NULL): running sum of squares over the pieces of a prompt that is fed piece by
+// piece (s_j^2 is a sum over tokens, Eq. 6); `first` starts it afresh.  score may then be NULL.
 __global__ void score_finish_kernel(const float *__restrict__ colpart, int n_row_chunks, int d_ff,
-                                    float *__restrict__ score) {
+                                    float *__restrict__ score, float *__restrict__ sumsq, int first) {
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= d_ff) return;
     float acc = 0.f;
     for (int c = 0; c < n_row_chunks; ++c) acc += colpart[(size_t)c * d_ff + j];
-    score[j] = sqrtf(acc);
+    if (sumsq != nullptr) {
+        if (!first) acc += sumsq[j];
+        sumsq[j] = acc;
+    }
+    if (score != nullptr) score[j] = sqrtf(acc);
 }
 
 // The statistic only needs Z, the down projection only Z as well: with the tensor-core path the
@@ -265,7 +271,8 @@ static SideLane *side_lane_of_current_device() {
 
 template <typename T>
 static griffin_status prefill_typed(const griffin_ff_desc *desc, const griffin_ff_weights *w, const void *x, int S,
-                                    void *y, float *score, uint8_t *scratch, void *ws, cudaStream_t stream) {
+                                    void *y, float *score, float *sumsq, int first, uint8_t *scratch, void *ws,
+                                    cudaStream_t stream) {
     const int d = desc->d, d_ff = desc->d_ff;
     const PrefillScratch ps = prefill_scratch(desc, S);
     T *z = reinterpret_cast<T *>(scratch + ps.z_off);
@@ -315,7 +322,8 @@ static griffin_status prefill_typed(const griffin_ff_desc *desc, const griffin_f
     const dim3 g4((d_ff + 127) / 128, ps.n_row_chunks);
     col_partial_kernel<<<g4, 256, 0, stat_stream>>>(z32, inv, S, d_ff, colpart);
     if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
-    score_finish_kernel<<<(d_ff + 255) / 256, 256, 0, stat_stream>>>(colpart, ps.n_row_chunks, d_ff, score);
+    score_finish_kernel<<<(d_ff + 255) / 256, 256, 0, stat_stream>>>(colpart, ps.n_row_chunks, d_ff, score, sumsq,
+                                                                             first);
     if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
     if (lane != nullptr &&
         (cudaEventRecord(lane->join, lane->stream) != cudaSuccess || cudaStreamWaitEvent(stream, lane->join, 0) != cudaSuccess))
@@ -324,10 +332,11 @@ static griffin_status prefill_typed(const griffin_ff_desc *desc, const griffin_f
 }
 
 griffin_status launch_prefill_score(const griffin_ff_desc *desc, const griffin_ff_weights *w, const void *x, int S,
-                                    void *y, float *score, uint8_t *scratch, void *ws, cudaStream_t stream) {
+                                    void *y, float *score, float *sumsq, int first, uint8_t *scratch, void *ws,
+                                    cudaStream_t stream) {
     if (desc->dtype == GRIFFIN_DT_F32)
-        return prefill_typed<float>(desc, w, x, S, y, score, scratch, ws, stream);
-    return prefill_typed<__nv_bfloat16>(desc, w, x, S, y, score, scratch, ws, stream);
+        return prefill_typed<float>(desc, w, x, S, y, score, sumsq, first, scratch, ws, stream);
+    return prefill_typed<__nv_bfloat16>(desc, w, x, S, y, score, sumsq, first, scratch, ws, stream);
 }
 
 }  // namespace griffin

@@ -66,6 +66,12 @@ def test_host_validation_rejects_before_any_launch(lib):
     assert f(C.byref(bad), C.byref(w), fake, 4, fake, fake, fake, 1 << 30, None) == G.ERR_UNSUPPORTED
     bad = G.make_desc(250, 688, "swiglu", "f32")
     assert f(C.byref(bad), C.byref(w), fake, 4, fake, fake, fake, 1 << 30, None) == G.ERR_ALIGNMENT
+    # prompt phase, piece by piece
+    fc = lib.griffin_ff_prefill_score_chunk
+    assert fc(C.byref(desc), C.byref(w), fake, 4, fake, None, fake, 1, fake, 1 << 30, None) == G.ERR_INVALID_ARG
+    assert fc(C.byref(desc), C.byref(w), fake, 0, fake, fake, None, 1, fake, 1 << 30, None) == G.ERR_INVALID_ARG
+    assert fc(C.byref(desc), C.byref(w), fake, 4, fake, odd, None, 1, fake, 1 << 30, None) == G.ERR_ALIGNMENT
+    assert fc(C.byref(desc), C.byref(w), fake, 4, fake, fake, None, 0, fake, 1000, None) == G.ERR_WORKSPACE
     # top-k
     t = lib.griffin_select_topk
     assert t(fake, 1, 688, 0, fake, None) == G.ERR_INVALID_ARG

@@ -357,6 +357,37 @@ def test_prefill_score_matches_oracle(dtype, act, S, d, d_ff):
     assert np.array_equal(np64(s2), s)                   # deterministic; y is optional
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("pieces,d,d_ff", [((100, 37, 119), 512, 1032), ((1, 1, 62), 256, 688), ((300,), 1024, 2816),
+                                           ((128, 128, 128, 128, 50), 1024, 2816)])
+def test_prefill_fed_piece_by_piece_gives_the_statistic_of_the_whole_prompt(dtype, pieces, d, d_ff):
+    """s_j^2 is a sum over tokens (Eq. 6): the pieces' sums of squares add up to the whole prompt's."""
+    S = sum(pieces)
+    L, host = make_layer(d, d_ff, dtype, act="swiglu", bias=(d == 512), seed=S + d, S_max=S)
+    x = rand((S, d), TD[dtype], 25) + rand((1, d), TD[dtype], 26, 4.0 / d ** 0.5)
+    xd = x.to(dev())
+    y = torch.empty((S, d), device=dev(), dtype=TD[dtype])
+    sumsq = torch.full((d_ff,), float("nan"), device=dev())        # the first piece must not read it
+    score = torch.empty((d_ff,), device=dev())
+    at = 0
+    for i, n in enumerate(pieces):
+        last = i == len(pieces) - 1
+        G.griffin_ff_prefill_score_chunk(L.desc, L.weights, xd[at:at + n], y[at:at + n], sumsq, score if last else None,
+                                         i == 0, L.ws)
+        at += n
+    assert L.status() == G.OK
+    ref_y, ref_z = O.ff_dense(np64(x), h64(host, "wg"), h64(host, "wu"), h64(host, "wd"), "swiglu",
+                              h64(host, "bg"), h64(host, "bu"), h64(host, "bd"))
+    ref_s = O.flock_score(ref_z)
+    assert rel_l2(np64(y), ref_y) < TOL_OUT[dtype]
+    s = np64(score)
+    assert np.all(np.abs(s - ref_s) <= score_tol(dtype) * ref_s + 1e-6 * np.sqrt(S / d_ff))
+    assert abs(float(np.sum(s * s)) - S) < 1e-5 * S
+    assert np.allclose(np64(sumsq), s * s, rtol=1e-6, atol=0)
+    _, s_whole = L.prefill(x)                                       # one call on the whole prompt
+    assert np.allclose(np64(s_whole), s, rtol=2 * score_tol(dtype), atol=1e-6 * np.sqrt(S / d_ff))
+
+
 @pytest.mark.parametrize("S,d,d_ff", [(256, 1024, 10240), (200, 2048, 9728)])
 def test_prefill_with_a_cut_last_round_of_tiles(S, d, d_ff):
     """160 (152) tiles of the first GEMM on 148 SMs: the last 12 (4) are cut along K into parts
