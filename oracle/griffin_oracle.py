@@ -16,7 +16,10 @@ activations", s [d_ff] the selection statistic, E the expert set, k = |E|.
 
 Pinning status (see tests/test_oracle_pins.py):
   * ff1_activations, ff_dense     pinned (brute force, identity weights,
-                                  closed-form sigma values)
+                                  closed-form sigma values; the blocks
+                                  without a gate: brute force, identity
+                                  weights, the gated form with a constant
+                                  second branch)
   * flock_score                   pinned (sum_j s_j^2 = S, S = 1, rank one,
                                   row-rescale invariance, permutation
                                   equivariance, brute force)
@@ -41,6 +44,12 @@ GEGLU_TANH = "geglu_tanh"
 REGLU = "reglu"
 GEGLU_ERF = "geglu_erf"
 ACTIVATIONS = (SWIGLU, GEGLU_TANH, REGLU, GEGLU_ERF)
+# FF blocks without a gate (Eq. 2, e.g. OPT): the name of the block -> the sigma it uses
+RELU = "relu"
+GELU_TANH = "gelu_tanh"
+GELU_ERF = "gelu_erf"
+SILU = "silu"
+NON_GATED = {RELU: REGLU, GELU_TANH: GEGLU_TANH, GELU_ERF: GEGLU_ERF, SILU: SWIGLU}
 
 _erf = np.vectorize(math.erf, otypes=[np.float64])
 
@@ -77,14 +86,21 @@ def ff1_activations(x, w_gate, w_up, act, b_gate=None, b_up=None):
 
     x is [S, d] (or [d] for one token); the result is [S, d_ff] (or [d_ff]).
     sigma acts on the gate branch only.
+
+    For a block without a gate (act in NON_GATED; Eq. 2) there is no W_g:
+    Z = sigma(X W_1^T + b_1); w_gate and b_gate must be None.
     """
-    x, w_gate, w_up = _f64(x), _f64(w_gate), _f64(w_up)
-    g = x @ w_gate.T
+    x, w_up = _f64(x), _f64(w_up)
     u = x @ w_up.T
-    if b_gate is not None:
-        g = g + _f64(b_gate)
     if b_up is not None:
         u = u + _f64(b_up)
+    if act in NON_GATED:
+        if w_gate is not None or b_gate is not None:
+            raise ValueError("a block without a gate has no W_g, b_g")
+        return sigma(u, NON_GATED[act])
+    g = x @ _f64(w_gate).T
+    if b_gate is not None:
+        g = g + _f64(b_gate)
     return sigma(g, act) * u
 
 
@@ -158,7 +174,7 @@ def compact_experts(e, w_gate, w_up, w_down, b_gate=None, b_up=None):
     """
     e = np.asarray(e, dtype=np.int64)
     return {
-        "w_gate": np.asarray(w_gate)[e, :],
+        "w_gate": None if w_gate is None else np.asarray(w_gate)[e, :],
         "w_up": np.asarray(w_up)[e, :],
         "w_down": np.asarray(w_down)[:, e],
         "b_gate": None if b_gate is None else np.asarray(b_gate)[e],

@@ -123,6 +123,62 @@ def test_sigma_is_on_the_gate_branch_only():
     assert not np.allclose(z, z_swapped)
 
 
+# ------------------------------------------- blocks without a gate (Eq. 2) ---
+
+@pytest.mark.parametrize("act", list(O.NON_GATED))
+@pytest.mark.parametrize("bias", [False, True])
+def test_non_gated_ff_brute_force(act, bias):
+    f = {"relu": lambda t: max(t, 0.0), "gelu_tanh": _gelu_tanh, "silu": _silu,
+         "gelu_erf": lambda t: 0.5 * t * math.erfc(-t / math.sqrt(2.0))}[act]
+    r = rng(21)
+    S, d, n = 4, 5, 7
+    x, w1, w2 = r.normal(size=(S, d)), r.normal(size=(n, d)), r.normal(size=(d, n))
+    b1, b2 = (r.normal(size=n), r.normal(size=d)) if bias else (None, None)
+    y, z = O.ff_dense(x, None, w1, w2, act, None, b1, b2)
+    for i in range(S):
+        zi = [f(sum(w1[j][c] * x[i][c] for c in range(d)) + (b1[j] if bias else 0.0)) for j in range(n)]
+        assert z[i] == pytest.approx(np.array(zi), rel=1e-12, abs=1e-13)
+        yi = [sum(w2[c][j] * zi[j] for j in range(n)) + (b2[c] if bias else 0.0) for c in range(d)]
+        assert y[i] == pytest.approx(np.array(yi), rel=1e-12, abs=1e-13)
+
+
+def test_non_gated_ff_special_cases():
+    r = rng(22)
+    x = r.normal(size=(3, 6))
+    eye = np.eye(6)
+    # W_1 = W_2 = I: Y = relu(X), and nothing is multiplied back in (unlike the gated form)
+    y, z = O.ff_dense(x, None, eye, eye, O.RELU)
+    assert np.array_equal(y, np.maximum(x, 0.0)) and np.array_equal(z, y)
+    # sigma(u) = sigma(u) * 1: the gated block whose second branch is the constant 1 is the same map
+    w1, b1 = r.normal(size=(8, 6)), r.normal(size=8)
+    gated = O.ff1_activations(x, w1, np.zeros((8, 6)), O.GEGLU_TANH, b1, np.ones(8))
+    assert O.ff1_activations(x, None, w1, O.GELU_TANH, None, b1) == pytest.approx(gated, abs=1e-15)
+    # a gate matrix has no place in such a block
+    with pytest.raises(ValueError):
+        O.ff1_activations(x, w1, w1, O.RELU)
+    # ReLU zeroes whole neurons: one that never fires has statistic 0 and is the first to be pruned
+    w1, b1 = r.normal(size=(6, 6)), np.zeros(6)
+    b1[2] = -1e3
+    z = O.ff1_activations(x, None, w1, O.RELU, None, b1)
+    s = O.flock_score(z)
+    assert np.all(z[:, 2] == 0.0) and s[2] == 0.0 and 2 not in O.select_topk(s, 5)
+
+
+def test_non_gated_pruned_ff_is_the_dense_one_with_the_other_neurons_zeroed():
+    r = rng(23)
+    x, w1, w2 = r.normal(size=(4, 6)), r.normal(size=(10, 6)), r.normal(size=(6, 10))
+    b1, b2 = r.normal(size=10), r.normal(size=6)
+    e = np.array([1, 4, 5, 9])
+    c = O.compact_experts(e, None, w1, w2, None, b1)
+    assert c["w_gate"] is None and c["b_gate"] is None
+    y_hat = O.ff_pruned(x, c, O.RELU, b2)
+    _, z = O.ff_dense(x, None, w1, w2, O.RELU, None, b1, b2)
+    mask = np.zeros(10); mask[e] = 1.0
+    assert y_hat == pytest.approx((z * mask) @ w2.T + b2, abs=1e-13)
+    full = O.compact_experts(np.arange(10), None, w1, w2, None, b1)
+    assert np.array_equal(O.ff_pruned(x, full, O.RELU, b2), O.ff_dense(x, None, w1, w2, O.RELU, None, b1, b2)[0])
+
+
 def test_ff_dense_single_token_matches_row_of_batch():
     # Section 3: the block acts independently on every row of X.
     r = rng(4)
