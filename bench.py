@@ -145,7 +145,7 @@ def oracle_sample(w, keep, layer, T_sample):
     import numpy as np
     from oracle import griffin_oracle as O
     from paper_2404_01365_b200 import synth
-    wg, wu, wd = (t.double().numpy() for t in synth.make_weights(w, layer))
+    wg, wu, wd = (None if t is None else t.double().numpy() for t in synth.make_weights(w, layer))
     x = synth.make_prompt(w, layer, 0).double().numpy()
     xd = synth.make_decode_inputs(w, layer, 0, T=T_sample).double().numpy()
     k = O.k_from_keep_ratio(w.d_ff, keep)
@@ -362,8 +362,9 @@ def run_ours(args, w, keep):
         # (two for fp32 storage)
         split = w.dtype == "bf16" and ((S + 127) // 128) * (w.d // 256 if w.d % 256 == 0 else w.d // 128) <= 74
         # ... and the finishing kernel of the first GEMM when its last round of 128x128 tiles is cut along K
-        g1_tiles = ((S + 127) // 128) * (w.d_ff // 128)
-        cut = (w.dtype == "bf16" and w.d % 128 == 0 and w.d_ff % 128 == 0 and 148 < g1_tiles <= 4 * 148
+        gated = G.act_is_gated(w.act)
+        g1_tiles = ((S + 127) // 128) * (w.d_ff // 128 if gated else w.d_ff // 256)
+        cut = (w.dtype == "bf16" and w.d % 128 == 0 and w.d_ff % (128 if gated else 256) == 0 and 148 < g1_tiles <= 4 * 148
                and 0 < g1_tiles % 148 <= 74 and w.d // 64 >= 16)
         launches = (L * B * (5 + (1 if split else 0) + (1 if cut else 0)) + 1 + (0 if indexed else L * B * 2) +
                     T * L * (1 if w.dtype == "bf16" else 2))

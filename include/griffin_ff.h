@@ -1,8 +1,8 @@
 /*
  * griffin_ff.h -- C ABI of libgriffin_ff.so
  *
- * GRIFFIN (arXiv 2404.01365) for one gated feed-forward (FF) block of a decoder layer,
- * as hand-written CUDA kernels for NVIDIA B200 (sm_100a).  Four steps:
+ * GRIFFIN (arXiv 2404.01365) for one feed-forward (FF) block of a decoder layer (gated, Eq. 3,
+ * or without a gate, Eq. 2), as hand-written CUDA kernels for NVIDIA B200 (sm_100a).  Four steps:
  *
  *   griffin_ff_prefill_score   prompt phase: full FF over the S prompt tokens and the
  *                              selection statistic s                       (Eqs. 1, 3, 6)
@@ -60,8 +60,17 @@ typedef enum {
     GRIFFIN_ACT_SWIGLU = 0,       /* sigma(t) = t / (1 + exp(-t))                                   */
     GRIFFIN_ACT_GEGLU_TANH = 1,   /* sigma(t) = t/2 (1 + tanh(sqrt(2/pi) (t + 0.044715 t^3)))       */
     GRIFFIN_ACT_REGLU = 2,        /* sigma(t) = max(t, 0)                                           */
-    GRIFFIN_ACT_GEGLU_ERF = 3     /* sigma(t) = t/2 (1 + erf(t / sqrt(2)))                          */
+    GRIFFIN_ACT_GEGLU_ERF = 3,    /* sigma(t) = t/2 (1 + erf(t / sqrt(2)))                          */
+    /* FF blocks WITHOUT a gate (Eq. 2, e.g. OPT): FF_1(x) = sigma(W_1 x + b_1).  There is no W_g:
+     * w_gate / b_gate (and w_gate_c / b_gate_c of a compact set) must be NULL, every other
+     * argument keeps its meaning, and each step moves two matrices instead of three. */
+    GRIFFIN_ACT_RELU = 4,         /* sigma = max(t, 0)                                              */
+    GRIFFIN_ACT_GELU_TANH = 5,    /* sigma = the tanh form of GEGLU_TANH                            */
+    GRIFFIN_ACT_GELU_ERF = 6,     /* sigma = the erf form of GEGLU_ERF                              */
+    GRIFFIN_ACT_SILU = 7          /* sigma = t / (1 + exp(-t))                                      */
 } griffin_act;
+/* Whether an activation code names a gated block (W_g present). */
+#define GRIFFIN_ACT_IS_GATED(act) ((act) >= GRIFFIN_ACT_SWIGLU && (act) <= GRIFFIN_ACT_GEGLU_ERF)
 
 typedef enum { GRIFFIN_DT_F32 = 0, GRIFFIN_DT_BF16 = 1 } griffin_dtype;
 
@@ -75,7 +84,7 @@ typedef struct {
 
 /* Full weights of one FF block (Eqs. 1 and 3).  Biases may be NULL (= absent). */
 typedef struct {
-    const void *w_gate;           /* [d_ff, d]  W_g                                     */
+    const void *w_gate;           /* [d_ff, d]  W_g (NULL for a block without a gate)   */
     const void *w_up;             /* [d_ff, d]  W_1                                     */
     const void *w_down;           /* [d, d_ff]  W_2                                     */
     const void *b_gate;           /* [d_ff] or NULL                                     */
@@ -89,7 +98,7 @@ typedef struct {
  * the full weights themselves are a valid compact set (k = ldk = d_ff), which is how the
  * unpruned FF is run through the same decode kernels. */
 typedef struct {
-    void *w_gate_c;               /* [k, d]                                             */
+    void *w_gate_c;               /* [k, d] (NULL for a block without a gate)           */
     void *w_up_c;                 /* [k, d]                                             */
     void *w_down_c;               /* [d, ldk]                                           */
     void *b_gate_c;               /* [k] or NULL                                        */
@@ -102,7 +111,7 @@ typedef struct {
  * matrices, so w_down_t is the TRANSPOSE of W_2 (made once, when the model is loaded).  Used
  * by griffin_ff_decode_indexed.  Biases may be NULL (= absent). */
 typedef struct {
-    const void *w_gate;           /* [d_ff, d]  W_g                                     */
+    const void *w_gate;           /* [d_ff, d]  W_g (NULL for a block without a gate)   */
     const void *w_up;             /* [d_ff, d]  W_1                                     */
     const void *w_down_t;         /* [d_ff, d]  W_2 transposed                          */
     const void *b_gate;           /* [d_ff] or NULL                                     */
@@ -149,7 +158,8 @@ griffin_status griffin_workspace_init(void *workspace, size_t ws_bytes, void *st
 
 /* Prompt phase (Section 4.2, "Prompt Phase Expert Neuron Selection").
  *   y[S, d]      = FF(X) = (sigma(X W_g^T + b_g) * (X W_1^T + b_1)) W_2^T + b_2   (Eqs. 1, 3)
- *                  -- the full block, never pruned, independent of k;
+ *                  -- the full block, never pruned, independent of k (without a gate, Eq. 2:
+ *                  FF(X) = sigma(X W_1^T + b_1) W_2^T + b_2);
  *   score[d_ff]  = s, s_j = || column j of Zbar ||_2, Zbar_i = Z_i / ||Z_i||_2   (Eq. 6);
  *                  a token whose activation row is all zero contributes nothing.
  * x [S, d] in, y [S, d] out (dtype of desc), score fp32 out.  1 <= S.  Z is held in the
@@ -195,7 +205,8 @@ griffin_status griffin_compact_experts(const griffin_ff_desc *desc, const griffi
                                        void *workspace /*may be NULL*/, void *stream);
 
 /* Generation phase (Eqs. 4, 5): for each of B sequences, with its own compact set,
- *   y[b] = W_2_hat (sigma(W_g_hat x[b] + b_g_hat) * (W_1_hat x[b] + b_1_hat)) + b_2.
+ *   y[b] = W_2_hat (sigma(W_g_hat x[b] + b_g_hat) * (W_1_hat x[b] + b_1_hat)) + b_2
+ * (without a gate: y[b] = W_2_hat sigma(W_1_hat x[b] + b_1_hat) + b_2).
  * sets: HOST array of B structs; every set must have the same k and ldk.  Entries may repeat
  * to share a set: when 2..8 sequences of a bf16 call all name the same buffers (one expert
  * set for the batch, Eq. 7) and d and ldk are multiples of 128, the weights are streamed

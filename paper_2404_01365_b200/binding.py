@@ -16,11 +16,18 @@ from . import build as _build
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(7)
 ACT_SWIGLU, ACT_GEGLU_TANH, ACT_REGLU, ACT_GEGLU_ERF = 0, 1, 2, 3
+ACT_RELU, ACT_GELU_TANH, ACT_GELU_ERF, ACT_SILU = 4, 5, 6, 7   # blocks without a gate (Eq. 2): w_gate is None
 DT_F32, DT_BF16 = 0, 1
 DECODE_DEFAULT, DECODE_OVERLAP_WEIGHT_PREFETCH, DECODE_TCGEN05 = 0, 1, 2
 MAX_BATCH = 32
 
-ACT_BY_NAME = {"swiglu": ACT_SWIGLU, "geglu_tanh": ACT_GEGLU_TANH, "reglu": ACT_REGLU, "geglu_erf": ACT_GEGLU_ERF}
+ACT_BY_NAME = {"swiglu": ACT_SWIGLU, "geglu_tanh": ACT_GEGLU_TANH, "reglu": ACT_REGLU, "geglu_erf": ACT_GEGLU_ERF,
+               "relu": ACT_RELU, "gelu_tanh": ACT_GELU_TANH, "gelu_erf": ACT_GELU_ERF, "silu": ACT_SILU}
+
+
+def act_is_gated(act):
+    act = ACT_BY_NAME[act] if isinstance(act, str) else int(act)
+    return ACT_SWIGLU <= act <= ACT_GEGLU_ERF
 DTYPE_BY_NAME = {"f32": DT_F32, "bf16": DT_BF16}
 
 EXPORTS = (
@@ -162,10 +169,11 @@ def make_compact(w_gate_c, w_up_c, w_down_c, k, ldk, b_gate_c=None, b_up_c=None)
 def alloc_compact(desc, k, device, torch_dtype, with_bias=False):
     """Allocates the buffers of one compact expert set (torch owns the memory)."""
     ldk = griffin_compact_ldk(k)
-    g = torch.empty((k, desc.d), device=device, dtype=torch_dtype)
+    gated = act_is_gated(desc.act)   # a block without a gate has no W_g_hat
+    g = torch.empty((k, desc.d), device=device, dtype=torch_dtype) if gated else None
     u = torch.empty((k, desc.d), device=device, dtype=torch_dtype)
     dn = torch.empty((desc.d, ldk), device=device, dtype=torch_dtype)
-    bg = torch.empty((k,), device=device, dtype=torch_dtype) if with_bias else None
+    bg = torch.empty((k,), device=device, dtype=torch_dtype) if with_bias and gated else None
     bu = torch.empty((k,), device=device, dtype=torch_dtype) if with_bias else None
     return make_compact(g, u, dn, k, ldk, bg, bu)
 

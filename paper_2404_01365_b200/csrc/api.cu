@@ -53,10 +53,13 @@ static griffin_status check_desc(const griffin_ff_desc *desc) {
     if (desc->d < 8 || desc->d_ff < 8) return GRIFFIN_ERR_INVALID_ARG;
     if (desc->d % 8 != 0 || desc->d_ff % 8 != 0) return GRIFFIN_ERR_ALIGNMENT;
     if (desc->dtype != GRIFFIN_DT_F32 && desc->dtype != GRIFFIN_DT_BF16) return GRIFFIN_ERR_UNSUPPORTED;
-    if (desc->act != GRIFFIN_ACT_SWIGLU && desc->act != GRIFFIN_ACT_GEGLU_TANH && desc->act != GRIFFIN_ACT_REGLU &&
-        desc->act != GRIFFIN_ACT_GEGLU_ERF)
-        return GRIFFIN_ERR_UNSUPPORTED;
+    if (desc->act < GRIFFIN_ACT_SWIGLU || desc->act > GRIFFIN_ACT_SILU) return GRIFFIN_ERR_UNSUPPORTED;
     return GRIFFIN_OK;
+}
+
+// A gated block (Eq. 3) needs W_g; a block without a gate (Eq. 2) must not name one.
+static bool gate_args_ok(const griffin_ff_desc *desc, const void *w_gate, const void *b_gate) {
+    return act_gated(desc->act) ? w_gate != nullptr : (w_gate == nullptr && b_gate == nullptr);
 }
 
 static size_t decode_scratch_bytes(const griffin_ff_desc *desc, int n_seq) {
@@ -116,8 +119,9 @@ griffin_status griffin_ff_prefill_score(const griffin_ff_desc *desc, const griff
                                         void *stream) {
     griffin_status st = check_desc(desc);
     if (st != GRIFFIN_OK) return st;
-    if (w == nullptr || w->w_gate == nullptr || w->w_up == nullptr || x == nullptr || score == nullptr || S < 1)
+    if (w == nullptr || w->w_up == nullptr || x == nullptr || score == nullptr || S < 1)
         return GRIFFIN_ERR_INVALID_ARG;
+    if (!gate_args_ok(desc, w->w_gate, w->b_gate)) return GRIFFIN_ERR_INVALID_ARG;
     if (y != nullptr && w->w_down == nullptr) return GRIFFIN_ERR_INVALID_ARG;
     if (!aligned16(w->w_gate) || !aligned16(w->w_up) || !aligned16(w->w_down) || !aligned16(x) || !aligned16(y) ||
         !aligned16(score))
@@ -136,8 +140,9 @@ griffin_status griffin_ff_prefill_score_chunk(const griffin_ff_desc *desc, const
                                               void *workspace, size_t ws_bytes, void *stream) {
     griffin_status st = check_desc(desc);
     if (st != GRIFFIN_OK) return st;
-    if (w == nullptr || w->w_gate == nullptr || w->w_up == nullptr || x == nullptr || sumsq == nullptr || S < 1)
+    if (w == nullptr || w->w_up == nullptr || x == nullptr || sumsq == nullptr || S < 1)
         return GRIFFIN_ERR_INVALID_ARG;
+    if (!gate_args_ok(desc, w->w_gate, w->b_gate)) return GRIFFIN_ERR_INVALID_ARG;
     if (y != nullptr && w->w_down == nullptr) return GRIFFIN_ERR_INVALID_ARG;
     if (!aligned16(w->w_gate) || !aligned16(w->w_up) || !aligned16(w->w_down) || !aligned16(x) || !aligned16(y) ||
         !aligned16(sumsq) || !aligned16(score))
@@ -169,7 +174,8 @@ griffin_status griffin_combine_scores(const float *score, const int32_t *prompt_
 }
 
 static griffin_status check_compact(const griffin_ff_desc *desc, const griffin_ff_compact *c) {
-    if (c->w_gate_c == nullptr || c->w_up_c == nullptr || c->w_down_c == nullptr) return GRIFFIN_ERR_INVALID_ARG;
+    if (c->w_up_c == nullptr || c->w_down_c == nullptr) return GRIFFIN_ERR_INVALID_ARG;
+    if (!gate_args_ok(desc, c->w_gate_c, c->b_gate_c)) return GRIFFIN_ERR_INVALID_ARG;
     if (c->k < 1 || c->k > desc->d_ff) return GRIFFIN_ERR_INVALID_ARG;
     if (c->ldk < c->k || c->ldk > desc->d_ff) return GRIFFIN_ERR_INVALID_ARG;
     if (c->ldk % 8 != 0) return GRIFFIN_ERR_ALIGNMENT;
@@ -182,7 +188,8 @@ griffin_status griffin_compact_experts(const griffin_ff_desc *desc, const griffi
     griffin_status st = check_desc(desc);
     if (st != GRIFFIN_OK) return st;
     if (w == nullptr || out == nullptr || idx == nullptr) return GRIFFIN_ERR_INVALID_ARG;
-    if (w->w_gate == nullptr || w->w_up == nullptr || w->w_down == nullptr) return GRIFFIN_ERR_INVALID_ARG;
+    if (w->w_up == nullptr || w->w_down == nullptr) return GRIFFIN_ERR_INVALID_ARG;
+    if (!gate_args_ok(desc, w->w_gate, w->b_gate)) return GRIFFIN_ERR_INVALID_ARG;
     if (!aligned16(w->w_gate) || !aligned16(w->w_up) || !aligned16(w->w_down)) return GRIFFIN_ERR_ALIGNMENT;
     st = check_compact(desc, out);
     if (st != GRIFFIN_OK) return st;
@@ -218,7 +225,8 @@ griffin_status griffin_ff_decode_indexed(const griffin_ff_desc *desc, int32_t B,
     griffin_status st = check_desc(desc);
     if (st != GRIFFIN_OK) return st;
     if (w == nullptr || idx == nullptr || x == nullptr || y == nullptr) return GRIFFIN_ERR_INVALID_ARG;
-    if (w->w_gate == nullptr || w->w_up == nullptr || w->w_down_t == nullptr) return GRIFFIN_ERR_INVALID_ARG;
+    if (w->w_up == nullptr || w->w_down_t == nullptr) return GRIFFIN_ERR_INVALID_ARG;
+    if (!gate_args_ok(desc, w->w_gate, w->b_gate)) return GRIFFIN_ERR_INVALID_ARG;
     if (B < 1 || k < 1 || k > desc->d_ff) return GRIFFIN_ERR_INVALID_ARG;
     if (flags & ~GRIFFIN_DECODE_OVERLAP_WEIGHT_PREFETCH) return GRIFFIN_ERR_INVALID_ARG;
     if (desc->dtype != GRIFFIN_DT_BF16 || B > GRIFFIN_MAX_BATCH || desc->d > GRIFFIN_MAX_D) return GRIFFIN_ERR_UNSUPPORTED;

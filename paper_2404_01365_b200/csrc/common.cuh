@@ -79,6 +79,20 @@ template <int ACT> __device__ __forceinline__ float sigma(float t) {
     }
 }
 
+// The sigma of an activation code, as the code of the gated form that uses the same function: the
+// kernels get this (0..3) as `act` plus, separately, whether the block has a gate (Eq. 3) or not
+// (Eq. 2).
+__host__ __device__ inline int act_sigma(int act) {
+    switch (act) {
+        case GRIFFIN_ACT_RELU: return GRIFFIN_ACT_REGLU;
+        case GRIFFIN_ACT_GELU_TANH: return GRIFFIN_ACT_GEGLU_TANH;
+        case GRIFFIN_ACT_GELU_ERF: return GRIFFIN_ACT_GEGLU_ERF;
+        case GRIFFIN_ACT_SILU: return GRIFFIN_ACT_SWIGLU;
+        default: return act;
+    }
+}
+__host__ __device__ inline bool act_gated(int act) { return GRIFFIN_ACT_IS_GATED(act); }
+
 __device__ __forceinline__ float sigma_rt(int act, float t) {
     switch (act) {
         case GRIFFIN_ACT_SWIGLU: return sigma<GRIFFIN_ACT_SWIGLU>(t);

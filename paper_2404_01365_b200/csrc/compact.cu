@@ -30,13 +30,14 @@ __device__ __forceinline__ void st_stream(uint4 *p, const uint4 &v) {
                  : "memory");
 }
 
-// dst_g[jj, :] = src_g[idx[jj], :], dst_u likewise; nv = 16-byte vectors per row.
+// dst_g[jj, :] = src_g[idx[jj], :], dst_u likewise; nv = 16-byte vectors per row.  n_mats = 1: only
+// the first pair of pointers is used (a block without a gate has W_1 alone).
 __global__ void __launch_bounds__(CP_THREADS) compact_rows_kernel(const uint4 *__restrict__ src_g,
                                                                   const uint4 *__restrict__ src_u,
                                                                   uint4 *__restrict__ dst_g, uint4 *__restrict__ dst_u,
                                                                   const int32_t *__restrict__ idx, int k, int d_ff,
-                                                                  int nv, void *ws) {
-    const long long total = 2ll * k * nv;
+                                                                  int nv, int n_mats, void *ws) {
+    const long long total = (long long)n_mats * k * nv;
     const long long stride = (long long)gridDim.x * CP_THREADS;
     constexpr int U = 4;
     for (long long v0 = (long long)blockIdx.x * CP_THREADS + threadIdx.x; v0 < total; v0 += stride * U) {
@@ -122,12 +123,14 @@ static griffin_status compact_typed(const griffin_ff_desc *desc, const griffin_f
     const int nv = d * (int)sizeof(U) / 16;
     const int sms = device_sm_count();
     if (sms <= 0) return GRIFFIN_ERR_CUDA;
-    const long long want = (2ll * k * nv + CP_THREADS * 4 - 1) / (CP_THREADS * 4);
+    const bool gated = w->w_gate != nullptr;  // (a block without a gate has W_1 alone, Eq. 2)
+    const long long want = ((gated ? 2ll : 1ll) * k * nv + CP_THREADS * 4 - 1) / (CP_THREADS * 4);
     int grid = (int)(want < (long long)sms * 8 ? want : (long long)sms * 8);
     if (grid < 1) grid = 1;
     compact_rows_kernel<<<grid, CP_THREADS, 0, stream>>>(
-        static_cast<const uint4 *>(w->w_gate), static_cast<const uint4 *>(w->w_up),
-        static_cast<uint4 *>(out->w_gate_c), static_cast<uint4 *>(out->w_up_c), idx, k, d_ff, nv, ws);
+        static_cast<const uint4 *>(gated ? w->w_gate : w->w_up), static_cast<const uint4 *>(w->w_up),
+        static_cast<uint4 *>(gated ? out->w_gate_c : out->w_up_c), static_cast<uint4 *>(out->w_up_c), idx, k, d_ff, nv,
+        gated ? 2 : 1, ws);
     if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
     compact_cols_kernel<U><<<(d + CP_ROWS_PER_CTA - 1) / CP_ROWS_PER_CTA, CP_THREADS, 0, stream>>>(
         static_cast<const U *>(w->w_down), static_cast<U *>(out->w_down_c), idx, d, d_ff, k, ldk, ws);

@@ -24,13 +24,15 @@ namespace griffin {
 // Kernel gate_up:
 //   z[b, j] = sigma(w_gate_c[j,:] . x[b] + b_gate_c[j]) * (w_up_c[j,:] . x[b] + b_up_c[j])
 // Work item = (sequence b, slice of neurons).  Stage = gate row j followed by up row j.
+// GATED = false (a block without a gate, Eq. 2): z[b, j] = sigma(w_up_c[j,:] . x[b] + b_up_c[j]),
+// stage = up row j alone.
 // ---------------------------------------------------------------------------------------
-template <typename T, int ITER>
+template <typename T, int ITER, bool GATED>
 __global__ void __launch_bounds__(DEC_THREADS) decode_gate_up_kernel(const __grid_constant__ DecodeParams p, int act) {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     constexpr int VEC = Elem<T>::VEC;
     const int row_bytes = p.d * (int)sizeof(T);
-    const int stage_bytes = 2 * row_bytes;
+    const int stage_bytes = (GATED ? 2 : 1) * row_bytes;
     const DecSmem s = carve(smem_raw, p.n_stages, stage_bytes);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -66,8 +68,8 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_gate_up_kernel(const __gri
                     }
                     uint8_t *dst = s.stages + (size_t)stage * stage_bytes;
                     mbar_arrive_expect_tx(&s.full[stage], stage_bytes);
-                    bulk_g2s(dst, g + (size_t)j * row_bytes, row_bytes, &s.full[stage]);
-                    bulk_g2s(dst + row_bytes, u + (size_t)j * row_bytes, row_bytes, &s.full[stage]);
+                    if (GATED) bulk_g2s(dst, g + (size_t)j * row_bytes, row_bytes, &s.full[stage]);
+                    bulk_g2s(dst + (GATED ? row_bytes : 0), u + (size_t)j * row_bytes, row_bytes, &s.full[stage]);
                 }
             }
             producer_drain(s, p.n_stages, it);
@@ -112,16 +114,16 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_gate_up_kernel(const __gri
                 const int col = (tid + i * DEC_CONSUMERS) * VEC;
                 if (col < p.d) {
                     float gf[VEC], uf[VEC];
-                    Elem<T>::unpack(*reinterpret_cast<const uint4 *>(src + (size_t)col * sizeof(T)), gf);
-                    Elem<T>::unpack(*reinterpret_cast<const uint4 *>(src + row_bytes + (size_t)col * sizeof(T)), uf);
+                    if (GATED) Elem<T>::unpack(*reinterpret_cast<const uint4 *>(src + (size_t)col * sizeof(T)), gf);
+                    Elem<T>::unpack(*reinterpret_cast<const uint4 *>(src + (GATED ? row_bytes : 0) + (size_t)col * sizeof(T)), uf);
 #pragma unroll
                     for (int e = 0; e < VEC; ++e) {
-                        ga = fmaf(gf[e], xr[i][e], ga);
+                        if (GATED) ga = fmaf(gf[e], xr[i][e], ga);
                         ua = fmaf(uf[e], xr[i][e], ua);
                     }
                 }
             }
-            ga = warp_sum(ga);
+            if (GATED) ga = warp_sum(ga);
             ua = warp_sum(ua);
             if (lane == 0) {
                 // every lane's shared-memory reads fed the shuffles above, so they are done
@@ -140,9 +142,9 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_gate_up_kernel(const __gri
                 ua += v.y;
             }
             const int j = j0 + tid;
-            if (p.seq[b].b_gate) ga += Elem<T>::to_float(static_cast<const T *>(p.seq[b].b_gate)[j]);
+            if (GATED && p.seq[b].b_gate) ga += Elem<T>::to_float(static_cast<const T *>(p.seq[b].b_gate)[j]);
             if (p.seq[b].b_up) ua += Elem<T>::to_float(static_cast<const T *>(p.seq[b].b_up)[j]);
-            p.z[(size_t)b * p.ldk + j] = sigma_rt(act, ga) * ua;
+            p.z[(size_t)b * p.ldk + j] = GATED ? sigma_rt(act, ga) * ua : sigma_rt(act, ua);
         }
         // the last slice also clears the padding of z (at most 7 entries)
         const int pad = tid - (DEC_CONSUMERS - 8);
@@ -331,8 +333,22 @@ int slices_for(int rows, int grid) {
     return grid * per;
 }
 
+template <typename T, bool GATED>
+static const void *gate_up_fn(int iter) {
+    switch (iter) {
+        case 1: return (const void *)decode_gate_up_kernel<T, 1, GATED>;
+        case 2: return (const void *)decode_gate_up_kernel<T, 2, GATED>;
+        case 3: return (const void *)decode_gate_up_kernel<T, 3, GATED>;
+        case 4: return (const void *)decode_gate_up_kernel<T, 4, GATED>;
+        case 5: case 6: return (const void *)decode_gate_up_kernel<T, 6, GATED>;
+        case 7: case 8: return (const void *)decode_gate_up_kernel<T, 8, GATED>;
+        default: return nullptr;
+    }
+}
+
+// act: the code of sigma (0..3); gated: whether the block has a gate (Eq. 3) or not (Eq. 2)
 template <typename T>
-static griffin_status decode_simt(DecodeParams &p, int act, uint32_t flags, cudaStream_t stream) {
+static griffin_status decode_simt(DecodeParams &p, int act, bool gated, uint32_t flags, cudaStream_t stream) {
     constexpr int VEC = Elem<T>::VEC;
     const int B = p.B;
     const int sms = device_sm_count();
@@ -340,22 +356,14 @@ static griffin_status decode_simt(DecodeParams &p, int act, uint32_t flags, cuda
     const bool overlap = (flags & GRIFFIN_DECODE_OVERLAP_WEIGHT_PREFETCH) != 0;
 
     {  // gate_up
-        const int stage_bytes = 2 * p.d * (int)sizeof(T);
+        const int stage_bytes = (gated ? 2 : 1) * p.d * (int)sizeof(T);
         p.n_stages = pick_stages(stage_bytes);
         p.n_slices = slices_for(p.k, sms);
         const int grid = min(sms, B * p.n_slices);
         const size_t smem = dec_smem_bytes(p.n_stages, stage_bytes);
         const int iter = (p.d + DEC_CONSUMERS * VEC - 1) / (DEC_CONSUMERS * VEC);
-        const void *fn = nullptr;
-        switch (iter) {
-            case 1: fn = (const void *)decode_gate_up_kernel<T, 1>; break;
-            case 2: fn = (const void *)decode_gate_up_kernel<T, 2>; break;
-            case 3: fn = (const void *)decode_gate_up_kernel<T, 3>; break;
-            case 4: fn = (const void *)decode_gate_up_kernel<T, 4>; break;
-            case 5: case 6: fn = (const void *)decode_gate_up_kernel<T, 6>; break;
-            case 7: case 8: fn = (const void *)decode_gate_up_kernel<T, 8>; break;
-            default: return GRIFFIN_ERR_UNSUPPORTED;
-        }
+        const void *fn = gated ? gate_up_fn<T, true>(iter) : gate_up_fn<T, false>(iter);
+        if (fn == nullptr) return GRIFFIN_ERR_UNSUPPORTED;
         if (ensure_dynamic_smem(fn, smem) != cudaSuccess) return GRIFFIN_ERR_CUDA;
         void *args[] = {&p, &act};
         if (launch_maybe_overlapped(fn, dim3(grid), dim3(DEC_THREADS), smem, stream, overlap, args) != cudaSuccess)
@@ -399,14 +407,17 @@ griffin_status launch_decode(const griffin_ff_desc *desc, int B, const griffin_f
     p.k = sets[0].k;
     p.ldk = sets[0].ldk;
     p.B = B;
-    if (desc->dtype == GRIFFIN_DT_F32) return decode_simt<float>(p, desc->act, flags, stream);
+    const int act = act_sigma(desc->act);
+    const bool gated = act_gated(desc->act);
+    if (desc->dtype == GRIFFIN_DT_F32) return decode_simt<float>(p, act, gated, flags, stream);
+    if (!gated) return decode_bf16_mma(p, act, false, flags, stream);  // (the tcgen05 kernels are built for gated blocks)
     // one expert set for several sequences (Eq. 7): only the tcgen05 kernel streams it once for all of them
     // (a shape that its plan cannot place in shared memory or TMEM after all goes to the warp-level kernel)
     if (decode_tc_shared(p) || ((flags & GRIFFIN_DECODE_TCGEN05) && decode_tc_supported(p))) {
-        const griffin_status st = decode_bf16_tc(p, desc->act, flags, stream);
+        const griffin_status st = decode_bf16_tc(p, act, flags, stream);
         if (st != GRIFFIN_ERR_UNSUPPORTED) return st;
     }
-    return decode_bf16_mma(p, desc->act, flags, stream);
+    return decode_bf16_mma(p, act, true, flags, stream);
 }
 
 // ---------------------------------------------------------------------------------------

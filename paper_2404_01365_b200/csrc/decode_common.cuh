@@ -111,7 +111,8 @@ cudaError_t launch_maybe_overlapped(const void *func, dim3 grid, dim3 block, siz
 int slices_for(int rows, int grid);
 
 // bf16 decode through warp-level MMA (decode_mma.cu).
-griffin_status decode_bf16_mma(DecodeParams &p, int act, uint32_t flags, cudaStream_t stream);
+// act: the code of sigma (0..3); gated: whether the block has a gate (Eq. 3) or not (Eq. 2).
+griffin_status decode_bf16_mma(DecodeParams &p, int act, bool gated, uint32_t flags, cudaStream_t stream);
 
 // bf16 decode through tcgen05 (decode_tc.cu): d and ldk multiples of 128, a workspace for the
 // meeting point.

@@ -94,8 +94,10 @@ __device__ __forceinline__ bool ring_put(const IdxSmem &s, int stage_bytes, int 
 }
 
 // WPG: consumer warps of a group per (gate, up) pair = 4 / R; NU: 16-byte units of a row per
-// consumer thread of a group in the second half (row_units <= 128 * NU).
-template <int WPG, int NU>
+// consumer thread of a group in the second half (row_units <= 128 * NU).  GATED = false: the block
+// has no gate (Eq. 2), z_j = sigma(W_1[j, :] . x + b_1[j]); a pair of the first half is then two
+// consecutive experts' rows of W_1, staged like the rows of W_2^T.
+template <int WPG, int NU, bool GATED>
 __global__ void __launch_bounds__(DEC_THREADS, 1) decode_indexed_kernel(const __grid_constant__ IndexedParams p, int act) {
     constexpr int R = DEC_GROUP_WARPS / WPG;
     extern __shared__ __align__(128) uint8_t smem_raw[];
@@ -141,7 +143,17 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) decode_indexed_kernel(const __
             int e1 = lane + 32 < n ? __ldg(idx + (size_t)b * k + r0 + 32 + lane) : 0;
             if ((unsigned)e0 >= d_ff) e0 = 0;
             if ((unsigned)e1 >= d_ff) e1 = 0;
-            for (int pg = 0; ok && pg < n; pg += R, ++pgc) {  // (gate, up) pairs
+            for (int rg = 0; !GATED && ok && rg < n; rg += 2 * R, ++pgc) {  // no gate: rows of W_1, two per pair
+                const int row = rg + lane;
+                const int e = item_expert(e0, e1, row & 63);
+                const bool mine = lane < 2 * R && row < n;
+                const uint32_t rows = (uint32_t)min(2 * R, n - rg);
+                const uint8_t *src = wu + (size_t)e * row_bytes;
+                RingPos cur = (pgc & 1) ? pos1 : pos0;
+                ok = ring_put(s, stage_bytes, ns2, pgc & 1, cur, rows * row_bytes, mine, src, row_bytes, lane, ws, 20);
+                if (pgc & 1) pos1 = cur; else pos0 = cur;
+            }
+            for (int pg = 0; GATED && ok && pg < n; pg += R, ++pgc) {  // (gate, up) pairs
                 const int pair = pg + (lane >> 1);
                 const int e = item_expert(e0, e1, pair & 63);
                 const bool mine = lane < 2 * R && pair < n;
@@ -210,10 +222,11 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) decode_indexed_kernel(const __
         if (*s.abort) ok = false;
 
         // ---- first half: z of the slice
-        for (int pg = 0; pg < n; pg += R, ++pgc) {
+        const int n_pairs = GATED ? n : (n + 1) >> 1;
+        for (int pg = 0; pg < n_pairs; pg += R, ++pgc) {
             if (!ok) continue;
             if ((int)(pgc & 1) != group) continue;
-            const bool have = pg + my_pair < n;
+            const bool have = pg + my_pair < n_pairs;
             float acc[MMA_ACCS][4] = {};
             const int stage = group * ns2 + pos.slot;
             if (!wait_or_abort(&s.full[stage], pos.round & 1, s.abort, ws, 22)) {
@@ -246,18 +259,25 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) decode_indexed_kernel(const __
         }
         group_barrier(group);  // this group's partial sums are in place
         if (*s.abort) ok = false;
-        if (tig < n && (int)((pgc0 + tig / R) & 1) == group) {
+        const int my_pair_of_item = GATED ? tig : tig >> 1;  // the pair that holds this thread's neuron
+        if (tig < n && (int)((pgc0 + my_pair_of_item / R) & 1) == group) {
             float a0 = 0.f, a1 = 0.f;
             for (int w = 0; w < WPG; ++w) {
-                const float2 v = part[tig * DEC_CONSUMER_WARPS + w];
+                const float2 v = part[my_pair_of_item * DEC_CONSUMER_WARPS + w];
                 a0 += v.x;
                 a1 += v.y;
             }
             float zv = 0.f;
             if ((unsigned)my_e < (unsigned)p.d_ff) {
-                if (p.b_gate) a0 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.b_gate)[my_e]);
-                if (p.b_up) a1 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.b_up)[my_e]);
-                zv = sigma_rt(act, a0) * a1;
+                if (GATED) {
+                    if (p.b_gate) a0 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.b_gate)[my_e]);
+                    if (p.b_up) a1 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.b_up)[my_e]);
+                    zv = sigma_rt(act, a0) * a1;
+                } else {
+                    float u = (tig & 1) ? a1 : a0;
+                    if (p.b_up) u += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.b_up)[my_e]);
+                    zv = sigma_rt(act, u);
+                }
             } else {
                 raise_status(ws, DEV_STATUS_BAD_INDEX, 23);
             }
@@ -467,14 +487,18 @@ griffin_status launch_decode_indexed(const griffin_ff_desc *desc, int B, const g
     const int wpg = DEC_GROUP_WARPS / pl.R;
     const int nu = (pl.row_units + 127) / 128;
     const void *fn = nullptr;
-    if (wpg == 1 && nu <= 2) fn = (const void *)decode_indexed_kernel<1, 2>;
-    else if (wpg == 2 && nu <= 4) fn = (const void *)decode_indexed_kernel<2, 4>;
-    else if (wpg == 4 && nu <= 8) fn = (const void *)decode_indexed_kernel<4, 8>;
+    const bool gated = act_gated(desc->act);
+    if (wpg == 1 && nu <= 2)
+        fn = gated ? (const void *)decode_indexed_kernel<1, 2, true> : (const void *)decode_indexed_kernel<1, 2, false>;
+    else if (wpg == 2 && nu <= 4)
+        fn = gated ? (const void *)decode_indexed_kernel<2, 4, true> : (const void *)decode_indexed_kernel<2, 4, false>;
+    else if (wpg == 4 && nu <= 8)
+        fn = gated ? (const void *)decode_indexed_kernel<4, 8, true> : (const void *)decode_indexed_kernel<4, 8, false>;
     else return GRIFFIN_ERR_UNSUPPORTED;
     const size_t smem = (size_t)p.n_stages * pl.stage_bytes + idx_fixed_smem(p.d, p.n_stages);
     if (smem > 227 * 1024) return GRIFFIN_ERR_UNSUPPORTED;
     if (ensure_dynamic_smem(fn, smem) != cudaSuccess) return GRIFFIN_ERR_CUDA;
-    int act = desc->act;
+    int act = act_sigma(desc->act);
     void *args[] = {&p, &act};
     const bool overlap = (flags & GRIFFIN_DECODE_OVERLAP_WEIGHT_PREFETCH) != 0;
     if (launch_maybe_overlapped(fn, dim3(grid), dim3(DEC_THREADS), smem, stream, overlap, args) != cudaSuccess)

@@ -47,6 +47,10 @@ namespace griffin {
 //                 item = (sequence, slice of neurons), pair = neuron.
 //   DOWN = true : down, y[b, c] = w_down_c[c, :] . z[b] + b_down[c];
 //                 item = (sequence, chunk of output rows), pair = two consecutive rows.
+// A block without a gate (Eq. 2) has a first half of its own, z[b, j] = sigma(up_j . x + b_up_j):
+// item = (sequence, slice of neurons), pair = two consecutive rows of W_1_hat, as in the down half.
+// The three are the MODEs below.
+constexpr int MODE_GATE_UP = 0, MODE_DOWN = 1, MODE_UP = 2;
 struct FusedPlan {
     MmaPlan gu, dn;   // per-half geometry (their n_stages / stage_bytes are overridden below)
     int slot_bytes;   // ring slot = the larger of the two halves' stages
@@ -66,9 +70,11 @@ __device__ __forceinline__ MmaSmem carve_fused(uint8_t *smem, const FusedPlan &f
 }
 
 // Producer side of one half.  Lane l < 2R copies row (l & 1) of pair (l >> 1).  Weights only.
-template <bool DOWN>
+template <int MODE>
 __device__ __forceinline__ bool produce_half(const DecodeParams &p, const MmaPlan &plan, const MmaSmem &s, int n_stages,
                                              int slot_bytes, int n_slices, RingPos (&pos)[2], uint32_t &pgc, int lane) {
+    constexpr bool DOWN = MODE == MODE_DOWN;
+    constexpr bool CONSEC = MODE != MODE_GATE_UP;  // a pair is two consecutive rows of one matrix
     const MmaPlan pl = plan;  // in registers: the asm statements in the loops clobber memory, and a reload costs a round trip
     void *const ws = p.ws;
     const int n_items = p.B * n_slices;
@@ -81,9 +87,9 @@ __device__ __forceinline__ bool produce_half(const DecodeParams &p, const MmaPla
         const int b = item / n_slices, sl = item - b * n_slices;
         const int r0 = (int)((long long)sl * total_rows / n_slices);
         const int r1 = (int)((long long)(sl + 1) * total_rows / n_slices);
-        const int n_pairs = DOWN ? (r1 - r0 + 1) / 2 : r1 - r0;
-        const uint8_t *mat =
-            static_cast<const uint8_t *>(DOWN ? p.seq[b].w_down : (my_row ? p.seq[b].w_up : p.seq[b].w_gate));
+        const int n_pairs = CONSEC ? (r1 - r0 + 1) / 2 : r1 - r0;
+        const uint8_t *mat = static_cast<const uint8_t *>(
+            DOWN ? p.seq[b].w_down : ((MODE == MODE_UP || my_row) ? p.seq[b].w_up : p.seq[b].w_gate));
         for (int pg = 0; pg < n_pairs; pg += pl.R, ++pgc) {
             // consumer group (pgc & 1) owns this pair group; each group has its own half of the
             // ring and its own count of stage uses, so that every barrier sees one strictly
@@ -91,10 +97,10 @@ __device__ __forceinline__ bool produce_half(const DecodeParams &p, const MmaPla
             // a parity that an older phase already satisfies)
             const int grp = pgc & 1;
             const int pair = pg + my_pair;
-            const int grow = DOWN ? r0 + 2 * pair + my_row : r0 + pair;  // row in the matrix
+            const int grow = CONSEC ? r0 + 2 * pair + my_row : r0 + pair;  // row in the matrix
             const bool mine = lane < 2 * pl.R && pair < n_pairs && grow < r1;
             // rows copied in this stage (the same for every chunk of the group)
-            const int rows_in_stage = DOWN ? min(2 * pl.R, r1 - r0 - 2 * pg) : 2 * min(pl.R, n_pairs - pg);
+            const int rows_in_stage = CONSEC ? min(2 * pl.R, r1 - r0 - 2 * pg) : 2 * min(pl.R, n_pairs - pg);
             RingPos cur = grp ? pos[1] : pos[0];  // (constant indices keep both in registers)
             for (int c = 0; c < pl.n_chunks; ++c, cur.advance(ns2)) {
                 const int units = min(pl.chunk_units, pl.row_units - c * pl.chunk_units);
@@ -126,10 +132,12 @@ __device__ __forceinline__ bool produce_half(const DecodeParams &p, const MmaPla
 // each lane keeps its units of it in registers (read straight from global memory, once per
 // item); otherwise (rows longer than MMA_CHUNK_UNITS_MAX units, down only) the vector is
 // staged in shared memory and read from there block by block.
-template <bool DOWN, bool VREG, int WPG>
+template <int MODE, bool VREG, int WPG>
 __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPlan &plan, const MmaSmem &s, int n_stages,
                                              int slot_bytes, int n_slices, RingPos &pos, uint32_t &pgc,
                                              int &item_parity, int act, int tid, int warp, int lane) {
+    constexpr bool DOWN = MODE == MODE_DOWN;
+    constexpr bool CONSEC = MODE != MODE_GATE_UP;  // a pair is two consecutive rows of one matrix
     const MmaPlan pl = plan;  // in registers: the asm statements in the loops clobber memory, and a reload costs a round trip
     void *const ws = p.ws;
     const int n_items = p.B * n_slices;
@@ -153,7 +161,7 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
         const int b = item / n_slices, sl = item - b * n_slices;
         const int r0 = (int)((long long)sl * total_rows / n_slices);
         const int r1 = (int)((long long)(sl + 1) * total_rows / n_slices);
-        const int n_pairs = DOWN ? (r1 - r0 + 1) / 2 : r1 - r0;
+        const int n_pairs = CONSEC ? (r1 - r0 + 1) / 2 : r1 - r0;
         float2 *part = s.part + item_parity * (DEC_MAX_ROWS * DEC_CONSUMER_WARPS);
         const uint32_t pgc0 = pgc;  // pair-group count at the start of the item: who owns which pair
         // the groups finish an item independently; before a further item (partial-sum buffers
@@ -228,7 +236,7 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
         // every thread of the group looks after the rows of the pairs its group owned
         const int tig = tid - group * (DEC_GROUP_WARPS * 32);
         const int my_row = tig;  // rows of the item: r0 + my_row (at most DEC_MAX_ROWS of them)
-        const int my_rows_pair = DOWN ? my_row >> 1 : my_row;
+        const int my_rows_pair = CONSEC ? my_row >> 1 : my_row;
         if (ok && my_row < r1 - r0 && (int)((pgc0 + my_rows_pair / pl.R) & 1) == group) {
             const int pair = my_rows_pair;
             float a0 = 0.f, a1 = 0.f;
@@ -237,7 +245,15 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
                 a0 += v.x;
                 a1 += v.y;
             }
-            if (!DOWN) {
+            if (MODE == MODE_UP) {
+                const int j = r0 + my_row;
+                float u = (my_row & 1) ? a1 : a0;
+                if (p.seq[b].b_up) u += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[b].b_up)[j]);
+                const float zv = sigma_rt(act, u);
+                const __nv_bfloat16 h = __float2bfloat16_rn(zv);
+                zbits[(size_t)b * 2 * p.ldk + j] = h;
+                if (Z_LO) zbits[(size_t)b * 2 * p.ldk + p.ldk + j] = __float2bfloat16_rn(zv - __bfloat162float(h));
+            } else if (!DOWN) {
                 const int j = r0 + my_row;
                 if (p.seq[b].b_gate) a0 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[b].b_gate)[j]);
                 if (p.seq[b].b_up) a1 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[b].b_up)[j]);
@@ -265,8 +281,10 @@ __device__ __forceinline__ bool consume_half(const DecodeParams &p, const MmaPla
 #ifndef GRIFFIN_DEC_MIN_CTAS
 #define GRIFFIN_DEC_MIN_CTAS 1
 #endif
+template <bool GATED>
 __global__ void __launch_bounds__(DEC_THREADS, GRIFFIN_DEC_MIN_CTAS) decode_fused_kernel(const __grid_constant__ DecodeParams p,
                                                                    const __grid_constant__ FusedPlan fp, int act) {
+    constexpr int FIRST = GATED ? MODE_GATE_UP : MODE_UP;
     extern __shared__ __align__(128) uint8_t smem_raw[];
     const MmaSmem s = carve_fused(smem_raw, fp);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -287,8 +305,8 @@ __global__ void __launch_bounds__(DEC_THREADS, GRIFFIN_DEC_MIN_CTAS) decode_fuse
         //      consumers are still waiting for the other CTAs' z
         RingPos pos[2] = {{0, 0, 0}, {0, 0, 0}};
         uint32_t pgc = 0;
-        if (produce_half<false>(p, fp.gu, s, fp.n_stages, fp.slot_bytes, p.n_slices, pos, pgc, lane))
-            produce_half<true>(p, fp.dn, s, fp.n_stages, fp.slot_bytes, p.n_slices_dn, pos, pgc, lane);
+        if (produce_half<FIRST>(p, fp.gu, s, fp.n_stages, fp.slot_bytes, p.n_slices, pos, pgc, lane))
+            produce_half<MODE_DOWN>(p, fp.dn, s, fp.n_stages, fp.slot_bytes, p.n_slices_dn, pos, pgc, lane);
         const uint32_t issued[2] = {pos[0].uses, pos[1].uses};
         if (lane == 0) producer_drain_mma(s, fp.n_stages, issued);
         return;
@@ -299,14 +317,14 @@ __global__ void __launch_bounds__(DEC_THREADS, GRIFFIN_DEC_MIN_CTAS) decode_fuse
     RingPos pos = {0, 0, 0};  // of this warp's group
     uint32_t pgc = 0;         // pair groups seen by everybody
     int item_parity = 0;
-#define GRIFFIN_CONSUME(DOWN_, VREG_, WPG_, PLAN_, SLICES_) \
-    consume_half<DOWN_, VREG_, WPG_>(p, PLAN_, s, fp.n_stages, fp.slot_bytes, SLICES_, pos, pgc, item_parity, act, tid, warp, lane)
+#define GRIFFIN_CONSUME(MODE_, VREG_, WPG_, PLAN_, SLICES_) \
+    consume_half<MODE_, VREG_, WPG_>(p, PLAN_, s, fp.n_stages, fp.slot_bytes, SLICES_, pos, pgc, item_parity, act, tid, warp, lane)
     // warps per pair as a compile-time constant: block offsets become immediates.  A row of
     // W_g_hat or W_1_hat (d <= GRIFFIN_MAX_D elements) is always one chunk.
     switch (fp.gu.R) {
-        case 4: GRIFFIN_CONSUME(false, true, 1, fp.gu, p.n_slices); break;
-        case 2: GRIFFIN_CONSUME(false, true, 2, fp.gu, p.n_slices); break;
-        default: GRIFFIN_CONSUME(false, true, 4, fp.gu, p.n_slices); break;
+        case 4: GRIFFIN_CONSUME(FIRST, true, 1, fp.gu, p.n_slices); break;
+        case 2: GRIFFIN_CONSUME(FIRST, true, 2, fp.gu, p.n_slices); break;
+        default: GRIFFIN_CONSUME(FIRST, true, 4, fp.gu, p.n_slices); break;
     }
     // each group reports on its own: 2 arrivals per CTA
     const int group = warp / DEC_GROUP_WARPS;
@@ -316,18 +334,18 @@ __global__ void __launch_bounds__(DEC_THREADS, GRIFFIN_DEC_MIN_CTAS) decode_fuse
     group_barrier(group);  // the group has seen everybody: z is complete
     if (fp.dn.n_chunks == 1) {
         switch (fp.dn.R) {
-            case 4: GRIFFIN_CONSUME(true, true, 1, fp.dn, p.n_slices_dn); break;
-            case 2: GRIFFIN_CONSUME(true, true, 2, fp.dn, p.n_slices_dn); break;
-            default: GRIFFIN_CONSUME(true, true, 4, fp.dn, p.n_slices_dn); break;
+            case 4: GRIFFIN_CONSUME(MODE_DOWN, true, 1, fp.dn, p.n_slices_dn); break;
+            case 2: GRIFFIN_CONSUME(MODE_DOWN, true, 2, fp.dn, p.n_slices_dn); break;
+            default: GRIFFIN_CONSUME(MODE_DOWN, true, 4, fp.dn, p.n_slices_dn); break;
         }
     } else {  // chunks of 8 KB or more: at most two pairs per stage
-        if (fp.dn.R == 2) GRIFFIN_CONSUME(true, false, 2, fp.dn, p.n_slices_dn);
-        else GRIFFIN_CONSUME(true, false, 4, fp.dn, p.n_slices_dn);
+        if (fp.dn.R == 2) GRIFFIN_CONSUME(MODE_DOWN, false, 2, fp.dn, p.n_slices_dn);
+        else GRIFFIN_CONSUME(MODE_DOWN, false, 4, fp.dn, p.n_slices_dn);
     }
 #undef GRIFFIN_CONSUME
 }
 
-griffin_status decode_bf16_mma(DecodeParams &p, int act, uint32_t flags, cudaStream_t stream) {
+griffin_status decode_bf16_mma(DecodeParams &p, int act, bool gated, uint32_t flags, cudaStream_t stream) {
     const int sms = device_sm_count();
     if (sms <= 0) return GRIFFIN_ERR_CUDA;
     if (p.ws == nullptr) return GRIFFIN_ERR_WORKSPACE;  // the meeting point's counters live in the header
@@ -345,7 +363,7 @@ griffin_status decode_bf16_mma(DecodeParams &p, int act, uint32_t flags, cudaStr
     const int grid = sms;
     const size_t smem = (size_t)fp.n_stages * fp.slot_bytes + fp.vec_bytes + mma_fixed_smem(fp.n_stages);
     if (smem > 227 * 1024) return GRIFFIN_ERR_UNSUPPORTED;
-    const void *fn = (const void *)decode_fused_kernel;
+    const void *fn = gated ? (const void *)decode_fused_kernel<true> : (const void *)decode_fused_kernel<false>;
     if (ensure_dynamic_smem(fn, smem) != cudaSuccess) return GRIFFIN_ERR_CUDA;
     void *args[] = {&p, &fp, &act};
     if (launch_maybe_overlapped(fn, dim3(grid), dim3(DEC_THREADS), smem, stream, overlap, args) != cudaSuccess)

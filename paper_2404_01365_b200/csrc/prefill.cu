@@ -50,7 +50,7 @@ PrefillScratch prefill_scratch(const griffin_ff_desc *desc, int S) {
         int bn = 0, splits = 1;
         gemm2_plan(S, desc->d, &bn, &splits);
         size_t need = splits > 1 ? (size_t)splits * S * desc->d * sizeof(float) : 0;
-        const size_t tail = gemm1_tail_bytes(S, desc->d, desc->d_ff);  // (used up before the down projection starts)
+        const size_t tail = gemm1_tail_bytes(S, desc->d, gemm1_col_tiles(desc));  // (used up before the down projection starts)
         if (tail > need) need = tail;
         if (need > 0) off = align_up(off + need, 256);
     }
@@ -80,8 +80,9 @@ __device__ __forceinline__ void load_tile_t(const T *__restrict__ src, int ld, i
     }
 }
 
-// Step 1 (SIMT): one CTA = 64 tokens x 64 neurons.
-template <typename T>
+// Step 1 (SIMT): one CTA = 64 tokens x 64 neurons.  GATED = false: the block has no gate (Eq. 2),
+// Z = sigma(X W_1^T + b_1), and w_gate / b_gate are not touched.
+template <typename T, bool GATED>
 __global__ void __launch_bounds__(PF_THREADS) ff1_simt_kernel(const T *__restrict__ x, const T *__restrict__ w_gate,
                                                               const T *__restrict__ w_up, const T *__restrict__ b_gate,
                                                               const T *__restrict__ b_up, T *__restrict__ z,
@@ -95,20 +96,20 @@ __global__ void __launch_bounds__(PF_THREADS) ff1_simt_kernel(const T *__restric
     float ga[4][4] = {}, ua[4][4] = {};
     for (int k0 = 0; k0 < d; k0 += PF_BK) {
         load_tile_t<T>(x, d, S, d, m0, k0, xs, tid);
-        load_tile_t<T>(w_gate, d, d_ff, d, n0, k0, gs, tid);
+        if (GATED) load_tile_t<T>(w_gate, d, d_ff, d, n0, k0, gs, tid);
         load_tile_t<T>(w_up, d, d_ff, d, n0, k0, us, tid);
         __syncthreads();
 #pragma unroll
         for (int kk = 0; kk < PF_BK; ++kk) {
             const float4 a = *reinterpret_cast<const float4 *>(&xs[kk][ty * 4]);
-            const float4 g = *reinterpret_cast<const float4 *>(&gs[kk][tx * 4]);
             const float4 u = *reinterpret_cast<const float4 *>(&us[kk][tx * 4]);
+            const float4 g = GATED ? *reinterpret_cast<const float4 *>(&gs[kk][tx * 4]) : u;
             const float av[4] = {a.x, a.y, a.z, a.w}, gv[4] = {g.x, g.y, g.z, g.w}, uv[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
             for (int i = 0; i < 4; ++i)
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    ga[i][j] = fmaf(av[i], gv[j], ga[i][j]);
+                    if (GATED) ga[i][j] = fmaf(av[i], gv[j], ga[i][j]);
                     ua[i][j] = fmaf(av[i], uv[j], ua[i][j]);
                 }
         }
@@ -123,9 +124,9 @@ __global__ void __launch_bounds__(PF_THREADS) ff1_simt_kernel(const T *__restric
             const int col = n0 + tx * 4 + j;
             if (row < S && col < d_ff) {
                 float g = ga[i][j], u = ua[i][j];
-                if (b_gate) g += Elem<T>::to_float(b_gate[col]);
+                if (GATED && b_gate) g += Elem<T>::to_float(b_gate[col]);
                 if (b_up) u += Elem<T>::to_float(b_up[col]);
-                const float zv = sigma_rt(act, g) * u;
+                const float zv = GATED ? sigma_rt(act, g) * u : sigma_rt(act, u);
                 z[(size_t)row * d_ff + col] = Elem<T>::from_float(zv);
                 if (zf) zf[(size_t)row * d_ff + col] = zv;
                 sq = fmaf(zv, zv, sq);
@@ -303,10 +304,15 @@ static griffin_status prefill_typed(const griffin_ff_desc *desc, const griffin_f
     } else {
         n_col_tiles = (d_ff + PF_BN - 1) / PF_BN;
         const dim3 g1(n_col_tiles, (S + PF_BM - 1) / PF_BM);
-        ff1_simt_kernel<T><<<g1, PF_THREADS, 0, stream>>>(
-            static_cast<const T *>(x), static_cast<const T *>(w->w_gate), static_cast<const T *>(w->w_up),
-            static_cast<const T *>(w->b_gate), static_cast<const T *>(w->b_up), z, zf, rowsq, S, d, d_ff, n_col_tiles,
-            desc->act);
+        if (act_gated(desc->act))
+            ff1_simt_kernel<T, true><<<g1, PF_THREADS, 0, stream>>>(
+                static_cast<const T *>(x), static_cast<const T *>(w->w_gate), static_cast<const T *>(w->w_up),
+                static_cast<const T *>(w->b_gate), static_cast<const T *>(w->b_up), z, zf, rowsq, S, d, d_ff,
+                n_col_tiles, desc->act);
+        else
+            ff1_simt_kernel<T, false><<<g1, PF_THREADS, 0, stream>>>(
+                static_cast<const T *>(x), nullptr, static_cast<const T *>(w->w_up), nullptr,
+                static_cast<const T *>(w->b_up), z, zf, rowsq, S, d, d_ff, n_col_tiles, act_sigma(desc->act));
         if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
     }
     if (!ff2_done && y != nullptr) {

@@ -1,8 +1,9 @@
 // Prompt-phase FF on the 5th-generation tensor cores (Eqs. 1 and 3 of the GRIFFIN paper), bf16
 // storage, fp32 accumulation:
-//   kernel<DUAL = true > : Z = sigma(X W_g^T + b_g) * (X W_1^T + b_1), also Z in fp32 and the
-//                          per-tile partial sums of squares of its rows (for the statistic)
-//   kernel<DUAL = false> : Y = Z W_2^T + b_2
+//   kernel<KIND = 1> : Z = sigma(X W_g^T + b_g) * (X W_1^T + b_1), also Z in fp32 and the
+//                      per-tile partial sums of squares of its rows (for the statistic)
+//   kernel<KIND = 2> : the same for a block without a gate (Eq. 2): Z = sigma(X W_1^T + b_1)
+//   kernel<KIND = 0> : Y = Z W_2^T + b_2
 //
 // One persistent CTA per SM, 192 threads in three roles:
 //   warp 0      TMA producer: cp.async.bulk.tensor (2-D tiles, 128-byte swizzle, no multicast)
@@ -17,6 +18,8 @@
 // For DUAL the gate and up tiles of the same 128 neurons are loaded one behind the other, so
 // that a single N = 256 MMA against the shared X tile fills columns 0..127 with the gate
 // and 128..255 with the up pre-activations: the epilogue thread that owns a row finds both.
+// Without a gate the same two loads take 256 consecutive neurons of W_1, and every accumulator
+// column is a neuron of its own.
 //
 // Every wait is bounded; after a give-up the CTA still frees its TMEM before it returns.
 #include "common.cuh"
@@ -51,6 +54,7 @@ struct TcParams {
     // whose raw accumulators (gate | up, fp32) go to tail_part [part][128 rows][256 columns]
     int tail_first, tail_ks;
     float *tail_part;
+    int gated;  // first GEMM: 1 = gate | up tiles of 128 neurons, 0 = 256 neurons of W_1 (no gate)
 };
 
 // Work item -> (row block m, column block n, K blocks [kb0, kb1), index of the cut tile's part or -1).
@@ -93,11 +97,13 @@ struct TcSmem {
 };
 constexpr size_t TC_TAIL_BYTES = (2 * TC_STAGES + 4) * sizeof(uint64_t) + 16;
 
-template <bool DUAL, int BN>
+constexpr int TC_PLAIN = 0, TC_GATED = 1, TC_WIDE = 2;
+template <int KIND, int BN>
 __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant__ CUtensorMap map_a,
                                                            const __grid_constant__ CUtensorMap map_b0,
                                                            const __grid_constant__ CUtensorMap map_b1,
                                                            const __grid_constant__ TcParams p) {
+    constexpr bool DUAL = KIND != TC_PLAIN;        // two weight loads of 128 rows per stage, N = 256
     constexpr int NT = DUAL ? 256 : BN;            // MMA N = TMEM columns of one accumulator stage
     constexpr int B_ROWS = DUAL ? 128 : BN;        // rows of one weight tile load
     constexpr int A_BYTES = TC_BM * TC_BK * 2;     // 16 KB
@@ -156,8 +162,10 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
                     uint8_t *a = s.stages + (size_t)stage * STAGE_BYTES;
                     mbar_arrive_expect_tx(&s.full[stage], STAGE_BYTES);
                     tma_load_2d(a, &map_a, kb * TC_BK, m * TC_BM, &s.full[stage]);
-                    tma_load_2d(a + A_BYTES, &map_b0, kb * TC_BK, n * B_ROWS, &s.full[stage]);
-                    if (DUAL) tma_load_2d(a + A_BYTES + B_ROWS * TC_BK * 2, &map_b1, kb * TC_BK, n * B_ROWS, &s.full[stage]);
+                    tma_load_2d(a + A_BYTES, &map_b0, kb * TC_BK, KIND == TC_WIDE ? n * 256 : n * B_ROWS, &s.full[stage]);
+                    if (DUAL)
+                        tma_load_2d(a + A_BYTES + B_ROWS * TC_BK * 2, &map_b1, kb * TC_BK,
+                                    KIND == TC_WIDE ? n * 256 + 128 : n * B_ROWS, &s.full[stage]);
                 }
             }
             // stay until every copy that was started has landed
@@ -224,6 +232,38 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
                     for (int v = 0; v < 8; ++v)
                         reinterpret_cast<float4 *>(dst + c)[v] = make_float4(a[4 * v], a[4 * v + 1], a[4 * v + 2], a[4 * v + 3]);
                 }
+            } else if (KIND == TC_WIDE) {
+                // no gate: every one of the 256 accumulator columns is a neuron, Z = sigma(acc + b_1)
+                float sq = 0.f;
+#pragma unroll 1
+                for (int c = 0; c < 256; c += 32) {
+                    float u[32];
+                    tmem_ld32(taddr + c, u);
+                    const int col = n * 256 + c;
+                    uint32_t packed[16];
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        float u0 = u[i], u1 = u[i + 1];
+                        if (p.bias1) { u0 += __bfloat162float(p.bias1[col + i]); u1 += __bfloat162float(p.bias1[col + i + 1]); }
+                        const float z0 = sigma_rt(p.act, u0), z1 = sigma_rt(p.act, u1);
+                        u[i] = z0;
+                        u[i + 1] = z1;
+                        sq = fmaf(z0, z0, sq);
+                        sq = fmaf(z1, z1, sq);
+                        const __nv_bfloat162 h = __floats2bfloat162_rn(z0, z1);
+                        packed[i >> 1] = *reinterpret_cast<const uint32_t *>(&h);
+                    }
+                    if (live) {
+                        uint4 *zo = reinterpret_cast<uint4 *>(p.out + (size_t)row * p.n_total + col);
+                        float4 *fo = reinterpret_cast<float4 *>(p.zf + (size_t)row * p.n_total + col);
+#pragma unroll
+                        for (int v = 0; v < 4; ++v)
+                            zo[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+#pragma unroll
+                        for (int v = 0; v < 8; ++v) fo[v] = make_float4(u[4 * v], u[4 * v + 1], u[4 * v + 2], u[4 * v + 3]);
+                    }
+                }
+                if (live) p.rowsq[(size_t)row * p.n_tiles + n] = sq;
             } else if (DUAL) {
                 float sq = 0.f;
 #pragma unroll 1
@@ -309,7 +349,9 @@ __global__ void __launch_bounds__(128) dual_tail_finish_kernel(TcParams p) {
     const int w = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     const int tile = p.tail_first + w / TC_BM, r = w % TC_BM, c = lane * 4;
     const int m = tile % p.m_tiles, n = tile / p.m_tiles;
-    const int row = m * TC_BM + r, col = n * 128 + c;
+    // with a gate the two halves of a part are the gate and up sums of the same 128 neurons; without
+    // one they are 256 neurons of W_1
+    const int row = m * TC_BM + r, col = p.gated ? n * 128 + c : n * 256 + c, col2 = p.gated ? col : col + 128;
     float4 g = make_float4(0.f, 0.f, 0.f, 0.f), u = g, a[4], b[4];
 #pragma unroll
     for (int sp = 0; sp < 4; ++sp) {  // at most four parts; all loads in flight together
@@ -327,12 +369,33 @@ __global__ void __launch_bounds__(128) dual_tail_finish_kernel(TcParams p) {
     }
     float gv[4] = {g.x, g.y, g.z, g.w}, uv[4] = {u.x, u.y, u.z, u.w}, z[4];
     float sq = 0.f;
+    if (!p.gated) {
+        float z2[4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        if (p.bias0) gv[i] += __bfloat162float(p.bias0[col + i]);
-        if (p.bias1) uv[i] += __bfloat162float(p.bias1[col + i]);
-        z[i] = sigma_rt(p.act, gv[i]) * uv[i];
-        sq = fmaf(z[i], z[i], sq);
+        for (int i = 0; i < 4; ++i) {
+            if (p.bias1) {
+                gv[i] += __bfloat162float(p.bias1[col + i]);
+                uv[i] += __bfloat162float(p.bias1[col2 + i]);
+            }
+            z[i] = sigma_rt(p.act, gv[i]);
+            z2[i] = sigma_rt(p.act, uv[i]);
+            sq = fmaf(z[i], z[i], sq);
+            sq = fmaf(z2[i], z2[i], sq);
+        }
+        if (row < p.S) {
+            const __nv_bfloat162 h0 = __floats2bfloat162_rn(z2[0], z2[1]), h1 = __floats2bfloat162_rn(z2[2], z2[3]);
+            *reinterpret_cast<uint2 *>(p.out + (size_t)row * p.n_total + col2) =
+                make_uint2(*reinterpret_cast<const uint32_t *>(&h0), *reinterpret_cast<const uint32_t *>(&h1));
+            *reinterpret_cast<float4 *>(p.zf + (size_t)row * p.n_total + col2) = make_float4(z2[0], z2[1], z2[2], z2[3]);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (p.bias0) gv[i] += __bfloat162float(p.bias0[col + i]);
+            if (p.bias1) uv[i] += __bfloat162float(p.bias1[col + i]);
+            z[i] = sigma_rt(p.act, gv[i]) * uv[i];
+            sq = fmaf(z[i], z[i], sq);
+        }
     }
     if (row < p.S) {
         const __nv_bfloat162 h0 = __floats2bfloat162_rn(z[0], z[1]), h1 = __floats2bfloat162_rn(z[2], z[3]);
@@ -369,8 +432,12 @@ __global__ void splitk_reduce_kernel(const float *__restrict__ part, const __nv_
 // ---------------------------------------------------------------------------------------
 constexpr int TC_TARGET_CTAS = 148;  // SMs of a B200: what a grid should fill
 
-void gemm1_tail_plan(int S, int d, int d_ff, int *tail_first, int *ks) {
-    const int tiles = ((S + TC_BM - 1) / TC_BM) * (d_ff / 128);
+int gemm1_col_tiles(const griffin_ff_desc *desc) {
+    return GRIFFIN_ACT_IS_GATED(desc->act) ? desc->d_ff / 128 : desc->d_ff / 256;
+}
+
+void gemm1_tail_plan(int S, int d, int n_col_tiles, int *tail_first, int *ks) {
+    const int tiles = ((S + TC_BM - 1) / TC_BM) * n_col_tiles;
     const int rem = tiles % TC_TARGET_CTAS;
     *tail_first = tiles;
     *ks = 1;
@@ -382,11 +449,11 @@ void gemm1_tail_plan(int S, int d, int d_ff, int *tail_first, int *ks) {
     }
 }
 
-size_t gemm1_tail_bytes(int S, int d, int d_ff) {
+size_t gemm1_tail_bytes(int S, int d, int n_col_tiles) {
     int first = 0, ks = 1;
-    gemm1_tail_plan(S, d, d_ff, &first, &ks);
+    gemm1_tail_plan(S, d, n_col_tiles, &first, &ks);
     if (ks <= 1) return 0;
-    const int tiles = ((S + TC_BM - 1) / TC_BM) * (d_ff / 128);
+    const int tiles = ((S + TC_BM - 1) / TC_BM) * n_col_tiles;
     return (size_t)(tiles - first) * ks * TC_BM * 256 * sizeof(float);
 }
 
@@ -415,19 +482,20 @@ static bool make_map(CUtensorMap *map, const void *base, int rows, int cols, int
 bool prefill_tc_supported(const griffin_ff_desc *desc, int S) {
     if (desc->dtype != GRIFFIN_DT_BF16 || S < 1) return false;
     if (desc->d % 128 != 0 || desc->d_ff % 128 != 0) return false;  // whole tiles in N, whole stages in K
+    if (!GRIFFIN_ACT_IS_GATED(desc->act) && desc->d_ff % 256 != 0) return false;  // (tiles of 256 neurons)
     return encode_tiled_fn() != nullptr;
 }
 
-template <bool DUAL, int BN>
+template <int KIND, int BN>
 static griffin_status launch_tc(const CUtensorMap &ma, const CUtensorMap &mb0, const CUtensorMap &mb1, const TcParams &p,
                                 int sms, cudaStream_t stream) {
-    constexpr int NT = DUAL ? 256 : BN;
+    constexpr int NT = KIND != TC_PLAIN ? 256 : BN;
     const size_t smem = 1024 + (size_t)TC_STAGES * (TC_BM * TC_BK * 2 + NT * TC_BK * 2) + TC_TAIL_BYTES;
-    const void *fn = (const void *)ff_tc_kernel<DUAL, BN>;
+    const void *fn = (const void *)ff_tc_kernel<KIND, BN>;
     if (ensure_dynamic_smem(fn, smem) != cudaSuccess) return GRIFFIN_ERR_CUDA;
     const int tiles = p.tail_ks > 1 ? p.tail_first + (p.m_tiles * p.n_tiles - p.tail_first) * p.tail_ks
                                     : p.m_tiles * p.n_tiles * p.splits;
-    ff_tc_kernel<DUAL, BN><<<tiles < sms ? tiles : sms, TC_THREADS, smem, stream>>>(ma, mb0, mb1, p);
+    ff_tc_kernel<KIND, BN><<<tiles < sms ? tiles : sms, TC_THREADS, smem, stream>>>(ma, mb0, mb1, p);
     return cudaGetLastError() == cudaSuccess ? GRIFFIN_OK : GRIFFIN_ERR_CUDA;
 }
 
@@ -438,28 +506,31 @@ griffin_status launch_prefill_tc(const griffin_ff_desc *desc, const griffin_ff_w
     const int sms = device_sm_count();
     if (sms <= 0) return GRIFFIN_ERR_CUDA;
     const int m_tiles = (S + TC_BM - 1) / TC_BM;
+    const bool gated = GRIFFIN_ACT_IS_GATED(desc->act);
     CUtensorMap mx, mg, mu;
-    if (!make_map(&mx, x, S, d, TC_BM) || !make_map(&mg, w->w_gate, d_ff, d, 128) ||
-        !make_map(&mu, w->w_up, d_ff, d, 128))
+    if (!make_map(&mx, x, S, d, TC_BM) || !make_map(&mu, w->w_up, d_ff, d, 128) ||
+        !make_map(&mg, gated ? w->w_gate : w->w_up, d_ff, d, 128))
         return GRIFFIN_ERR_CUDA;
     TcParams p = {};
     p.S = S;
     p.n_total = d_ff;
     p.K = d;
     p.m_tiles = m_tiles;
-    p.n_tiles = d_ff / 128;
-    p.bias0 = static_cast<const __nv_bfloat16 *>(w->b_gate);
+    p.n_tiles = gemm1_col_tiles(desc);
+    p.gated = gated ? 1 : 0;
+    p.bias0 = static_cast<const __nv_bfloat16 *>(gated ? w->b_gate : nullptr);
     p.bias1 = static_cast<const __nv_bfloat16 *>(w->b_up);
     p.out = z;
     p.zf = zf;
     p.rowsq = rowsq;
-    p.act = desc->act;
+    p.act = act_sigma(desc->act);
     p.ws = ws;
     p.splits = 1;
-    gemm1_tail_plan(S, d, d_ff, &p.tail_first, &p.tail_ks);
+    gemm1_tail_plan(S, d, p.n_tiles, &p.tail_first, &p.tail_ks);
     p.tail_part = ypart;  // (the down projection's partials use the same scratch, later)
     *n_col_tiles = p.n_tiles;
-    griffin_status st = launch_tc<true, 128>(mx, mg, mu, p, sms, stream);
+    griffin_status st = gated ? launch_tc<TC_GATED, 128>(mx, mg, mu, p, sms, stream)
+                              : launch_tc<TC_WIDE, 128>(mx, mg, mu, p, sms, stream);
     if (st == GRIFFIN_OK && p.tail_ks > 1) {
         dual_tail_finish_kernel<<<(p.m_tiles * p.n_tiles - p.tail_first) * (TC_BM / 4), 128, 0, stream>>>(p);
         if (cudaGetLastError() != cudaSuccess) st = GRIFFIN_ERR_CUDA;
@@ -485,7 +556,8 @@ griffin_status launch_prefill_tc(const griffin_ff_desc *desc, const griffin_ff_w
     q.splits = splits;
     q.part = splits > 1 ? ypart : nullptr;
     q.tail_ks = 1;
-    st = bn == 256 ? launch_tc<false, 256>(mz, md, md, q, sms, stream) : launch_tc<false, 128>(mz, md, md, q, sms, stream);
+    st = bn == 256 ? launch_tc<TC_PLAIN, 256>(mz, md, md, q, sms, stream)
+                   : launch_tc<TC_PLAIN, 128>(mz, md, md, q, sms, stream);
     if (st != GRIFFIN_OK || splits == 1) return st;
     const size_t n_elems = (size_t)S * d;
     splitk_reduce_kernel<<<(unsigned)((n_elems / 4 + 255) / 256), 256, 0, stream>>>(

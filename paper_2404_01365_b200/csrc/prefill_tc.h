@@ -13,13 +13,17 @@ namespace griffin {
 // arithmetic on the shape, so that workspace sizing and launch agree.
 void gemm2_plan(int S, int d, int *bn, int *splits);
 
-// The first GEMM has m_tiles x (d_ff / 128) tiles for one CTA per SM.  When the last round of
+// Column tiles of the first GEMM: 128 neurons each with a gate (gate | up side by side in the
+// accumulator), 256 without.
+int gemm1_col_tiles(const griffin_ff_desc *desc);
+
+// The first GEMM has m_tiles x n_col_tiles tiles for one CTA per SM.  When the last round of
 // tiles would leave more than half of the SMs idle, those tiles are cut along K into *ks parts
 // (2..4) whose fp32 partial accumulators meet in a small finishing kernel: *tail_first is the
 // first tile that is cut (= the number of tiles when none is).  Pure arithmetic on the shape.
-void gemm1_tail_plan(int S, int d, int d_ff, int *tail_first, int *ks);
+void gemm1_tail_plan(int S, int d, int n_col_tiles, int *tail_first, int *ks);
 // Bytes of fp32 scratch that the parts of the cut tiles need (0 when none is cut).
-size_t gemm1_tail_bytes(int S, int d, int d_ff);
+size_t gemm1_tail_bytes(int S, int d, int n_col_tiles);
 
 // Whether the tensor-core kernels take this shape (bf16, d and d_ff multiples of 64, ...).
 bool prefill_tc_supported(const griffin_ff_desc *desc, int S);

@@ -25,6 +25,7 @@ class FFStack:
         self.device = device
         self.tdtype = torch.float32 if dtype == "f32" else torch.bfloat16
         self.desc = G.make_desc(d, d_ff, act, dtype)
+        self.n_mats = 3 if G.act_is_gated(act) else 2   # a block without a gate has no W_g (w_gate is None)
         self.ldk = G.griffin_compact_ldk(k)
         self.ws = G.alloc_workspace(self.desc, S_max, n_seq, device)
         self.indexed = indexed
@@ -74,11 +75,11 @@ class FFStack:
     # ---- accounting (bytes and flops the algorithm needs, not what was moved) -----------
     def decode_bytes_per_call(self):
         b = 4 if self.tdtype == torch.float32 else 2
-        return self.n_seq * (3 * self.k * self.d * b + 2 * self.d * b)
+        return self.n_seq * (self.n_mats * self.k * self.d * b + 2 * self.d * b)
 
     def prefill_flops(self, S):
-        return 6 * S * self.d * self.d_ff
+        return 2 * self.n_mats * S * self.d * self.d_ff
 
     def compact_bytes(self):
         b = 4 if self.tdtype == torch.float32 else 2
-        return 2 * 3 * self.k * self.d * b
+        return 2 * self.n_mats * self.k * self.d * b

@@ -26,6 +26,8 @@ F32 = "f32"
 BF16 = "bf16"
 SWIGLU = "swiglu"
 GEGLU_TANH = "geglu_tanh"
+RELU = "relu"                      # a block without a gate (Eq. 2 of the paper, as in OPT)
+NON_GATED = ("relu", "gelu_tanh", "gelu_erf", "silu")
 
 _T_W_GATE, _T_W_UP, _T_W_DOWN, _T_DIR, _T_NORM, _T_PROMPT, _T_DECODE = range(7)
 
@@ -64,6 +66,8 @@ WORKLOADS = {
         Workload("llama2_13b", 3, 5120, 13824, 2048, 256, 8, (0.5,), BF16, SWIGLU, 40, (4.0, 4.0)),
         Workload("mistral_7b", 4, 4096, 14336, 4096, 512, 4, (0.25, 0.5, 0.75, 1.0), BF16, SWIGLU, 32,
                  (1.0, 8.0)),
+        # not one of the five measured workloads: the FF shape of OPT-6.7B, a ReLU block without a gate
+        Workload("opt_6p7b", 5, 4096, 16384, 512, 128, 1, (0.5,), BF16, RELU, 32, (4.0, 4.0)),
     )
 }
 
@@ -109,9 +113,12 @@ def make_weights(w: Workload, layer: int, device="cpu"):
 
     Entries are i.i.d. N(0, 1/d) for the gate and up projections and
     N(0, 1/d_ff) for the down projection, rounded to the storage dtype.
+    w_gate is None for a block without a gate.
     """
     dt = w.torch_dtype
-    wg = _randn((w.d_ff, w.d), _gen(w, layer, 0, _T_W_GATE, device), device, w.d ** -0.5).to(dt)
+    wg = None
+    if w.act not in NON_GATED:
+        wg = _randn((w.d_ff, w.d), _gen(w, layer, 0, _T_W_GATE, device), device, w.d ** -0.5).to(dt)
     wu = _randn((w.d_ff, w.d), _gen(w, layer, 0, _T_W_UP, device), device, w.d ** -0.5).to(dt)
     wd = _randn((w.d, w.d_ff), _gen(w, layer, 0, _T_W_DOWN, device), device, w.d_ff ** -0.5).to(dt)
     return wg, wu, wd

@@ -75,7 +75,7 @@ class GpuLayer:
 
     def compact(self, e):
         k = e.numel()
-        cs = G.alloc_compact(self.desc, k, dev(), self.tdtype, with_bias=self.t["bg"] is not None)
+        cs = G.alloc_compact(self.desc, k, dev(), self.tdtype, with_bias=self.t["bu"] is not None)
         G.griffin_compact_experts(self.desc, self.weights, e, cs, self.ws)
         return cs
 

@@ -62,10 +62,24 @@ def test_host_validation_rejects_before_any_launch(lib):
     assert f(C.byref(desc), C.byref(w), odd, 4, fake, fake, fake, 1 << 30, None) == G.ERR_ALIGNMENT
     assert f(C.byref(desc), C.byref(w), fake, 4, fake, fake, None, 0, None) == G.ERR_WORKSPACE
     assert f(C.byref(desc), C.byref(w), fake, 4, fake, fake, fake, 1000, None) == G.ERR_WORKSPACE
-    bad = G.make_desc(256, 688, 7, "f32")
+    bad = G.make_desc(256, 688, 8, "f32")   # beyond the last activation code
     assert f(C.byref(bad), C.byref(w), fake, 4, fake, fake, fake, 1 << 30, None) == G.ERR_UNSUPPORTED
     bad = G.make_desc(250, 688, "swiglu", "f32")
     assert f(C.byref(bad), C.byref(w), fake, 4, fake, fake, fake, 1 << 30, None) == G.ERR_ALIGNMENT
+    # a block without a gate (Eq. 2) must not name W_g or b_g, a gated one (Eq. 3) must name W_g
+    relu = G.make_desc(256, 688, "relu", "f32")
+    w_ng = G.FFWeights(None, fake, fake, None, None, None)
+    assert f(C.byref(relu), C.byref(w), fake, 4, fake, fake, fake, 1 << 30, None) == G.ERR_INVALID_ARG
+    assert f(C.byref(relu), C.byref(G.FFWeights(None, fake, fake, fake, None, None)), fake, 4, fake, fake, fake,
+             1 << 30, None) == G.ERR_INVALID_ARG
+    assert f(C.byref(desc), C.byref(w_ng), fake, 4, fake, fake, fake, 1 << 30, None) == G.ERR_INVALID_ARG
+    assert f(C.byref(relu), C.byref(w_ng), fake, 4, fake, fake, fake, 1000, None) == G.ERR_WORKSPACE  # passes the gate check
+    cs_g = G.FFCompact(fake, fake, fake, None, None, 344, 344)
+    cs_ng = G.FFCompact(None, fake, fake, None, None, 344, 344)
+    fd = lib.griffin_ff_decode
+    assert fd(C.byref(relu), 1, C.byref(cs_g), None, fake, fake, fake, 1 << 30, 0, None) == G.ERR_INVALID_ARG
+    assert fd(C.byref(desc), 1, C.byref(cs_ng), None, fake, fake, fake, 1 << 30, 0, None) == G.ERR_INVALID_ARG
+    assert fd(C.byref(relu), 1, C.byref(cs_ng), None, fake, fake, fake, 100, 0, None) == G.ERR_WORKSPACE
     # prompt phase, piece by piece
     fc = lib.griffin_ff_prefill_score_chunk
     assert fc(C.byref(desc), C.byref(w), fake, 4, fake, None, fake, 1, fake, 1 << 30, None) == G.ERR_INVALID_ARG

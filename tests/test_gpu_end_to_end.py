@@ -25,7 +25,7 @@ def run_block(w, layer, keep, n_seq, oracle_seqs, steps):
     assert k == O.k_from_keep_ratio(w.d_ff, keep)
     wg, wu, wd = synth.make_weights(w, layer)
     stack = FFStack(w.d, w.d_ff, w.act, w.dtype, 1, n_seq, w.S, k, dev())
-    wg_d, wu_d, wd_d = wg.to(dev()), wu.to(dev()), wd.to(dev())
+    wg_d, wu_d, wd_d = None if wg is None else wg.to(dev()), wu.to(dev()), wd.to(dev())   # (no W_g without a gate)
     stack.add_block(wg_d, wu_d, wd_d)
     X = [synth.make_prompt(w, layer, q) for q in range(n_seq)]
     XD = torch.stack([synth.make_decode_inputs(w, layer, q) for q in range(n_seq)], 1)  # [T, n_seq, d]
@@ -50,7 +50,7 @@ def run_block(w, layer, keep, n_seq, oracle_seqs, steps):
     E = stack.idx[0].cpu().numpy()
     S_gpu = np64(stack.score[0])
 
-    wg64, wu64, wd64 = np64(wg), np64(wu), np64(wd)
+    wg64, wu64, wd64 = None if wg is None else np64(wg), np64(wu), np64(wd)
     swaps = 0
     for q in oracle_seqs:
         y_ref, z_ref = O.ff_dense(np64(X[q]), wg64, wu64, wd64, w.act)
@@ -84,6 +84,7 @@ SMALL = {
     "gemma_7b": dict(d=384, d_ff=3072, S=128, T=6),
     "llama2_13b": dict(d=640, d_ff=1728, S=160, T=4),
     "mistral_7b": dict(d=512, d_ff=1792, S=200, T=4),
+    "opt_6p7b": dict(d=512, d_ff=2048, S=96, T=6),     # a ReLU block without a gate (Eq. 2)
 }
 
 
@@ -130,6 +131,11 @@ def test_full_size_llama2_7b_blocks():
     w = synth.WORKLOADS["llama2_7b"]
     for layer in (0, w.L // 2, w.L - 1):
         run_block(w, layer, 0.5, 1, [0], _steps(w.T))
+
+
+def test_full_size_opt_6p7b_block_without_a_gate():
+    w = synth.WORKLOADS["opt_6p7b"]
+    run_block(w, 1, 0.5, 1, [0], _steps(w.T))
 
 
 def test_full_size_gemma_7b_block():

@@ -14,9 +14,10 @@ TD = {"f32": torch.float32, "bf16": torch.bfloat16}
 
 def make_layer(d, d_ff, dtype, act="swiglu", bias=False, seed=0, S_max=0, n_seq=1):
     td = TD[dtype]
-    wg, wu = rand((d_ff, d), td, seed + 1, d ** -0.5), rand((d_ff, d), td, seed + 2, d ** -0.5)
+    gated = G.act_is_gated(act)     # a block without a gate (Eq. 2) has no W_g, b_g
+    wg, wu = rand((d_ff, d), td, seed + 1, d ** -0.5) if gated else None, rand((d_ff, d), td, seed + 2, d ** -0.5)
     wd = rand((d, d_ff), td, seed + 3, d_ff ** -0.5)
-    bg = rand((d_ff,), td, seed + 4, 0.3) if bias else None
+    bg = rand((d_ff,), td, seed + 4, 0.3) if bias and gated else None
     bu = rand((d_ff,), td, seed + 5, 0.3) if bias else None
     bd = rand((d,), td, seed + 6, 0.3) if bias else None
     host = dict(wg=wg, wu=wu, wd=wd, bg=bg, bu=bu, bd=bd)

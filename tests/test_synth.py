@@ -11,6 +11,8 @@ def test_workloads_match_the_named_shapes():
     assert (w["gemma_7b"].d, w["gemma_7b"].d_ff, w["gemma_7b"].act) == (3072, 24576, synth.GEGLU_TANH)
     assert (w["llama2_13b"].d, w["llama2_13b"].d_ff, w["llama2_13b"].B) == (5120, 13824, 8)
     assert w["mistral_7b"].keeps == (0.25, 0.5, 0.75, 1.0)
+    assert (w["opt_6p7b"].d, w["opt_6p7b"].d_ff, w["opt_6p7b"].act) == (4096, 16384, synth.RELU)
+    assert synth.make_weights(synth.scaled(w["opt_6p7b"], d=64, d_ff=96), 0)[0] is None   # no W_g without a gate
 
 
 def test_generation_is_reproducible_and_unit_addressable():
