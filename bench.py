@@ -358,15 +358,16 @@ def run_ours(args, w, keep):
         pf_ms = phase_ms[0] / K / (L * B)
         # kernels launched per step: prompt phase = 2 GEMM kernels (+1 when the down projection is
         # K-split, i.e. when its 128x256 tiles number at most half the SMs) + 3 statistic kernels;
-        # one top-k launch for all blocks; 2 compaction kernels; one fused kernel per decode call
+        # one top-k launch for all blocks; 1 compaction kernel; one fused kernel per decode call
         # (two for fp32 storage)
-        split = w.dtype == "bf16" and ((S + 127) // 128) * (w.d // 256 if w.d % 256 == 0 else w.d // 128) <= 74
-        # ... and the finishing kernel of the first GEMM when its last round of 128x128 tiles is cut along K
+        m_tiles = (S + 127) // 128
+        split = w.dtype == "bf16" and m_tiles * (w.d // 256 if w.d % 256 == 0 else w.d // 128) <= 74
+        # ... and the finishing kernel of the first GEMM when its last round of tiles is cut along K
         gated = G.act_is_gated(w.act)
-        g1_tiles = ((S + 127) // 128) * (w.d_ff // 128 if gated else w.d_ff // 256)
+        g1_tiles = m_tiles * (w.d_ff // 128 if gated else w.d_ff // 256)
         cut = (w.dtype == "bf16" and w.d % 128 == 0 and w.d_ff % (128 if gated else 256) == 0 and 148 < g1_tiles <= 4 * 148
                and 0 < g1_tiles % 148 <= 74 and w.d // 64 >= 16)
-        launches = (L * B * (5 + (1 if split else 0) + (1 if cut else 0)) + 1 + (0 if indexed else L * B * 2) +
+        launches = (L * B * (5 + (1 if split else 0) + (1 if cut else 0)) + 1 + (0 if indexed else L * B) +
                     T * L * (1 if w.dtype == "bf16" else 2))
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,

@@ -2,9 +2,12 @@
 // W_1_hat = W_1[E, :], W_2_hat = W_2[:, E], plus the matching bias entries.  Bit copies, so
 // elements are moved as raw 16- or 32-bit words.
 //
-//   rows kernel     16-byte vector copy of the selected rows of W_g and W_1; consecutive
+// One launch per call: the CTAs of a grid are split between the three parts below (columns first:
+// its CTAs carry the most work each), so that no part waits for another's tail or launch.
+//
+//   rows part       16-byte vector copy of the selected rows of W_g and W_1; consecutive
 //                   threads move consecutive vectors of one row (coalesced both ways).
-//   columns kernel  W_2 is [d, d_ff] row-major, so selecting columns is a gather inside
+//   columns part    W_2 is [d, d_ff] row-major, so selecting columns is a gather inside
 //                   each row.  One CTA takes four rows; a thread reads 16 bytes' worth of
 //                   output columns of E once, picks those elements from each of the four
 //                   rows (E is ascending and dense, so neighbouring threads hit
@@ -32,15 +35,15 @@ __device__ __forceinline__ void st_stream(uint4 *p, const uint4 &v) {
 
 // dst_g[jj, :] = src_g[idx[jj], :], dst_u likewise; nv = 16-byte vectors per row.  n_mats = 1: only
 // the first pair of pointers is used (a block without a gate has W_1 alone).
-__global__ void __launch_bounds__(CP_THREADS) compact_rows_kernel(const uint4 *__restrict__ src_g,
-                                                                  const uint4 *__restrict__ src_u,
-                                                                  uint4 *__restrict__ dst_g, uint4 *__restrict__ dst_u,
-                                                                  const int32_t *__restrict__ idx, int k, int d_ff,
-                                                                  int nv, int n_mats, void *ws) {
+// Block `bid` of `nblocks` that share the work.
+__device__ __forceinline__ void compact_rows_part(const uint4 *__restrict__ src_g, const uint4 *__restrict__ src_u,
+                                                  uint4 *__restrict__ dst_g, uint4 *__restrict__ dst_u,
+                                                  const int32_t *__restrict__ idx, int k, int d_ff, int nv, int n_mats,
+                                                  void *ws, int bid, int nblocks) {
     const long long total = (long long)n_mats * k * nv;
-    const long long stride = (long long)gridDim.x * CP_THREADS;
+    const long long stride = (long long)nblocks * CP_THREADS;
     constexpr int U = 4;
-    for (long long v0 = (long long)blockIdx.x * CP_THREADS + threadIdx.x; v0 < total; v0 += stride * U) {
+    for (long long v0 = (long long)bid * CP_THREADS + threadIdx.x; v0 < total; v0 += stride * U) {
         uint4 val[U];
         uint4 *dst[U];
 #pragma unroll
@@ -68,9 +71,10 @@ __global__ void __launch_bounds__(CP_THREADS) compact_rows_kernel(const uint4 *_
 }
 
 template <typename U>
-__global__ void compact_bias_kernel(const U *__restrict__ src_g, const U *__restrict__ src_u, U *__restrict__ dst_g,
-                                    U *__restrict__ dst_u, const int32_t *__restrict__ idx, int k, int d_ff) {
-    const int jj = blockIdx.x * blockDim.x + threadIdx.x;
+__device__ __forceinline__ void compact_bias_part(const U *__restrict__ src_g, const U *__restrict__ src_u,
+                                                  U *__restrict__ dst_g, U *__restrict__ dst_u,
+                                                  const int32_t *__restrict__ idx, int k, int d_ff, int bid) {
+    const int jj = bid * CP_THREADS + threadIdx.x;
     if (jj >= k) return;
     const int e = idx[jj];
     const bool ok = e >= 0 && e < d_ff;
@@ -78,13 +82,13 @@ __global__ void compact_bias_kernel(const U *__restrict__ src_g, const U *__rest
     if (src_u && dst_u) dst_u[jj] = ok ? src_u[e] : (U)0;
 }
 
-// dst[c, jj] = src[c, idx[jj]] for jj < k, 0 for k <= jj < ldk.
+// dst[c, jj] = src[c, idx[jj]] for jj < k, 0 for k <= jj < ldk.  Block `bid` takes rows 4 bid .. 4 bid + 3.
 template <typename U>
-__global__ void __launch_bounds__(CP_THREADS) compact_cols_kernel(const U *__restrict__ src, U *__restrict__ dst,
-                                                                  const int32_t *__restrict__ idx, int d, int d_ff,
-                                                                  int k, int ldk, void *ws) {
+__device__ __forceinline__ void compact_cols_part(const U *__restrict__ src, U *__restrict__ dst,
+                                                  const int32_t *__restrict__ idx, int d, int d_ff, int k, int ldk,
+                                                  void *ws, int bid) {
     constexpr int VEC = 16 / (int)sizeof(U);
-    const int c0 = blockIdx.x * CP_ROWS_PER_CTA;
+    const int c0 = bid * CP_ROWS_PER_CTA;
     const int nvec = ldk / VEC;
     for (int v = threadIdx.x; v < nvec; v += CP_THREADS) {
         int e[VEC];
@@ -116,6 +120,31 @@ __global__ void __launch_bounds__(CP_THREADS) compact_cols_kernel(const U *__res
     }
 }
 
+struct CompactArgs {
+    const void *src_g, *src_u, *src_d, *src_bg, *src_bu;
+    void *dst_g, *dst_u, *dst_d, *dst_bg, *dst_bu;
+    const int32_t *idx;
+    void *ws;
+    int d, d_ff, k, ldk, nv, n_mats;
+    int cols_blocks, rows_blocks;  // CTAs [0, cols_blocks) gather columns, the next rows_blocks copy rows, the rest biases
+};
+
+template <typename U>
+__global__ void __launch_bounds__(CP_THREADS) compact_kernel(const __grid_constant__ CompactArgs a) {
+    const int bid = blockIdx.x;
+    if (bid < a.cols_blocks)
+        compact_cols_part<U>(static_cast<const U *>(a.src_d), static_cast<U *>(a.dst_d), a.idx, a.d, a.d_ff, a.k, a.ldk,
+                             a.ws, bid);
+    else if (bid < a.cols_blocks + a.rows_blocks)
+        compact_rows_part(static_cast<const uint4 *>(a.src_g), static_cast<const uint4 *>(a.src_u),
+                          static_cast<uint4 *>(a.dst_g), static_cast<uint4 *>(a.dst_u), a.idx, a.k, a.d_ff, a.nv, a.n_mats,
+                          a.ws, bid - a.cols_blocks, a.rows_blocks);
+    else
+        compact_bias_part<U>(static_cast<const U *>(a.src_bg), static_cast<const U *>(a.src_bu),
+                             static_cast<U *>(a.dst_bg), static_cast<U *>(a.dst_bu), a.idx, a.k, a.d_ff,
+                             bid - a.cols_blocks - a.rows_blocks);
+}
+
 template <typename U>
 static griffin_status compact_typed(const griffin_ff_desc *desc, const griffin_ff_weights *w, const int32_t *idx,
                                     const griffin_ff_compact *out, void *ws, cudaStream_t stream) {
@@ -127,20 +156,31 @@ static griffin_status compact_typed(const griffin_ff_desc *desc, const griffin_f
     const long long want = ((gated ? 2ll : 1ll) * k * nv + CP_THREADS * 4 - 1) / (CP_THREADS * 4);
     int grid = (int)(want < (long long)sms * 8 ? want : (long long)sms * 8);
     if (grid < 1) grid = 1;
-    compact_rows_kernel<<<grid, CP_THREADS, 0, stream>>>(
-        static_cast<const uint4 *>(gated ? w->w_gate : w->w_up), static_cast<const uint4 *>(w->w_up),
-        static_cast<uint4 *>(gated ? out->w_gate_c : out->w_up_c), static_cast<uint4 *>(out->w_up_c), idx, k, d_ff, nv,
-        gated ? 2 : 1, ws);
+    CompactArgs a = {};
+    a.src_g = gated ? w->w_gate : w->w_up;
+    a.src_u = w->w_up;
+    a.dst_g = gated ? out->w_gate_c : out->w_up_c;
+    a.dst_u = out->w_up_c;
+    a.src_d = w->w_down;
+    a.dst_d = out->w_down_c;
+    a.src_bg = w->b_gate;
+    a.src_bu = w->b_up;
+    a.dst_bg = out->b_gate_c;
+    a.dst_bu = out->b_up_c;
+    a.idx = idx;
+    a.ws = ws;
+    a.d = d;
+    a.d_ff = d_ff;
+    a.k = k;
+    a.ldk = ldk;
+    a.nv = nv;
+    a.n_mats = gated ? 2 : 1;
+    a.cols_blocks = (d + CP_ROWS_PER_CTA - 1) / CP_ROWS_PER_CTA;
+    a.rows_blocks = grid;
+    const bool biases = (w->b_gate && out->b_gate_c) || (w->b_up && out->b_up_c);
+    const int bias_blocks = biases ? (k + CP_THREADS - 1) / CP_THREADS : 0;
+    compact_kernel<U><<<a.cols_blocks + a.rows_blocks + bias_blocks, CP_THREADS, 0, stream>>>(a);
     if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
-    compact_cols_kernel<U><<<(d + CP_ROWS_PER_CTA - 1) / CP_ROWS_PER_CTA, CP_THREADS, 0, stream>>>(
-        static_cast<const U *>(w->w_down), static_cast<U *>(out->w_down_c), idx, d, d_ff, k, ldk, ws);
-    if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
-    if ((w->b_gate && out->b_gate_c) || (w->b_up && out->b_up_c)) {
-        compact_bias_kernel<U><<<(k + 255) / 256, 256, 0, stream>>>(
-            static_cast<const U *>(w->b_gate), static_cast<const U *>(w->b_up), static_cast<U *>(out->b_gate_c),
-            static_cast<U *>(out->b_up_c), idx, k, d_ff);
-        if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
-    }
     return GRIFFIN_OK;
 }
 
