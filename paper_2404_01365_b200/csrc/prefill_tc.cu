@@ -5,16 +5,20 @@
 //   kernel<KIND = 2> : the same for a block without a gate (Eq. 2): Z = sigma(X W_1^T + b_1)
 //   kernel<KIND = 0> : Y = Z W_2^T + b_2
 //
-// One persistent CTA per SM, 192 threads in three roles:
+// One persistent CTA per SM, 320 threads in three roles:
 //   warp 0      TMA producer: cp.async.bulk.tensor (2-D tiles, 128-byte swizzle, no multicast)
 //               of a 128 x 64 tile of the left operand and a BN x 64 tile of the weights
 //               into a ring of shared-memory stages;
 //   warp 1      MMA issuer: one elected thread issues tcgen05.mma (M = 128, N = BN, K = 16,
 //               operands from shared memory through matrix descriptors, accumulator in TMEM),
 //               releases each stage with tcgen05.commit; it also owns the TMEM allocation;
-//   warps 2-5   epilogue: tcgen05.ld of the accumulator (one row per thread), activation and
-//               gating (or bias), stores.  TMEM holds two accumulator stages, so the epilogue
-//               of one tile runs under the MMAs of the next.
+//   warps 2-9   epilogue: tcgen05.ld of the accumulator (one row per thread), activation and
+//               gating (or bias), stores.  A warp may read the TMEM lanes 32 (w mod 4) .. + 31, so
+//               warps w and w + 4 share a quarter of the rows and take half of the columns each
+//               (measured: with four warps the epilogue of a tile took 23 us of dependent
+//               latencies, one warp per scheduler, and the last one of a CTA is never hidden).
+//               TMEM holds two accumulator stages, so the epilogue of one tile runs under the
+//               MMAs of the next.
 // For DUAL the gate and up tiles of the same 128 neurons are loaded one behind the other, so
 // that a single N = 256 MMA against the shared X tile fills columns 0..127 with the gate
 // and 128..255 with the up pre-activations: the epilogue thread that owns a row finds both.
@@ -31,7 +35,8 @@ namespace griffin {
 
 constexpr int TC_BM = 128;        // rows (tokens) per tile
 constexpr int TC_BK = 64;         // K per stage: 64 bf16 = one 128-byte swizzle row
-constexpr int TC_THREADS = 192;
+constexpr int TC_EPI_WARPS = 8;   // two per TMEM lane quarter
+constexpr int TC_THREADS = 64 + 32 * TC_EPI_WARPS;
 #ifndef GRIFFIN_TC_STAGES
 #define GRIFFIN_TC_STAGES 4
 #endif
@@ -45,7 +50,7 @@ struct TcParams {
     const __nv_bfloat16 *bias0, *bias1;  // DUAL: b_gate, b_up; otherwise b_down, unused (may be null)
     __nv_bfloat16 *out;                  // Z or Y, [S, n_total]
     float *zf;                           // DUAL: Z in fp32, [S, n_total]
-    float *rowsq;                        // DUAL: [S, n_tiles] partial sums of squares of the fp32 rows
+    float *rowsq;                        // DUAL: [S, 2 n_tiles] partial sums of squares of the fp32 rows (two column halves per tile)
     int splits;                          // K splits (1 unless the plain GEMM has too few tiles)
     float *part;                         // splits > 1: fp32 partial outputs [splits, S, n_total]
     int act;
@@ -128,7 +133,7 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&s.acc_full[i], 1);
-            mbar_init(&s.acc_empty[i], 4);  // one arrival per epilogue warp
+            mbar_init(&s.acc_empty[i], TC_EPI_WARPS);  // one arrival per epilogue warp
         }
         *s.abort = 0;
         mbar_fence_init();
@@ -207,15 +212,17 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
             }
         }
     } else {
-        // ---------------- epilogue (warps 2..5) ----------------
+        // ---------------- epilogue (warps 2..9) ----------------
         const int wq = warp & 3;                 // the TMEM lane quarter this warp may read
+        const int half = (warp - 2) >> 2;        // which half of the tile's columns this warp takes
         const int row_in_tile = wq * 32 + lane;  // one output row per thread
         uint32_t tcount = 0;
         for (int tile = blockIdx.x; tile < n_tiles_total; tile += gridDim.x, ++tcount) {
             const TcItem ti = tc_item(p, tile, kb_total);
             const int m = ti.m, n = ti.n, sp = ti.sp;
             const int acc = tcount & 1;
-            if (!wait_or_abort(&s.acc_full[acc], (tcount >> 1) & 1, s.abort, p.ws, 23)) break;
+            // (256 threads wait here for most of a tile's main loop: they sleep between polls)
+            if (!wait_or_abort_relaxed(&s.acc_full[acc], (tcount >> 1) & 1, s.abort, p.ws, 23)) break;
             tc_fence_after_sync();
             const int row = m * TC_BM + row_in_tile;
             const bool live = row < p.S;
@@ -225,7 +232,7 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
                 // kernel adds the parts and does what the epilogue below does
                 float *dst = p.tail_part + ((size_t)ti.part * TC_BM + row_in_tile) * 256;
 #pragma unroll 1
-                for (int c = 0; c < 256; c += 32) {
+                for (int c = half * 128; c < half * 128 + 128; c += 32) {
                     float a[32];
                     tmem_ld32(taddr + c, a);
 #pragma unroll
@@ -236,7 +243,7 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
                 // no gate: every one of the 256 accumulator columns is a neuron, Z = sigma(acc + b_1)
                 float sq = 0.f;
 #pragma unroll 1
-                for (int c = 0; c < 256; c += 32) {
+                for (int c = half * 128; c < half * 128 + 128; c += 32) {
                     float u[32];
                     tmem_ld32(taddr + c, u);
                     const int col = n * 256 + c;
@@ -263,14 +270,13 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
                         for (int v = 0; v < 8; ++v) fo[v] = make_float4(u[4 * v], u[4 * v + 1], u[4 * v + 2], u[4 * v + 3]);
                     }
                 }
-                if (live) p.rowsq[(size_t)row * p.n_tiles + n] = sq;
+                if (live) p.rowsq[(size_t)row * (2 * p.n_tiles) + 2 * n + half] = sq;
             } else if (DUAL) {
                 float sq = 0.f;
 #pragma unroll 1
-                for (int c = 0; c < 128; c += 32) {
+                for (int c = half * 64; c < half * 64 + 64; c += 32) {
                     float g[32], u[32];
-                    tmem_ld32(taddr + c, g);
-                    tmem_ld32(taddr + 128 + c, u);
+                    tmem_ld32x2(taddr + c, taddr + 128 + c, g, u);
                     const int col = n * 128 + c;
                     uint32_t packed[16];
 #pragma unroll
@@ -296,10 +302,10 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
                         for (int v = 0; v < 8; ++v) fo[v] = make_float4(g[4 * v], g[4 * v + 1], g[4 * v + 2], g[4 * v + 3]);
                     }
                 }
-                if (live) p.rowsq[(size_t)row * p.n_tiles + n] = sq;
+                if (live) p.rowsq[(size_t)row * (2 * p.n_tiles) + 2 * n + half] = sq;
             } else {
 #pragma unroll 1
-                for (int c = 0; c < BN; c += 32) {
+                for (int c = half * (BN / 2); c < half * (BN / 2) + BN / 2; c += 32) {
                     float a[32];
                     tmem_ld32(taddr + c, a);
                     const int col = n * BN + c;
@@ -404,7 +410,7 @@ __global__ void __launch_bounds__(128) dual_tail_finish_kernel(TcParams p) {
         *reinterpret_cast<float4 *>(p.zf + (size_t)row * p.n_total + col) = make_float4(z[0], z[1], z[2], z[3]);
     }
     sq = warp_sum(sq);
-    if (lane == 0 && row < p.S) p.rowsq[(size_t)row * p.n_tiles + n] = sq;
+    if (lane < 2 && row < p.S) p.rowsq[(size_t)row * (2 * p.n_tiles) + 2 * n + lane] = lane == 0 ? sq : 0.f;
 }
 
 // y = bf16(sum over K splits of part + bias), four columns per thread, splits added in order.
@@ -528,7 +534,7 @@ griffin_status launch_prefill_tc(const griffin_ff_desc *desc, const griffin_ff_w
     p.splits = 1;
     gemm1_tail_plan(S, d, p.n_tiles, &p.tail_first, &p.tail_ks);
     p.tail_part = ypart;  // (the down projection's partials use the same scratch, later)
-    *n_col_tiles = p.n_tiles;
+    *n_col_tiles = 2 * p.n_tiles;  // partial row sums per token: one per tile and column half
     griffin_status st = gated ? launch_tc<TC_GATED, 128>(mx, mg, mu, p, sms, stream)
                               : launch_tc<TC_WIDE, 128>(mx, mg, mu, p, sms, stream);
     if (st == GRIFFIN_OK && p.tail_ks > 1) {
