@@ -94,13 +94,53 @@ __device__ __forceinline__ TcItem tc_item(const TcParams &p, int item, int kb_to
     return t;
 }
 
+// Output staging of the epilogue warps.  A thread of an epilogue warp holds one ROW of the tile, so a
+// store straight from its registers scatters every instruction over 32 rows, 16 bytes each; those
+// requests queue behind the TMA loads on the SM's way to L2 and made the epilogue of a tile take
+// 18-23 us.  Instead the warp passes its 32 rows, 64 bytes of each at a time, through a small buffer
+// of its own in shared memory and writes them back so that an instruction covers 8 rows x 64
+// contiguous bytes.
+constexpr int TC_STG_PITCH = 80;                  // 64 data bytes + 16 of padding per staged row
+constexpr int TC_STG_BYTES = 32 * TC_STG_PITCH;   // per epilogue warp
+// v: this thread's 64 bytes of its row; g: global address of the block's first row at the wanted
+// column; rows at and beyond rows_live are not written.
+__device__ __forceinline__ void store_rows64(uint8_t *stg, const uint4 (&v)[4], void *g, size_t row_pitch_bytes,
+                                             int rows_live, int lane) {
+    uint4 *mine = reinterpret_cast<uint4 *>(stg + lane * TC_STG_PITCH);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) mine[i] = v[i];
+    __syncwarp();
+    const int piece = lane & 3, r0 = lane >> 2;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int r = r0 + 8 * j;
+        const uint4 t = *reinterpret_cast<const uint4 *>(stg + r * TC_STG_PITCH + piece * 16);
+        if (r < rows_live) *reinterpret_cast<uint4 *>(static_cast<uint8_t *>(g) + (size_t)r * row_pitch_bytes + piece * 16) = t;
+    }
+    __syncwarp();
+}
+// 32 fp32 values of this thread's row (128 bytes) as two such passes.
+__device__ __forceinline__ void store_rows_f32x32(uint8_t *stg, const float (&a)[32], float *g, size_t row_pitch_bytes,
+                                                  int rows_live, int lane) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        uint4 v[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            v[i] = make_uint4(__float_as_uint(a[16 * h + 4 * i]), __float_as_uint(a[16 * h + 4 * i + 1]),
+                              __float_as_uint(a[16 * h + 4 * i + 2]), __float_as_uint(a[16 * h + 4 * i + 3]));
+        store_rows64(stg, v, g + 16 * h, row_pitch_bytes, rows_live, lane);
+    }
+}
+
 struct TcSmem {
     uint8_t *stages;
     uint64_t *full, *empty, *acc_full, *acc_empty;
     uint32_t *tmem_slot;
+    uint8_t *stg;  // TC_EPI_WARPS staging buffers
     volatile int *abort;
 };
-constexpr size_t TC_TAIL_BYTES = (2 * TC_STAGES + 4) * sizeof(uint64_t) + 16;
+constexpr size_t TC_TAIL_BYTES = (2 * TC_STAGES + 4) * sizeof(uint64_t) + 16 + TC_EPI_WARPS * TC_STG_BYTES;
 
 constexpr int TC_PLAIN = 0, TC_GATED = 1, TC_WIDE = 2;
 template <int KIND, int BN>
@@ -124,6 +164,7 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
     s.acc_empty = s.acc_full + 2;
     s.tmem_slot = reinterpret_cast<uint32_t *>(s.acc_empty + 2);
     s.abort = reinterpret_cast<volatile int *>(s.tmem_slot + 1);
+    s.stg = reinterpret_cast<uint8_t *>(s.full) + (2 * TC_STAGES + 4) * sizeof(uint64_t) + 16;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
@@ -216,6 +257,7 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
         const int wq = warp & 3;                 // the TMEM lane quarter this warp may read
         const int half = (warp - 2) >> 2;        // which half of the tile's columns this warp takes
         const int row_in_tile = wq * 32 + lane;  // one output row per thread
+        uint8_t *const stg = s.stg + (warp - 2) * TC_STG_BYTES;
         uint32_t tcount = 0;
         for (int tile = blockIdx.x; tile < n_tiles_total; tile += gridDim.x, ++tcount) {
             const TcItem ti = tc_item(p, tile, kb_total);
@@ -226,18 +268,18 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
             tc_fence_after_sync();
             const int row = m * TC_BM + row_in_tile;
             const bool live = row < p.S;
+            const int row0 = m * TC_BM + wq * 32;  // first row of this warp's block of 32
+            const int rows_live = p.S - row0;      // rows of the block that exist (may be <= 0 or > 32)
             const uint32_t taddr = tmem_base + ((uint32_t)(wq * 32) << 16) + (uint32_t)(acc * NT);
             if (DUAL && ti.part >= 0) {
                 // a part of a cut tile: the raw accumulators leave in fp32 (gate | up); the finishing
                 // kernel adds the parts and does what the epilogue below does
-                float *dst = p.tail_part + ((size_t)ti.part * TC_BM + row_in_tile) * 256;
+                float *dst = p.tail_part + ((size_t)ti.part * TC_BM + wq * 32) * 256;
 #pragma unroll 1
                 for (int c = half * 128; c < half * 128 + 128; c += 32) {
                     float a[32];
                     tmem_ld32(taddr + c, a);
-#pragma unroll
-                    for (int v = 0; v < 8; ++v)
-                        reinterpret_cast<float4 *>(dst + c)[v] = make_float4(a[4 * v], a[4 * v + 1], a[4 * v + 2], a[4 * v + 3]);
+                    store_rows_f32x32(stg, a, dst + c, 256 * sizeof(float), 32, lane);
                 }
             } else if (KIND == TC_WIDE) {
                 // no gate: every one of the 256 accumulator columns is a neuron, Z = sigma(acc + b_1)
@@ -260,14 +302,13 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
                         const __nv_bfloat162 h = __floats2bfloat162_rn(z0, z1);
                         packed[i >> 1] = *reinterpret_cast<const uint32_t *>(&h);
                     }
-                    if (live) {
-                        uint4 *zo = reinterpret_cast<uint4 *>(p.out + (size_t)row * p.n_total + col);
-                        float4 *fo = reinterpret_cast<float4 *>(p.zf + (size_t)row * p.n_total + col);
+                    {
+                        uint4 pk[4];
 #pragma unroll
                         for (int v = 0; v < 4; ++v)
-                            zo[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
-#pragma unroll
-                        for (int v = 0; v < 8; ++v) fo[v] = make_float4(u[4 * v], u[4 * v + 1], u[4 * v + 2], u[4 * v + 3]);
+                            pk[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+                        store_rows64(stg, pk, p.out + (size_t)row0 * p.n_total + col, (size_t)p.n_total * 2, rows_live, lane);
+                        store_rows_f32x32(stg, u, p.zf + (size_t)row0 * p.n_total + col, (size_t)p.n_total * 4, rows_live, lane);
                     }
                 }
                 if (live) p.rowsq[(size_t)row * (2 * p.n_tiles) + 2 * n + half] = sq;
@@ -292,14 +333,13 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
                         const __nv_bfloat162 h = __floats2bfloat162_rn(z0, z1);
                         packed[i >> 1] = *reinterpret_cast<const uint32_t *>(&h);
                     }
-                    if (live) {
-                        uint4 *zo = reinterpret_cast<uint4 *>(p.out + (size_t)row * p.n_total + col);
-                        float4 *fo = reinterpret_cast<float4 *>(p.zf + (size_t)row * p.n_total + col);
+                    {
+                        uint4 pk[4];
 #pragma unroll
                         for (int v = 0; v < 4; ++v)
-                            zo[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
-#pragma unroll
-                        for (int v = 0; v < 8; ++v) fo[v] = make_float4(g[4 * v], g[4 * v + 1], g[4 * v + 2], g[4 * v + 3]);
+                            pk[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+                        store_rows64(stg, pk, p.out + (size_t)row0 * p.n_total + col, (size_t)p.n_total * 2, rows_live, lane);
+                        store_rows_f32x32(stg, g, p.zf + (size_t)row0 * p.n_total + col, (size_t)p.n_total * 4, rows_live, lane);
                     }
                 }
                 if (live) p.rowsq[(size_t)row * (2 * p.n_tiles) + 2 * n + half] = sq;
@@ -310,11 +350,8 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
                     tmem_ld32(taddr + c, a);
                     const int col = n * BN + c;
                     if (p.splits > 1) {  // partial sums leave in fp32; bias and rounding happen in the reduction
-                        if (live) {
-                            float4 *po = reinterpret_cast<float4 *>(p.part + ((size_t)sp * p.S + row) * p.n_total + col);
-#pragma unroll
-                            for (int v = 0; v < 8; ++v) po[v] = make_float4(a[4 * v], a[4 * v + 1], a[4 * v + 2], a[4 * v + 3]);
-                        }
+                        store_rows_f32x32(stg, a, p.part + ((size_t)sp * p.S + row0) * p.n_total + col,
+                                          (size_t)p.n_total * 4, rows_live, lane);
                         continue;
                     }
                     uint32_t packed[16];
@@ -325,11 +362,12 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
                         const __nv_bfloat162 h = __floats2bfloat162_rn(y0, y1);
                         packed[i >> 1] = *reinterpret_cast<const uint32_t *>(&h);
                     }
-                    if (live) {
-                        uint4 *yo = reinterpret_cast<uint4 *>(p.out + (size_t)row * p.n_total + col);
+                    {
+                        uint4 pk[4];
 #pragma unroll
                         for (int v = 0; v < 4; ++v)
-                            yo[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+                            pk[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+                        store_rows64(stg, pk, p.out + (size_t)row0 * p.n_total + col, (size_t)p.n_total * 2, rows_live, lane);
                     }
                 }
             }
