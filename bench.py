@@ -69,6 +69,26 @@ def measured_tensor_peaks():
         return 1590.0, 1400.0
 
 
+def down_projection_splits(S, d, d_ff):
+    """How many K splits the library's down projection takes for this shape (its own rule, restated here
+    only to count the launches of a step: with a split there is one more kernel per prompt)."""
+    bn = 256 if d % 256 == 0 else 128
+    tiles = ((S + 127) // 128) * (d // bn)
+    tile_us = 2.0 * 128 * bn * d_ff / 10e12 * 1e6
+    cost1 = best_cost = None
+    best = 1
+    for sp in range(1, 5):
+        rounds = (tiles * sp + 147) // 148
+        cost = rounds * tile_us / sp
+        if sp > 1:
+            cost += 2.0 * sp * S * d * 4.0 / 4e12 * 1e6 + 3.0
+        if sp == 1:
+            cost1 = best_cost = cost
+        elif cost < 0.9 * cost1 and cost < best_cost:
+            best_cost, best = cost, sp
+    return best
+
+
 def recorded_traffic():
     """DRAM bytes per decode call from the committed ncu summary, if the kernel source is
     unchanged since that capture; otherwise None."""
@@ -361,7 +381,7 @@ def run_ours(args, w, keep):
         # one top-k launch for all blocks; 1 compaction kernel; one fused kernel per decode call
         # (two for fp32 storage)
         m_tiles = (S + 127) // 128
-        split = w.dtype == "bf16" and m_tiles * (w.d // 256 if w.d % 256 == 0 else w.d // 128) <= 74
+        split = w.dtype == "bf16" and down_projection_splits(S, w.d, w.d_ff) > 1
         # ... and the finishing kernel of the first GEMM when its last round of tiles is cut along K
         gated = G.act_is_gated(w.act)
         g1_tiles = m_tiles * (w.d_ff // 128 if gated else w.d_ff // 256)

@@ -48,7 +48,7 @@ PrefillScratch prefill_scratch(const griffin_ff_desc *desc, int S) {
     ps.ypart_off = off;  // fp32 partial outputs of a K-split down projection (bf16 tensor-core path)
     if (desc->dtype != GRIFFIN_DT_F32) {
         int bn = 0, splits = 1;
-        gemm2_plan(S, desc->d, &bn, &splits);
+        gemm2_plan(S, desc->d, desc->d_ff, &bn, &splits);
         size_t need = splits > 1 ? (size_t)splits * S * desc->d * sizeof(float) : 0;
         const size_t tail = gemm1_tail_bytes(S, desc->d, gemm1_col_tiles(desc));  // (used up before the down projection starts)
         if (tail > need) need = tail;

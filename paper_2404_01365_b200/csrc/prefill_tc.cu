@@ -501,12 +501,28 @@ size_t gemm1_tail_bytes(int S, int d, int n_col_tiles) {
     return (size_t)(tiles - first) * ks * TC_BM * 256 * sizeof(float);
 }
 
-void gemm2_plan(int S, int d, int *bn, int *splits) {
+void gemm2_plan(int S, int d, int d_ff, int *bn, int *splits) {
     const int m_tiles = (S + TC_BM - 1) / TC_BM;
     *bn = d % 256 == 0 ? 256 : 128;
     const int tiles = m_tiles * (d / *bn);
-    int sp = TC_TARGET_CTAS / (tiles > 0 ? tiles : 1);
-    *splits = sp < 1 ? 1 : (sp > 4 ? 4 : sp);
+    // Uniform K splits, 1..4, by a small cost model in microseconds: the rounds that tiles x splits work
+    // items need on one CTA per SM, at the measured pace of a long tile (about 10 TFLOP/s per SM), plus,
+    // when there is a split, the fp32 partial sums written and read back (about 4 TB/s) and the launch of
+    // the kernel that adds them.  A split must win by a tenth to be taken.
+    const double tile_us = 2.0 * TC_BM * (double)*bn * (double)d_ff / 10e12 * 1e6;
+    double cost1 = 0.0, best_cost = 0.0;
+    int best = 1;
+    for (int sp = 1; sp <= 4; ++sp) {
+        const int rounds = (tiles * sp + TC_TARGET_CTAS - 1) / TC_TARGET_CTAS;
+        double cost = rounds * tile_us / sp;
+        if (sp > 1) cost += 2.0 * sp * (double)S * (double)d * 4.0 / 4e12 * 1e6 + 3.0;
+        if (sp == 1) cost1 = best_cost = cost;
+        else if (cost < 0.9 * cost1 && cost < best_cost) {
+            best_cost = cost;
+            best = sp;
+        }
+    }
+    *splits = best;
 }
 
 // Row-major bf16 matrix [rows, cols] (cols contiguous); box = box_rows x 64 columns, 128-byte swizzle,
@@ -584,7 +600,7 @@ griffin_status launch_prefill_tc(const griffin_ff_desc *desc, const griffin_ff_w
 
     // Y = Z W_2^T + b_2
     int bn = 128, splits = 1;
-    gemm2_plan(S, d, &bn, &splits);
+    gemm2_plan(S, d, d_ff, &bn, &splits);
     CUtensorMap mz, md;
     if (!make_map(&mz, z, S, d_ff, TC_BM) || !make_map(&md, w->w_down, d, d_ff, bn)) return GRIFFIN_ERR_CUDA;
     TcParams q = {};

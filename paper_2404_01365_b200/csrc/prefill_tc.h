@@ -9,9 +9,10 @@
 namespace griffin {
 
 // Tiling of the down projection Y = Z W_2^T for S tokens: tile width (128 or 256 outputs) and the
-// number of K splits (1..4; more than one when whole tiles would leave most SMs idle).  Pure
-// arithmetic on the shape, so that workspace sizing and launch agree.
-void gemm2_plan(int S, int d, int *bn, int *splits);
+// number of K splits (1..4; more than one when that fills the SMs better than whole tiles and the
+// fp32 partial sums cost less than it saves).  Pure arithmetic on the shape, so that workspace sizing
+// and launch agree.
+void gemm2_plan(int S, int d, int d_ff, int *bn, int *splits);
 
 // Column tiles of the first GEMM: 128 neurons each with a gate (gate | up side by side in the
 // accumulator), 256 without.
