@@ -89,6 +89,16 @@ def down_projection_splits(S, d, d_ff):
     return best
 
 
+def down_projection_tail_cut(S, d, d_ff):
+    """Whether the library cuts the last round of the down projection's tiles along K (one more kernel per
+    prompt); its rule, restated to count launches."""
+    if d % 256 != 0 or down_projection_splits(S, d, d_ff) != 1:
+        return False
+    tiles = ((S + 127) // 128) * (d // 256)
+    rem = tiles % 148
+    return tiles > 148 and 0 < rem and 2 * rem <= 148 and d_ff // 64 >= 16
+
+
 def recorded_traffic():
     """DRAM bytes per decode call from the committed ncu summary, if the kernel source is
     unchanged since that capture; otherwise None."""
@@ -387,7 +397,8 @@ def run_ours(args, w, keep):
         g1_tiles = m_tiles * (w.d_ff // 128 if gated else w.d_ff // 256)
         cut = (w.dtype == "bf16" and w.d % 128 == 0 and w.d_ff % (128 if gated else 256) == 0 and 148 < g1_tiles <= 4 * 148
                and 0 < g1_tiles % 148 <= 74 and w.d // 64 >= 16)
-        launches = (L * B * (5 + (1 if split else 0) + (1 if cut else 0)) + 1 + (0 if indexed else L * B) +
+        cut2 = w.dtype == "bf16" and w.d % 128 == 0 and w.d_ff % (128 if gated else 256) == 0 and down_projection_tail_cut(S, w.d, w.d_ff)
+        launches = (L * B * (5 + (1 if split else 0) + (1 if cut else 0) + (1 if cut2 else 0)) + 1 + (0 if indexed else L * B) +
                     T * L * (1 if w.dtype == "bf16" else 2))
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,

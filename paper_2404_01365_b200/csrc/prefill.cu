@@ -52,6 +52,8 @@ PrefillScratch prefill_scratch(const griffin_ff_desc *desc, int S) {
         size_t need = splits > 1 ? (size_t)splits * S * desc->d * sizeof(float) : 0;
         const size_t tail = gemm1_tail_bytes(S, desc->d, gemm1_col_tiles(desc));  // (used up before the down projection starts)
         if (tail > need) need = tail;
+        const size_t tail2 = gemm2_tail_bytes(S, desc->d, desc->d_ff);
+        if (tail2 > need) need = tail2;
         if (need > 0) off = align_up(off + need, 256);
     }
     ps.total = off;

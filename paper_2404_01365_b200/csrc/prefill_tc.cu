@@ -55,8 +55,8 @@ struct TcParams {
     float *part;                         // splits > 1: fp32 partial outputs [splits, S, n_total]
     int act;
     void *ws;
-    // DUAL only: tiles from tail_first on are cut along K into tail_ks parts (tail_ks = 1: none is),
-    // whose raw accumulators (gate | up, fp32) go to tail_part [part][128 rows][256 columns]
+    // Tiles 256 columns wide only: tiles from tail_first on are cut along K into tail_ks parts (tail_ks = 1:
+    // none is), whose raw accumulators (fp32; gate | up in the first GEMM) go to tail_part [part][128 rows][256 columns]
     int tail_first, tail_ks;
     float *tail_part;
     int gated;  // first GEMM: 1 = gate | up tiles of 128 neurons, 0 = 256 neurons of W_1 (no gate)
@@ -271,7 +271,7 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
             const int row0 = m * TC_BM + wq * 32;  // first row of this warp's block of 32
             const int rows_live = p.S - row0;      // rows of the block that exist (may be <= 0 or > 32)
             const uint32_t taddr = tmem_base + ((uint32_t)(wq * 32) << 16) + (uint32_t)(acc * NT);
-            if (DUAL && ti.part >= 0) {
+            if ((DUAL || BN == 256) && ti.part >= 0) {
                 // a part of a cut tile: the raw accumulators leave in fp32 (gate | up); the finishing
                 // kernel adds the parts and does what the epilogue below does
                 float *dst = p.tail_part + ((size_t)ti.part * TC_BM + wq * 32) * 256;
@@ -451,6 +451,42 @@ __global__ void __launch_bounds__(128) dual_tail_finish_kernel(TcParams p) {
     if (lane < 2 && row < p.S) p.rowsq[(size_t)row * (2 * p.n_tiles) + 2 * n + lane] = lane == 0 ? sq : 0.f;
 }
 
+// Finishes the cut tiles of the down projection: one warp per (cut tile, row), eight outputs per lane.
+// The parts are added in order, then b_2, then rounded to bf16.
+__global__ void __launch_bounds__(128) plain_tail_finish_kernel(TcParams p) {
+    const int w = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    const int tile = p.tail_first + w / TC_BM, r = w % TC_BM, c = lane * 8;
+    const int m = tile % p.m_tiles, n = tile / p.m_tiles;
+    const int row = m * TC_BM + r, col = n * 256 + c;
+    float4 a[4][2];
+#pragma unroll
+    for (int sp = 0; sp < 4; ++sp) {  // at most four parts; all loads in flight together
+        a[sp][0] = a[sp][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (sp < p.tail_ks) {
+            const float4 *src = reinterpret_cast<const float4 *>(
+                p.tail_part + ((size_t)((tile - p.tail_first) * p.tail_ks + sp) * TC_BM + r) * 256 + c);
+            a[sp][0] = __ldcs(src);
+            a[sp][1] = __ldcs(src + 1);
+        }
+    }
+    float v[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int sp = 0; sp < 4; ++sp) {  // added in order (absent parts are zeros)
+        v[0] += a[sp][0].x; v[1] += a[sp][0].y; v[2] += a[sp][0].z; v[3] += a[sp][0].w;
+        v[4] += a[sp][1].x; v[5] += a[sp][1].y; v[6] += a[sp][1].z; v[7] += a[sp][1].w;
+    }
+    if (row >= p.S) return;
+    uint32_t packed[4];
+#pragma unroll
+    for (int i = 0; i < 8; i += 2) {
+        float y0 = v[i], y1 = v[i + 1];
+        if (p.bias0) { y0 += __bfloat162float(p.bias0[col + i]); y1 += __bfloat162float(p.bias0[col + i + 1]); }
+        const __nv_bfloat162 h = __floats2bfloat162_rn(y0, y1);
+        packed[i >> 1] = *reinterpret_cast<const uint32_t *>(&h);
+    }
+    *reinterpret_cast<uint4 *>(p.out + (size_t)row * p.n_total + col) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+}
+
 // y = bf16(sum over K splits of part + bias), four columns per thread, splits added in order.
 __global__ void splitk_reduce_kernel(const float *__restrict__ part, const __nv_bfloat16 *__restrict__ bias,
                                      __nv_bfloat16 *__restrict__ y, int splits, size_t n_elems, int n_total) {
@@ -523,6 +559,30 @@ void gemm2_plan(int S, int d, int d_ff, int *bn, int *splits) {
         }
     }
     *splits = best;
+}
+
+// The same cut for the down projection when it runs in whole tiles 256 outputs wide: where the last
+// round of tiles would leave at least half of the SMs idle, its tiles are cut along K into 2..4 parts.
+void gemm2_tail_plan(int S, int d, int d_ff, int *tail_first, int *ks) {
+    int bn = 0, splits = 1;
+    gemm2_plan(S, d, d_ff, &bn, &splits);
+    const int tiles = ((S + TC_BM - 1) / TC_BM) * (d / (bn > 0 ? bn : 1));
+    const int rem = tiles % TC_TARGET_CTAS;
+    *tail_first = tiles;
+    *ks = 1;
+    if (bn == 256 && splits == 1 && tiles > TC_TARGET_CTAS && rem > 0 && 2 * rem <= TC_TARGET_CTAS && d_ff / TC_BK >= 16) {
+        const int k = TC_TARGET_CTAS / rem;
+        *ks = k > 4 ? 4 : k;
+        *tail_first = tiles - rem;
+    }
+}
+
+size_t gemm2_tail_bytes(int S, int d, int d_ff) {
+    int first = 0, ks = 1;
+    gemm2_tail_plan(S, d, d_ff, &first, &ks);
+    if (ks <= 1) return 0;
+    const int tiles = ((S + TC_BM - 1) / TC_BM) * (d / 256);
+    return (size_t)(tiles - first) * ks * TC_BM * 256 * sizeof(float);
 }
 
 // Row-major bf16 matrix [rows, cols] (cols contiguous); box = box_rows x 64 columns, 128-byte swizzle,
@@ -616,8 +676,15 @@ griffin_status launch_prefill_tc(const griffin_ff_desc *desc, const griffin_ff_w
     q.splits = splits;
     q.part = splits > 1 ? ypart : nullptr;
     q.tail_ks = 1;
+    gemm2_tail_plan(S, d, d_ff, &q.tail_first, &q.tail_ks);
+    q.tail_part = ypart;
+    if (q.tail_ks > 1) q.bias0 = static_cast<const __nv_bfloat16 *>(w->b_down);
     st = bn == 256 ? launch_tc<TC_PLAIN, 256>(mz, md, md, q, sms, stream)
                    : launch_tc<TC_PLAIN, 128>(mz, md, md, q, sms, stream);
+    if (st == GRIFFIN_OK && q.tail_ks > 1) {
+        plain_tail_finish_kernel<<<(q.m_tiles * q.n_tiles - q.tail_first) * (TC_BM / 4), 128, 0, stream>>>(q);
+        if (cudaGetLastError() != cudaSuccess) st = GRIFFIN_ERR_CUDA;
+    }
     if (st != GRIFFIN_OK || splits == 1) return st;
     const size_t n_elems = (size_t)S * d;
     splitk_reduce_kernel<<<(unsigned)((n_elems / 4 + 255) / 256), 256, 0, stream>>>(

@@ -26,6 +26,10 @@ void gemm1_tail_plan(int S, int d, int n_col_tiles, int *tail_first, int *ks);
 // Bytes of fp32 scratch that the parts of the cut tiles need (0 when none is cut).
 size_t gemm1_tail_bytes(int S, int d, int n_col_tiles);
 
+// The same cut for the last round of the down projection's tiles (whole tiles 256 outputs wide only).
+void gemm2_tail_plan(int S, int d, int d_ff, int *tail_first, int *ks);
+size_t gemm2_tail_bytes(int S, int d, int d_ff);
+
 // Whether the tensor-core kernels take this shape (bf16, d and d_ff multiples of 64, ...).
 bool prefill_tc_supported(const griffin_ff_desc *desc, int S);
 

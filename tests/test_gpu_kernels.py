@@ -408,6 +408,25 @@ def test_prefill_with_a_cut_last_round_of_tiles(S, d, d_ff):
     assert np.array_equal(np64(s2), s)
 
 
+def test_prefill_down_projection_with_a_cut_last_round_of_tiles():
+    """160 tiles of the second GEMM (5 row blocks x 32 blocks of 256 outputs) on 148 SMs: the last 12 are
+    cut along K into four parts whose partial accumulators meet in a finishing kernel."""
+    S, d, d_ff = 640, 8192, 1024
+    L, host = make_layer(d, d_ff, "bf16", act="swiglu", bias=True, seed=S + d_ff, S_max=S)
+    x = rand((S, d), torch.bfloat16, 17) + rand((1, d), torch.bfloat16, 18, 4.0 / d ** 0.5)
+    y, s = L.prefill(x)
+    ref_y, ref_z = O.ff_dense(np64(x), h64(host, "wg"), h64(host, "wu"), h64(host, "wd"), "swiglu",
+                              h64(host, "bg"), h64(host, "bu"), h64(host, "bd"))
+    assert L.status() == G.OK
+    y = np64(y)
+    assert rel_l2(y, ref_y) < TOL_OUT["bf16"]
+    for r0, c0 in ((0, 0), (512, 7936), (639, 8191 - 255)):      # whole tiles and cut ones, corner by corner
+        blk = (slice(r0, min(S, r0 + 128)), slice(c0, c0 + 256))
+        assert rel_l2(y[blk], ref_y[blk]) < TOL_OUT["bf16"]
+    ref_s = O.flock_score(ref_z)
+    assert np.all(np.abs(np64(s) - ref_s) <= score_tol("bf16") * ref_s + 1e-6 * np.sqrt(S / d_ff))
+
+
 def test_prefill_zero_row_contributes_nothing():
     S, d, d_ff = 16, 64, 96
     L, host = make_layer(d, d_ff, "f32", S_max=S)
