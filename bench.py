@@ -261,19 +261,21 @@ def run_ours(args, w, keep):
     stream = torch.cuda.current_stream()
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(max(1, args.steps))]
 
-    def step(ev=None):
+    def step(ev=None, after_prompt=None, before_decode=None):
         record = ev is not None
         if record: ev[0].record(stream)
         for l in range(L):
             for q in range(B):
                 stack.prefill_score(l, q, X[l, q], Y[l, q])
         if record: ev[1].record(stream)
+        if after_prompt is not None: after_prompt()
         stack.select_all()
         if record: ev[2].record(stream)
         for l in range(0 if indexed else L):
             for q in range(B):
                 stack.compact(l, q)
         if record: ev[3].record(stream)
+        if before_decode is not None: before_decode()
         if dec_graph[0] is not None:
             dec_graph[0].replay()
         else:
@@ -350,12 +352,24 @@ def run_ours(args, w, keep):
     if not args.no_e2e:
         Xh, XDh = X.cpu().pin_memory(), XD.cpu().pin_memory()
         Yh, YDh = torch.empty_like(Xh).pin_memory(), torch.empty_like(XDh).pin_memory()
+        # Every copy of a step is inside the timed region; the two that the phase running at the time does not
+        # depend on go over copy streams of their own (the decode inputs come in under the prompt phase, the
+        # prompt outputs leave under the decode phase), and the step ends when all of them have.
+        copy_in, copy_out = torch.cuda.Stream(), torch.cuda.Stream()
+
+        def prompt_outputs_leave():
+            copy_out.wait_stream(stream)            # the prompt phase has written Y
+            with torch.cuda.stream(copy_out):
+                Yh.copy_(Y, non_blocking=True)
+
         def step_e2e():
             X.copy_(Xh, non_blocking=True)
-            XD.copy_(XDh, non_blocking=True)
-            step()
-            Yh.copy_(Y, non_blocking=True)
+            copy_in.wait_stream(stream)             # the previous step's decode has read XD
+            with torch.cuda.stream(copy_in):
+                XD.copy_(XDh, non_blocking=True)
+            step(after_prompt=prompt_outputs_leave, before_decode=lambda: stream.wait_stream(copy_in))
             YDh.copy_(YD, non_blocking=True)
+            stream.wait_stream(copy_out)
         step_e2e()
         barrier()
         b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

@@ -21,11 +21,10 @@ PREFILL_SHAPES = [(64, 256, 688), (1, 64, 96), (37, 72, 200), (130, 512, 1408), 
                   (300, 1024, 4096), (256, 1024, 20480)]
 
 
-@pytest.mark.parametrize("dtype", ["f32", "bf16"])
-@pytest.mark.parametrize("S,d,d_ff", PREFILL_SHAPES)
+# (the largest case is there for the tensor-core tiling, which is bf16 only)
+@pytest.mark.parametrize("dtype,S,d,d_ff", [(dt, *shape) for dt in ("f32", "bf16") for shape in PREFILL_SHAPES
+                                            if not (dt == "f32" and shape[2] > 5000)])
 def test_prefill_score_without_a_gate_matches_oracle(dtype, S, d, d_ff):
-    if dtype == "f32" and d_ff > 5000:
-        pytest.skip("the tensor-core cases are bf16 only")
     act = ACTS[(S + d_ff // 8) % 4]
     L, host = make_layer(d, d_ff, dtype, act=act, bias=(S in (37, 130, 256)), seed=S + d, S_max=S)
     x = rand((S, d), TD[dtype], 5) + rand((1, d), TD[dtype], 6, 4.0 / d ** 0.5)
