@@ -128,7 +128,7 @@ typedef struct {
  * stream WRITES the compact weights this call reads (do not set it on the first decode
  * call after griffin_compact_experts). */
 #define GRIFFIN_DECODE_OVERLAP_WEIGHT_PREFETCH 1u
-/* bf16 only: use the tcgen05 kernel (the weights go from shared memory straight into the
+/* bf16, gated blocks only (ignored otherwise): use the tcgen05 kernel (the weights go from shared memory straight into the
  * 5th-generation tensor cores) for shapes that it takes (d and ldk multiples of 128); other
  * shapes, and calls without the flag, run the warp-level (mma.sync) kernel.  Results agree
  * within the documented tolerance.  On the measured workloads the warp-level kernel is the
@@ -210,7 +210,7 @@ griffin_status griffin_compact_experts(const griffin_ff_desc *desc, const griffi
  * sets: HOST array of B structs; every set must have the same k and ldk.  Entries may repeat
  * to share a set: when 2..8 sequences of a bf16 call all name the same buffers (one expert
  * set for the batch, Eq. 7) and d and ldk are multiples of 128, the weights are streamed
- * once and every row meets all B vectors (otherwise each sequence is a pass of its own).  b_down [d] or NULL is shared by all sequences.  x [B, d] in,
+ * once and every row meets all B vectors (otherwise, and for blocks without a gate, each sequence is a pass of its own).  b_down [d] or NULL is shared by all sequences.  x [B, d] in,
  * y [B, d] out.  1 <= B <= GRIFFIN_MAX_BATCH, d <= GRIFFIN_MAX_D.  flags: GRIFFIN_DECODE_*.
  * The activations z_hat [B, ldk] pass through the workspace (4 bytes per entry).  With bf16
  * storage the call is one kernel whose CTAs (one per SM) meet half-way through a counter in
