@@ -40,6 +40,32 @@ def test_prefill_score_without_a_gate_matches_oracle(dtype, S, d, d_ff):
     assert np.array_equal(np64(s2), s)
 
 
+@pytest.mark.parametrize("dtype,pieces,d,d_ff", [("bf16", (100, 37, 119), 512, 1024), ("bf16", (300, 1, 211), 1024, 4096),
+                                                 ("f32", (1, 1, 62), 256, 688)])
+def test_prefill_without_a_gate_fed_piece_by_piece(dtype, pieces, d, d_ff):
+    """The statistic's sums of squares carried across the pieces of a prompt (Eq. 6) for a block without a gate."""
+    S, act = sum(pieces), "gelu_tanh"
+    L, host = make_layer(d, d_ff, dtype, act=act, bias=True, seed=S + d, S_max=S)
+    x = rand((S, d), TD[dtype], 25) + rand((1, d), TD[dtype], 26, 4.0 / d ** 0.5)
+    xd = x.to(dev())
+    y = torch.empty((S, d), device=dev(), dtype=TD[dtype])
+    sumsq = torch.full((d_ff,), float("nan"), device=dev())        # the first piece must not read it
+    score = torch.empty((d_ff,), device=dev())
+    at = 0
+    for i, n in enumerate(pieces):
+        last = i == len(pieces) - 1
+        G.griffin_ff_prefill_score_chunk(L.desc, L.weights, xd[at:at + n], y[at:at + n], sumsq, score if last else None,
+                                         i == 0, L.ws)
+        at += n
+    assert L.status() == G.OK
+    ref_y, ref_z = O.ff_dense(np64(x), None, h64(host, "wu"), h64(host, "wd"), act, None, h64(host, "bu"), h64(host, "bd"))
+    ref_s = O.flock_score(ref_z)
+    assert rel_l2(np64(y), ref_y) < TOL_OUT[dtype]
+    s = np64(score)
+    assert np.all(np.abs(s - ref_s) <= score_tol(dtype) * ref_s + 1e-6 * np.sqrt(S / d_ff))
+    assert abs(float(np.sum(s * s)) - S) < 1e-5 * S
+
+
 @pytest.mark.parametrize("act", ACTS)
 def test_prefill_sigma_of_each_block_without_a_gate(act):
     L, host = make_layer(512, 1024, "bf16", act=act, bias=True, seed=11, S_max=96)
