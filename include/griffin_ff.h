@@ -29,6 +29,20 @@
  *   - Calls that share a workspace must be ordered on one stream (they may not overlap on
  *     the GPU).
  *   - No exceptions cross this boundary; every call returns a griffin_status.
+ *   - Device-side waits are bounded (about two seconds of SM clocks).  A kernel whose wait runs
+ *     out raises the workspace's status word and returns; griffin_check_device_status then says
+ *     GRIFFIN_ERR_TIMEOUT, the outputs of that call are undefined, and the workspace must be
+ *     cleared with griffin_workspace_init before its next use (the word stays raised until then).
+ *   - What the library keeps between calls, per process: small host-side tables (SM count and
+ *     granted shared-memory limits per device, guarded by a mutex) and, for the bf16 prompt
+ *     phase, one non-blocking side stream and two events per host thread and device, created by
+ *     that thread's first griffin_ff_prefill_score[_chunk] call on the device and never
+ *     destroyed: the statistic's kernels run there beside the down projection and rejoin
+ *     `stream` before the call returns.  Make that first call outside any stream capture.  Set
+ *     the environment variable GRIFFIN_NO_SIDE_STREAM (to anything) before the first call to
+ *     keep every kernel on the caller's stream.
+ *   - Entry points may be called from several host threads at once, on different streams and
+ *     workspaces.
  */
 #ifndef GRIFFIN_FF_H
 #define GRIFFIN_FF_H
@@ -141,6 +155,12 @@ const char *griffin_status_string(griffin_status st);
 /* Library ABI version (GRIFFIN_FF_VERSION at build time). */
 int32_t griffin_version(void);
 
+/* Number of kernels the library has launched (or recorded into a stream capture) in this process
+ * so far, over all devices and threads.  A diagnostic: the difference across a piece of work says
+ * how many launches it took.  Replaying a captured graph does not go through the library and is not
+ * counted. */
+uint64_t griffin_kernel_launches(void);
+
 /* k for a keep ratio (= 1 - the paper's "FF sparsity", Section 5): floor(keep*d_ff + 0.5)
  * clamped to [1, d_ff].  Host-only arithmetic. */
 int32_t griffin_k_from_keep_ratio(int32_t d_ff, double keep);
@@ -153,7 +173,8 @@ int32_t griffin_compact_ldk(int32_t k);
  * invalid. */
 size_t griffin_workspace_bytes(const griffin_ff_desc *desc, int32_t S_max, int32_t n_seq_max);
 
-/* Clears the workspace header (device status word).  Enqueue once before first use. */
+/* Clears the workspace header (device status word, meeting counters of the one-kernel decode calls).
+ * Enqueue once before first use, and again after a GRIFFIN_ERR_TIMEOUT. */
 griffin_status griffin_workspace_init(void *workspace, size_t ws_bytes, void *stream);
 
 /* Prompt phase (Section 4.2, "Prompt Phase Expert Neuron Selection").
@@ -257,16 +278,27 @@ griffin_status griffin_ff_decode_indexed(const griffin_ff_desc *desc, int32_t B,
  *   - The first call on each device looks up the array's device address (with that device
  *     current); make that first call outside any stream capture.
  *   - All calls on a device share the one array.  It keeps whatever the previous call left
- *     there; nothing in it needs to start at zero, because every entry the second kernel
- *     reads has been written by the first kernel of the same call.  Two calls that overlap
- *     on the GPU (different streams) race on it: keep calls on one device ordered.
- *   - There is no status word: should a bounded wait inside a kernel give up, the call's
- *     output is incomplete and nothing reports it.  Callers that need that report use
- *     griffin_ff_decode. */
+ *     there.  The scratch proper needs no clearing, because every entry the second half of a
+ *     call reads has been written by its first half.  In front of it the array carries the
+ *     256 bytes that a workspace starts with: a status word and the counters through which the
+ *     CTAs of the one-kernel bf16 decode meet half-way.  They are zero when the library is
+ *     loaded; the counters run round and stay in step from call to call as long as every call
+ *     runs to its end (every CTA reports in exactly once per call, also after a give-up).
+ *     Two calls that overlap on the GPU (different streams) race on the array: keep the calls
+ *     on one device ordered.
+ *   - Should a bounded wait inside a kernel give up, the call's output is incomplete;
+ *     griffin_ff_decode_static_status reports it (and clears the header again). */
 #define GRIFFIN_STATIC_SCRATCH_BYTES (1u << 20)
 griffin_status griffin_ff_decode_static(const griffin_ff_desc *desc, int32_t B,
                                         const griffin_ff_compact *sets /*host*/, const void *b_down,
                                         const void *x, void *y, uint32_t flags, void *stream);
+
+/* Companion of griffin_ff_decode_static (no counterpart in the paper either): synchronises `stream`,
+ * reads the status word in front of the current device's static array and returns what
+ * griffin_check_device_status would for a workspace.  When the word was raised, the header (word
+ * and meeting counters) is cleared again, so that the array is fit for the next call; call it only
+ * while no griffin_ff_decode_static call is running on the device.  Allocates nothing. */
+griffin_status griffin_ff_decode_static_status(void *stream);
 
 /* Synchronises `stream`, then reads the workspace's device status word.  GRIFFIN_OK,
  * GRIFFIN_ERR_TIMEOUT (a bounded wait inside a kernel gave up), GRIFFIN_ERR_INVALID_ARG

@@ -35,6 +35,7 @@ EXPORTS = (
     "griffin_workspace_bytes", "griffin_workspace_init", "griffin_ff_prefill_score", "griffin_select_topk",
     "griffin_combine_scores", "griffin_compact_experts", "griffin_ff_decode", "griffin_check_device_status",
     "griffin_ff_decode_static", "griffin_ff_decode_indexed", "griffin_ff_prefill_score_chunk",
+    "griffin_kernel_launches", "griffin_ff_decode_static_status",
 )
 
 
@@ -79,6 +80,8 @@ def load(path=None):
     lib.griffin_status_string.argtypes = [C.c_int]
     lib.griffin_version.restype = i32
     lib.griffin_version.argtypes = []
+    lib.griffin_kernel_launches.restype = C.c_uint64
+    lib.griffin_kernel_launches.argtypes = []
     lib.griffin_k_from_keep_ratio.restype = i32
     lib.griffin_k_from_keep_ratio.argtypes = [i32, C.c_double]
     lib.griffin_compact_ldk.restype = i32
@@ -104,6 +107,8 @@ def load(path=None):
     lib.griffin_ff_decode_indexed.argtypes = [C.POINTER(FFDesc), i32, C.POINTER(FFWeightsNM), vp, i32, vp, vp, vp, sz, u32, vp]
     lib.griffin_ff_decode_static.restype = C.c_int
     lib.griffin_ff_decode_static.argtypes = [C.POINTER(FFDesc), i32, C.POINTER(FFCompact), vp, vp, vp, u32, vp]
+    lib.griffin_ff_decode_static_status.restype = C.c_int
+    lib.griffin_ff_decode_static_status.argtypes = [vp]
     lib.griffin_check_device_status.restype = C.c_int
     lib.griffin_check_device_status.argtypes = [vp, vp]
     _lib = lib
@@ -131,6 +136,11 @@ def status_string(st):
 
 def griffin_version():
     return load().griffin_version()
+
+
+def griffin_kernel_launches():
+    """Kernels launched by the library in this process so far."""
+    return int(load().griffin_kernel_launches())
 
 
 def griffin_k_from_keep_ratio(d_ff, keep):
@@ -260,6 +270,11 @@ def griffin_ff_decode_static(desc, sets, b_down, x, y, flags=DECODE_DEFAULT, str
     arr = sets if isinstance(sets, C.Array) else compact_array(sets)
     _check(load().griffin_ff_decode_static(C.byref(desc), len(arr), arr, _ptr(b_down), _ptr(x), _ptr(y), int(flags),
                                            _stream(stream)), "griffin_ff_decode_static")
+
+
+def griffin_ff_decode_static_status(stream=None):
+    """Status of the static-scratch decode calls on the current device (synchronises the stream)."""
+    return load().griffin_ff_decode_static_status(_stream(stream))
 
 
 def griffin_check_device_status(ws, stream=None):

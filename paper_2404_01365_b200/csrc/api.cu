@@ -1,6 +1,9 @@
 // C ABI entry points: host-side validation, workspace carve-up, dispatch to the launchers.
 #include <math.h>
 
+#include <atomic>
+#include <mutex>
+
 #include "common.cuh"
 #include "launch.h"
 
@@ -8,16 +11,19 @@ using namespace griffin;
 
 namespace griffin {
 
+static std::atomic<uint64_t> g_launches{0};
+void count_launches(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
 int device_sm_count() {
-    static int cached[64] = {0};
+    static std::atomic<int> cached[64];  // (zero-initialised; two threads that race both store the same value)
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return -1;
-    if (cached[dev] == 0) {
-        int n = 0;
+    int n = cached[dev].load(std::memory_order_relaxed);
+    if (n == 0) {
         if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -1;
-        cached[dev] = n;
+        cached[dev].store(n, std::memory_order_relaxed);
     }
-    return cached[dev];
+    return n;
 }
 
 cudaError_t ensure_dynamic_smem(const void *fn, size_t bytes) {
@@ -29,9 +35,11 @@ cudaError_t ensure_dynamic_smem(const void *fn, size_t bytes) {
     };
     static Entry table[128];
     static int n_entries = 0;
+    static std::mutex table_mutex;  // entry points may be called from several host threads
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lock(table_mutex);
     for (int i = 0; i < n_entries; ++i)
         if (table[i].fn == fn && table[i].dev == dev) {
             if (table[i].bytes >= bytes) return cudaSuccess;
@@ -82,6 +90,8 @@ const char *griffin_status_string(griffin_status st) {
 }
 
 int32_t griffin_version(void) { return GRIFFIN_FF_VERSION; }
+
+uint64_t griffin_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
 
 int32_t griffin_k_from_keep_ratio(int32_t d_ff, double keep) {
     if (d_ff < 1) return 0;
@@ -256,6 +266,10 @@ griffin_status griffin_ff_decode_static(const griffin_ff_desc *desc, int32_t B, 
     if (!aligned16(x) || !aligned16(y)) return GRIFFIN_ERR_ALIGNMENT;
     // the size check against GRIFFIN_STATIC_SCRATCH_BYTES happens in the launcher, before any CUDA call
     return launch_decode_static(desc, B, sets, b_down, x, y, flags, static_cast<cudaStream_t>(stream));
+}
+
+griffin_status griffin_ff_decode_static_status(void *stream) {
+    return static_scratch_status(static_cast<cudaStream_t>(stream));
 }
 
 griffin_status griffin_check_device_status(const void *workspace, void *stream) {

@@ -135,10 +135,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
 // Every device-side wait gives up after this many SM clock cycles (about 2 s).
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;
 
-// Barrier wait that gives up after WAIT_LIMIT_CYCLES, or as soon as another thread of the CTA
-// has given up.  On a give-up the status word is raised and false is returned.
+// Barrier wait that gives up after `limit` SM clock cycles (WAIT_LIMIT_CYCLES everywhere in the
+// library; only the self-test of this primitive passes a shorter one), or as soon as another
+// thread of the CTA has given up.  On a give-up the status word is raised and false is returned.
 __device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort, void *ws,
-                                              int where) {
+                                              int where, long long limit = WAIT_LIMIT_CYCLES) {
     // Fast path: plain polling.  The clock is only consulted every few thousand polls, so a
     // wait that succeeds (every wait of a healthy run) never pays for reading it.
     if (mbar_try_wait(bar, parity)) return true;
@@ -152,7 +153,7 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, vo
         for (int i = 0; i < 4096; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort) return false;
-        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+        if (clock64() - t0 > limit) {
             *abort = 1;
             raise_status(ws, DEV_STATUS_TIMEOUT, where);
             return false;

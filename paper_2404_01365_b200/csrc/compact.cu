@@ -180,6 +180,7 @@ static griffin_status compact_typed(const griffin_ff_desc *desc, const griffin_f
     const bool biases = (w->b_gate && out->b_gate_c) || (w->b_up && out->b_up_c);
     const int bias_blocks = biases ? (k + CP_THREADS - 1) / CP_THREADS : 0;
     compact_kernel<U><<<a.cols_blocks + a.rows_blocks + bias_blocks, CP_THREADS, 0, stream>>>(a);
+    count_launches(1);
     if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
     return GRIFFIN_OK;
 }

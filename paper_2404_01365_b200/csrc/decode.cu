@@ -16,6 +16,8 @@
 //     the previous kernel on the stream has finished; everything that depends on that
 //     kernel (x, z, y) is touched only after griddepcontrol.wait.
 // Results are deterministic: every sum has a fixed order.
+#include <atomic>
+
 #include "decode_common.cuh"
 
 namespace griffin {
@@ -311,6 +313,7 @@ cudaError_t launch_maybe_overlapped(const void *func, dim3 grid, dim3 block, siz
     attr[0].val.programmaticStreamSerializationAllowed = overlap ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    count_launches(1);
     return cudaLaunchKernelExC(&cfg, func, args);
 }
 
@@ -430,15 +433,30 @@ griffin_status launch_decode(const griffin_ff_desc *desc, int B, const griffin_f
 static __device__ __align__(256) unsigned char g_static_decode_scratch[256 + GRIFFIN_STATIC_SCRATCH_BYTES];
 
 static unsigned char *static_scratch_of_current_device() {
-    static unsigned char *addr[64] = {nullptr};
+    static std::atomic<unsigned char *> addr[64];  // (zero-initialised; two threads that race both store the same address)
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-    if (addr[dev] == nullptr) {
+    unsigned char *a = addr[dev].load(std::memory_order_acquire);
+    if (a == nullptr) {
         void *p = nullptr;
         if (cudaGetSymbolAddress(&p, g_static_decode_scratch) != cudaSuccess) return nullptr;
-        addr[dev] = static_cast<unsigned char *>(p);
+        a = static_cast<unsigned char *>(p);
+        addr[dev].store(a, std::memory_order_release);
     }
-    return addr[dev];
+    return a;
+}
+
+griffin_status static_scratch_status(cudaStream_t stream) {
+    unsigned char *base = static_scratch_of_current_device();
+    if (base == nullptr) return GRIFFIN_ERR_CUDA;
+    WsHeader h;
+    if (cudaMemcpyAsync(&h, base, sizeof(h), cudaMemcpyDeviceToHost, stream) != cudaSuccess) return GRIFFIN_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return GRIFFIN_ERR_CUDA;
+    if (h.status == DEV_STATUS_OK) return GRIFFIN_OK;
+    if (cudaMemsetAsync(base, 0, WS_HEADER_BYTES, stream) != cudaSuccess || cudaStreamSynchronize(stream) != cudaSuccess)
+        return GRIFFIN_ERR_CUDA;
+    if (h.status == DEV_STATUS_TIMEOUT) return GRIFFIN_ERR_TIMEOUT;
+    return h.status == DEV_STATUS_BAD_INDEX ? GRIFFIN_ERR_INVALID_ARG : GRIFFIN_ERR_CUDA;
 }
 
 griffin_status launch_decode_static(const griffin_ff_desc *desc, int B, const griffin_ff_compact *sets,

@@ -101,6 +101,13 @@ __device__ __forceinline__ bool grid_meet(unsigned int *counter, unsigned int n,
     }
 }
 
+// The arrival alone, for a party that has given up on its work: the other parties of this launch are not
+// held up by it and the counter stays in phase for the next launch.
+__device__ __forceinline__ void grid_arrive_only(unsigned int *counter, unsigned int n) {
+    __threadfence();
+    atomicInc(counter, 2 * n - 1);
+}
+
 // Launches `func`, optionally allowing it to start before the previous kernel on the stream
 // has completed (programmatic dependent launch).
 cudaError_t launch_maybe_overlapped(const void *func, dim3 grid, dim3 block, size_t smem, cudaStream_t stream,

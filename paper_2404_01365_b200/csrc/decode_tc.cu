@@ -551,11 +551,19 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     }
                 }
             }
-            if (!stop && half == 0) {
-                // ---- the meeting point: this CTA's z entries are written; the thread that reports in makes them visible
-                bool bad = epi_barrier_or(false);
-                if (et == 0) bad = !grid_meet(&static_cast<WsHeader *>(p.ws)->meet_tc, gridDim.x, s.abort, p.ws);
-                if (epi_barrier_or(bad)) stop = true;
+            if (half == 0) {
+                // ---- the meeting point: this CTA's z entries are written; the thread that reports in makes them visible.
+                // (`stop` is the same in every epilogue thread: it only changes behind epi_barrier_or.)  After a give-up
+                // the CTA still reports in, without waiting: the counter runs round modulo twice the number of
+                // CTAs and is never reset, so every CTA must add exactly one arrival per launch, or every later
+                // call on this workspace would meet out of phase.
+                if (stop) {
+                    if (et == 0) grid_arrive_only(&static_cast<WsHeader *>(p.ws)->meet_tc, gridDim.x);
+                } else {
+                    bool bad = epi_barrier_or(false);
+                    if (et == 0) bad = !grid_meet(&static_cast<WsHeader *>(p.ws)->meet_tc, gridDim.x, s.abort, p.ws);
+                    if (epi_barrier_or(bad)) stop = true;
+                }
             }
         }
     }

@@ -13,6 +13,9 @@ namespace griffin {
 // Number of SMs of the current device (cached per device); <= 0 on error.
 int device_sm_count();
 
+// Adds n to the count of kernels this library has launched in this process (griffin_kernel_launches).
+void count_launches(int n);
+
 // Raises the opt-in dynamic shared memory limit of `fn` on the current device when needed.
 cudaError_t ensure_dynamic_smem(const void *fn, size_t bytes);
 
@@ -22,6 +25,9 @@ griffin_status launch_decode(const griffin_ff_desc *desc, int B, const griffin_f
 // Decode with the z scratch in the library's own static device array (no workspace).
 griffin_status launch_decode_static(const griffin_ff_desc *desc, int B, const griffin_ff_compact *sets,
                                     const void *b_down, const void *x, void *y, uint32_t flags, cudaStream_t stream);
+
+// Status word in front of the current device's static array; clears the header when it was raised.
+griffin_status static_scratch_status(cudaStream_t stream);
 
 // Index-direct decode (decode_indexed.cu): expert rows read in place from neuron-major weights.
 constexpr int IDX_MAX_GRID = 148;  // CTAs (= partial-sum rows per sequence in the workspace) at most

@@ -16,6 +16,8 @@
 //
 // This file holds the fp32-FMA (SIMT) matrix kernels, which serve the fp32 storage type
 // and any shape the tensor-core path does not take, plus steps 3-5 and the dispatcher.
+#include <stdlib.h>
+
 #include <type_traits>
 
 #include "common.cuh"
@@ -250,7 +252,8 @@ __global__ void score_finish_kernel(const float *__restrict__ colpart, int n_row
 // The statistic only needs Z, the down projection only Z as well: with the tensor-core path the
 // statistic kernels run on a stream of the library's own beside the second GEMM (whose
 // persistent CTAs leave room for them on every SM) and join the caller's stream at the end.
-// One lane per host thread and device, created at first use and kept.
+// One lane per host thread and device, created at first use and kept.  With the environment
+// variable GRIFFIN_NO_SIDE_STREAM set there is none: everything stays on the caller's stream.
 struct SideLane {
     cudaStream_t stream;
     cudaEvent_t fork, join;
@@ -259,6 +262,8 @@ static SideLane *side_lane_of_current_device() {
     constexpr int MAX_DEV = 64;
     static thread_local SideLane lanes[MAX_DEV];
     static thread_local int state[MAX_DEV];  // 0 untried, 1 ready, -1 unavailable
+    static const bool disabled = getenv("GRIFFIN_NO_SIDE_STREAM") != nullptr;
+    if (disabled) return nullptr;
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEV) return nullptr;
     if (state[dev] == 0) {
@@ -306,15 +311,17 @@ static griffin_status prefill_typed(const griffin_ff_desc *desc, const griffin_f
     } else {
         n_col_tiles = (d_ff + PF_BN - 1) / PF_BN;
         const dim3 g1(n_col_tiles, (S + PF_BM - 1) / PF_BM);
-        if (act_gated(desc->act))
+        if (act_gated(desc->act)) {
             ff1_simt_kernel<T, true><<<g1, PF_THREADS, 0, stream>>>(
                 static_cast<const T *>(x), static_cast<const T *>(w->w_gate), static_cast<const T *>(w->w_up),
                 static_cast<const T *>(w->b_gate), static_cast<const T *>(w->b_up), z, zf, rowsq, S, d, d_ff,
                 n_col_tiles, desc->act);
-        else
+        } else {
             ff1_simt_kernel<T, false><<<g1, PF_THREADS, 0, stream>>>(
                 static_cast<const T *>(x), nullptr, static_cast<const T *>(w->w_up), nullptr,
                 static_cast<const T *>(w->b_up), z, zf, rowsq, S, d, d_ff, n_col_tiles, act_sigma(desc->act));
+        }
+        count_launches(1);
         if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
     }
     if (!ff2_done && y != nullptr) {
@@ -322,21 +329,31 @@ static griffin_status prefill_typed(const griffin_ff_desc *desc, const griffin_f
         ff2_simt_kernel<T><<<g2, PF_THREADS, 0, stream>>>(z, static_cast<const T *>(w->w_down),
                                                           static_cast<const T *>(w->b_down), static_cast<T *>(y), S, d,
                                                           d_ff);
+        count_launches(1);
         if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
     }
+    griffin_status st = GRIFFIN_OK;
     row_inv_kernel<<<(S + 7) / 8, 256, 0, stat_stream>>>(rowsq, S, n_col_tiles, inv);
-    if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
+    count_launches(1);
+    if (cudaGetLastError() != cudaSuccess) st = GRIFFIN_ERR_CUDA;
     const float *z32 = kBf16 ? zf : reinterpret_cast<const float *>(z);
     const dim3 g4((d_ff + 127) / 128, ps.n_row_chunks);
-    col_partial_kernel<<<g4, 256, 0, stat_stream>>>(z32, inv, S, d_ff, colpart);
-    if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
-    score_finish_kernel<<<(d_ff + 255) / 256, 256, 0, stat_stream>>>(colpart, ps.n_row_chunks, d_ff, score, sumsq,
-                                                                             first);
-    if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
+    if (st == GRIFFIN_OK) {
+        col_partial_kernel<<<g4, 256, 0, stat_stream>>>(z32, inv, S, d_ff, colpart);
+        count_launches(1);
+        if (cudaGetLastError() != cudaSuccess) st = GRIFFIN_ERR_CUDA;
+    }
+    if (st == GRIFFIN_OK) {
+        score_finish_kernel<<<(d_ff + 255) / 256, 256, 0, stat_stream>>>(colpart, ps.n_row_chunks, d_ff, score, sumsq,
+                                                                                 first);
+        count_launches(1);
+        if (cudaGetLastError() != cudaSuccess) st = GRIFFIN_ERR_CUDA;
+    }
+    // whatever went to the side stream rejoins the caller's stream, also when a launch above failed
     if (lane != nullptr &&
         (cudaEventRecord(lane->join, lane->stream) != cudaSuccess || cudaStreamWaitEvent(stream, lane->join, 0) != cudaSuccess))
         return GRIFFIN_ERR_CUDA;
-    return GRIFFIN_OK;
+    return st;
 }
 
 griffin_status launch_prefill_score(const griffin_ff_desc *desc, const griffin_ff_weights *w, const void *x, int S,

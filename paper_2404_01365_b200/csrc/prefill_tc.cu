@@ -631,6 +631,7 @@ static griffin_status launch_tc(const CUtensorMap &ma, const CUtensorMap &mb0, c
     const int tiles = p.tail_ks > 1 ? p.tail_first + (p.m_tiles * p.n_tiles - p.tail_first) * p.tail_ks
                                     : p.m_tiles * p.n_tiles * p.splits;
     ff_tc_kernel<KIND, BN><<<tiles < sms ? tiles : sms, TC_THREADS, smem, stream>>>(ma, mb0, mb1, p);
+    count_launches(1);
     return cudaGetLastError() == cudaSuccess ? GRIFFIN_OK : GRIFFIN_ERR_CUDA;
 }
 
@@ -668,6 +669,7 @@ griffin_status launch_prefill_tc(const griffin_ff_desc *desc, const griffin_ff_w
                               : launch_tc<TC_WIDE, 128>(mx, mg, mu, p, sms, stream);
     if (st == GRIFFIN_OK && p.tail_ks > 1) {
         dual_tail_finish_kernel<<<(p.m_tiles * p.n_tiles - p.tail_first) * (TC_BM / 4), 128, 0, stream>>>(p);
+        count_launches(1);
         if (cudaGetLastError() != cudaSuccess) st = GRIFFIN_ERR_CUDA;
     }
     if (st == GRIFFIN_OK && after_ff1 != nullptr && cudaEventRecord(after_ff1, stream) != cudaSuccess) return GRIFFIN_ERR_CUDA;
@@ -698,12 +700,14 @@ griffin_status launch_prefill_tc(const griffin_ff_desc *desc, const griffin_ff_w
                    : launch_tc<TC_PLAIN, 128>(mz, md, md, q, sms, stream);
     if (st == GRIFFIN_OK && q.tail_ks > 1) {
         plain_tail_finish_kernel<<<(q.m_tiles * q.n_tiles - q.tail_first) * (TC_BM / 4), 128, 0, stream>>>(q);
+        count_launches(1);
         if (cudaGetLastError() != cudaSuccess) st = GRIFFIN_ERR_CUDA;
     }
     if (st != GRIFFIN_OK || splits == 1) return st;
     const size_t n_elems = (size_t)S * d;
     splitk_reduce_kernel<<<(unsigned)((n_elems / 4 + 255) / 256), 256, 0, stream>>>(
         ypart, static_cast<const __nv_bfloat16 *>(w->b_down), static_cast<__nv_bfloat16 *>(y), splits, n_elems, d);
+    count_launches(1);
     return cudaGetLastError() == cudaSuccess ? GRIFFIN_OK : GRIFFIN_ERR_CUDA;
 }
 

@@ -105,16 +105,15 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 
 // The driver's tensor-map encoder, looked up through the runtime (the library does not link libcuda).
 inline EncodeTiledFn encode_tiled_fn() {
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
+    // (a function-local static is initialised once, also when several host threads get here together)
+    static const EncodeTiledFn fn = [] {
         void *sym = nullptr;
         cudaDriverEntryPointQueryResult qres;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
             qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(sym);
-    }
+            return reinterpret_cast<EncodeTiledFn>(sym);
+        return static_cast<EncodeTiledFn>(nullptr);
+    }();
     return fn;
 }
 

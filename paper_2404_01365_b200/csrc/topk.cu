@@ -120,6 +120,7 @@ __global__ void combine_scores_kernel(const float *__restrict__ score, const __g
 
 griffin_status launch_select_topk(const float *score, int n_seq, int d_ff, int k, int32_t *idx, cudaStream_t stream) {
     select_topk_kernel<<<n_seq, TOPK_THREADS, 0, stream>>>(score, d_ff, k, idx);
+    count_launches(1);
     return cudaGetLastError() == cudaSuccess ? GRIFFIN_OK : GRIFFIN_ERR_CUDA;
 }
 
@@ -128,6 +129,7 @@ griffin_status launch_combine_scores(const float *score, const int32_t *prompt_l
     CombineWeights cw;
     for (int i = 0; i < n_seq; ++i) cw.w[i] = (float)(1.0 / sqrt((double)prompt_len_host[i]));
     combine_scores_kernel<<<(d_ff + 255) / 256, 256, 0, stream>>>(score, cw, n_seq, d_ff, out);
+    count_launches(1);
     return cudaGetLastError() == cudaSuccess ? GRIFFIN_OK : GRIFFIN_ERR_CUDA;
 }
 
