@@ -476,6 +476,28 @@ def section_entry(w, B, keep, dev, args, peaks, with_dense):
     return entry
 
 
+def shared_set_entry(w, keep, dev, args, peaks):
+    """Decode with ONE expert set for the whole batch (the batch statistic of Eq. 7): the compact weights are
+    streamed once per call whatever the batch, so the algorithmic bytes are those of one sequence plus the
+    vectors.  Timed on the decode calls alone, T x L of them per repetition, for batches of 2, 4 and 8."""
+    import torch
+    job = Job(w, 8, keep, w.L, dev, 0, False, not args.no_graph)
+    job.warm_up(1)                                   # fills the expert sets; the first sequence's is the one shared
+    st, out = job.stack, {}
+    for Bs in (2, 4, 8):
+        arrays = [job.G.compact_array([st.sets[l][0]] * Bs) for l in range(w.L)]
+        us = job.time_decode_only(arrays, Bs, 2)
+        nbytes = st.n_mats * job.k * w.d * w.elem_bytes + Bs * 2 * w.d * w.elem_bytes
+        out[f"B{Bs}"] = {"us_per_call": us, "tokens_per_s_per_layer": Bs / (us * 1e-6), "gbs": nbytes / (us * 1e-6) / 1e9,
+                         "frac_of_hbm": nbytes / (us * 1e-6) / 1e9 / peaks[0], "algorithmic_bytes_per_call": nbytes}
+    if job.stack.status() != job.G.OK:
+        raise RuntimeError("device status word raised")
+    job = None
+    release()
+    return {"workload": w.name, "keep": keep, "k": out and int(max(1, min(w.d_ff, int(keep * w.d_ff + 0.5)))), "L": w.L, "T": w.T,
+            "what": "decode calls whose sequences all name one compact expert set", "decode": out}
+
+
 def run_ours(args, w, keep):
     import torch
     import torch.distributed as dist
@@ -613,6 +635,7 @@ def run_ours(args, w, keep):
         for kp in W["mistral_7b"].keeps:
             sect.append(section_entry(W["mistral_7b"], W["mistral_7b"].B, kp, dev, args, peaks, False))
         line["workloads"] = sect
+        line["shared_expert_set"] = shared_set_entry(W["llama2_7b"], 0.5, dev, args, peaks)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(w, keep)
     if rank == 0:

@@ -143,10 +143,11 @@ typedef struct {
  * call after griffin_compact_experts). */
 #define GRIFFIN_DECODE_OVERLAP_WEIGHT_PREFETCH 1u
 /* bf16, gated blocks only (ignored otherwise): use the tcgen05 kernel (the weights go from shared memory straight into the
- * 5th-generation tensor cores) for shapes that it takes (d and ldk multiples of 128); other
- * shapes, and calls without the flag, run the warp-level (mma.sync) kernel.  Results agree
- * within the documented tolerance.  On the measured workloads the warp-level kernel is the
- * faster of the two, which is why it is the default. */
+ * 5th-generation tensor cores) for shapes that it takes (d and ldk multiples of 128; with one
+ * shared expert set 2..8 sequences); other shapes, and calls without the flag, run the
+ * warp-level (mma.sync) kernels.  Results agree within the documented tolerance.  On the
+ * measured workloads the warp-level kernels are the faster ones, which is why they are the
+ * default. */
 #define GRIFFIN_DECODE_TCGEN05 2u
 
 /* Status text for a code (static string, never NULL). */
@@ -229,9 +230,11 @@ griffin_status griffin_compact_experts(const griffin_ff_desc *desc, const griffi
  *   y[b] = W_2_hat (sigma(W_g_hat x[b] + b_g_hat) * (W_1_hat x[b] + b_1_hat)) + b_2
  * (without a gate: y[b] = W_2_hat sigma(W_1_hat x[b] + b_1_hat) + b_2).
  * sets: HOST array of B structs; every set must have the same k and ldk.  Entries may repeat
- * to share a set: when 2..8 sequences of a bf16 call all name the same buffers (one expert
- * set for the batch, Eq. 7) and d and ldk are multiples of 128, the weights are streamed
- * once and every row meets all B vectors (otherwise, and for blocks without a gate, each sequence is a pass of its own).  b_down [d] or NULL is shared by all sequences.  x [B, d] in,
+ * to share a set: when all the sequences of a bf16 call name the same buffers (one expert
+ * set for the batch, Eq. 7), the weights are streamed once for every 8 sequences (fewer when
+ * d or ldk is so large that 8 vectors do not fit in shared memory beside the weight stages)
+ * and every weight row meets all those vectors at once; with distinct sets each sequence is
+ * a pass of its own.  b_down [d] or NULL is shared by all sequences.  x [B, d] in,
  * y [B, d] out.  1 <= B <= GRIFFIN_MAX_BATCH, d <= GRIFFIN_MAX_D.  flags: GRIFFIN_DECODE_*.
  * The activations z_hat [B, ldk] pass through the workspace (4 bytes per entry).  With bf16
  * storage the call is one kernel whose CTAs (one per SM) meet half-way through a counter in

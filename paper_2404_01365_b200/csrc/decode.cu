@@ -413,10 +413,15 @@ griffin_status launch_decode(const griffin_ff_desc *desc, int B, const griffin_f
     const int act = act_sigma(desc->act);
     const bool gated = act_gated(desc->act);
     if (desc->dtype == GRIFFIN_DT_F32) return decode_simt<float>(p, act, gated, flags, stream);
-    if (!gated) return decode_bf16_mma(p, act, false, flags, stream);  // (the tcgen05 kernels are built for gated blocks)
-    // one expert set for several sequences (Eq. 7): only the tcgen05 kernel streams it once for all of them
-    // (a shape that its plan cannot place in shared memory or TMEM after all goes to the warp-level kernel)
-    if (decode_tc_shared(p) || ((flags & GRIFFIN_DECODE_TCGEN05) && decode_tc_supported(p))) {
+    const bool want_tc = gated && (flags & GRIFFIN_DECODE_TCGEN05) != 0;  // (the tcgen05 kernels are built for gated blocks)
+    // one expert set for several sequences (Eq. 7): streamed once for up to 8 of them at a time
+    if (decode_shared_set(p) && !(want_tc && decode_tc_shared(p))) {
+        const griffin_status st = decode_bf16_shared(p, act, gated, flags, stream);
+        if (st != GRIFFIN_ERR_UNSUPPORTED) return st;
+    }
+    if (!gated) return decode_bf16_mma(p, act, false, flags, stream);
+    // (a shape that the tcgen05 plan cannot place in shared memory or TMEM after all goes to the warp-level kernel)
+    if (want_tc && decode_tc_supported(p)) {
         const griffin_status st = decode_bf16_tc(p, act, flags, stream);
         if (st != GRIFFIN_ERR_UNSUPPORTED) return st;
     }

@@ -15,11 +15,12 @@ import numpy as np
 NORTH_STAR_L2 = {"f32": 1e-4, "bf16": 2e-2}      # the stated bounds on the relative L2 error
 # bf16 storage: y is rounded to bf16 (half an ulp = 2^-9 of the element, elements reach 4-5 rms) and the
 # activations between the two products are rounded to bf16 (2^-9 each, averaging out over k terms);
-# measured worst case over the suite: relative L2 2.6e-3, largest element error 0.016 rms.
+# measured worst case over the suite (1123 outputs): relative L2 3.0e-3, largest element error 0.019 rms.
 # fp32 storage: fp32 accumulation over d and k terms in a fixed but different order from the oracle's;
-# measured worst case: relative L2 4e-7, largest element error 2e-6 rms.
-TEST_L2 = {"f32": 5e-6, "bf16": 6e-3}
-TEST_MAX_OVER_RMS = {"f32": 2e-5, "bf16": 0.04}
+# measured worst case (231 outputs): relative L2 1.3e-6, largest element error 1.2e-5 rms.
+# The bounds are about 2.6 times (bf16) and 3-4 times (fp32) those worst cases.
+TEST_L2 = {"f32": 5e-6, "bf16": 8e-3}
+TEST_MAX_OVER_RMS = {"f32": 4e-5, "bf16": 0.05}
 
 _stats = {}
 

@@ -184,8 +184,13 @@ SHARED_SET_SHAPES = [
     (4096, 11008, 5504, 8, "swiglu", False),   # the most that one call streams together
     (2048, 5632, 2816, 5, "reglu", True),
     (1024, 2816, 1408, 2, "geglu_erf", True),
-    (8192, 1024, 512, 8, "swiglu", False),     # the vectors would not leave room for the ring: one pass per sequence
-    (1000, 1504, 751, 4, "swiglu", False),     # shapes that only the warp-level kernel takes
+    (8192, 1024, 512, 8, "swiglu", False),     # the widest rows: shorter chunks make room for the eight vectors
+    (1000, 1504, 751, 4, "swiglu", False),     # rows that end inside a block of four units; odd k
+    (4096, 11008, 11008, 8, "swiglu", False),  # the unpruned block: eight vectors of 22 KB, taken in two passes of four
+    (1024, 2816, 1408, 11, "swiglu", True),    # more than eight sequences: a pass of eight and a pass of three
+    (64, 96, 37, 2, "reglu", True),            # fewer neurons than CTAs: most work items are empty
+    (2048, 8192, 4000, 6, "relu", True),       # a block without a gate (Eq. 2)
+    (1024, 4096, 2048, 8, "gelu_tanh", False),  # ... and another
 ]
 
 
@@ -200,12 +205,19 @@ def test_decode_with_one_shared_set_matches_oracle_and_separate_calls(d, d_ff, k
     ref = O.ff_pruned(np64(x), c, act, h64(host, "bd"))
     y = L.decode([cs] * B, x)
     y2 = L.decode([cs] * B, x, G.DECODE_OVERLAP_WEIGHT_PREFETCH)
+    y3 = L.decode([cs] * B, x)
     assert L.status() == G.OK
-    assert torch.equal(y, y2)
+    assert torch.equal(y, y2) and torch.equal(y, y3)     # bitwise reproducible
     for b in range(B):
         assert_output(np64(y[b]), ref[b], "bf16", b)
         y1 = L.decode([cs], x[b:b + 1])   # the same sequence on its own
         assert_output(np64(y[b]), np64(y1[0]), "bf16", b, scale=2.0)
+    # the opt-in tcgen05 kernel has a shared-set mode of its own (gated blocks, 2..8 sequences, whole windows);
+    # where it does not apply the flag changes nothing
+    yt = L.decode([cs] * B, x, G.DECODE_TCGEN05)
+    assert L.status() == G.OK
+    for b in range(B):
+        assert_output(np64(yt[b]), ref[b], "bf16", ("tcgen05", b))
 
 
 # Decode straight from the full weights through the index list: d, d_ff, k, B, activation, biases

@@ -42,7 +42,9 @@ def test_a_wait_that_nobody_ends_gives_up_reports_a_timeout_and_the_workspace_wo
     torch.cuda.synchronize()                               # the kernel returned: the wait was bounded
     gave_up, cycles = (int(v) for v in out.cpu())
     assert gave_up == 1
-    assert limit < cycles < 200 * limit                    # it waited the limit out, and not much more
+    # it waited the limit out, and not much more: the clock is only read between rounds of a few thousand
+    # polls (each of which the hardware may hold for microseconds), so the give-up comes tens of milliseconds late
+    assert limit < cycles < 400_000_000
     assert L.status() == G.ERR_TIMEOUT
     assert L.status() == G.ERR_TIMEOUT                     # the word stays raised until the workspace is initialised
     G.griffin_workspace_init(L.ws)
