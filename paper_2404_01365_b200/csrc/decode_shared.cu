@@ -11,33 +11,35 @@
 // multicast) and runs ahead of the previous kernel on the stream and of the meeting point, two groups of
 // four consumer warps that take alternate row groups, a wrap-around counter in the workspace header as the
 // meeting point.  What differs is how a stage meets the vectors in mma.sync.m16n8k16:
-//   * the B operand's 8 columns are the (up to) 8 VECTORS, the A operand's 16 rows are 16 staged WEIGHT
-//     ROWS, so every product of the tile is used (the single-vector kernel uses the diagonal only).  A stage
-//     is a "row group": 8 gate rows and the 8 up rows of the same neurons (then C[j][n] and C[j+8][n] are the
-//     two factors of z[n][neuron j]), or 16 rows of W_1_hat (a block without a gate), or 16 rows of W_2_hat;
-//     long rows are cut into chunks of at most 2 KB, one chunk of all 16 rows per stage.
-//   * lane (g, t) of a warp (g = lane / 4, t = lane % 4) reads one 16-byte unit of rows g and g + 8 and of
-//     vector g: unit 4 b + t of block b (a block is 64 bytes of every row).  The unit's first four elements
-//     feed one MMA and the last four a second one; the MMA sums over K, so any assignment of elements to K
-//     positions works as long as all rows and all vectors agree, and here lane t supplies the same unit of
-//     each.  Staged rows and vectors lie at a pitch of 64 bytes modulo 128, so the two rows (or vectors)
-//     that a quarter warp reads together fall into different banks.
-//   * the four warps of a group share a stage by blocks; their partial 16 x 8 tiles meet in shared memory
+//   * the A operand's rows are the (up to) 8 VECTORS (rows 8..15 are zero), the B operand's 8 columns are 8
+//     staged WEIGHT ROWS, so every product of the upper half of the tile is used (the single-vector kernel
+//     uses a diagonal only).  A stage is a "row group": 4 gate rows and the 4 up rows of the same neurons, or
+//     8 rows of W_1_hat (a block without a gate), or 8 rows of W_2_hat; long rows are cut into chunks of at
+//     most 4 KB, one chunk of all 8 rows per stage.  (Measured: a bulk copy costs the SM 55-65 ns whatever its
+//     size, so 2 KB pieces cap the stream at 4.7-4.9 TB/s; with 16 weight rows on the A operand a stage of 4 KB
+//     pieces would be 64 KB and the ring too shallow, hence the weights sit on the 8-wide operand.)
+//   * lane (g, t) of a warp (g = lane / 4, t = lane % 4) reads one 16-byte unit of weight row g and of vector
+//     g: unit 4 b + t of block b (a block is 64 bytes of every row).  The unit's first four elements feed one
+//     MMA and the last four a second one; the MMA sums over K, so any assignment of elements to K positions
+//     works as long as all rows and all vectors agree, and here lane t supplies the same unit of each.  Staged
+//     rows and vectors lie at a pitch of 64 bytes modulo 128, so the two rows (or vectors) that a quarter warp
+//     reads together fall into different banks.  C[v][r] = vector v . row r sits in lane (v, r / 2).
+//   * the four warps of a group share a stage by blocks; their partial 8 x 8 tiles meet in shared memory
 //     after the last chunk of the row group, in a fixed order: results are bitwise reproducible.
 //   * the vectors stay in shared memory for a whole half (x, then z, which every CTA reads back from L2
-//     after the meeting).  When 8 vectors and a ring of four stages do not fit together, the chunks get
-//     shorter, and beyond that the batch is split into passes of fewer vectors.
+//     after the meeting), brought in by bulk copies.  When 8 vectors and a ring of four stages do not fit
+//     together, the chunks get shorter, and beyond that the batch is split into passes of fewer vectors.
 #include "decode_mma.cuh"
 
 namespace griffin {
 
-constexpr int SH_ROWS = 16;    // weight rows per stage = M of the MMA
-constexpr int SH_MAX_VEC = 8;  // vectors per pass = N of the MMA
+constexpr int SH_ROWS = 8;     // weight rows per stage = N of the MMA
+constexpr int SH_MAX_VEC = 8;  // vectors per pass (rows 0..7 of the MMA's M = 16)
 constexpr int SH_PAD = 64;     // bytes that shift consecutive rows / vectors to other banks
 constexpr int SH_BATCH = 4;    // blocks whose loads are issued before their MMAs
 constexpr int SH_THREADS = DEC_CONSUMERS + 2 * 32;  // 8 consumer warps + one producer warp per consumer group
 constexpr int SH_PART_FLOATS = SH_ROWS * SH_MAX_VEC;                          // one warp's partial tile
-constexpr int SH_PART_BYTES = 2 * 2 * DEC_GROUP_WARPS * SH_PART_FLOATS * 4;  // [group][parity][warp][16 x 8]
+constexpr int SH_PART_BYTES = 2 * 2 * DEC_GROUP_WARPS * SH_PART_FLOATS * 4;  // [group][parity][warp][8 x 8]
 constexpr int MODE_GATE_UP = 0, MODE_DOWN = 1, MODE_UP = 2;
 
 struct SharedPlan {
@@ -78,9 +80,9 @@ static inline size_t shared_smem_bytes(const SharedPlan &pl) {
 
 // Producer side of one half.  There are two producer warps, one per consumer group: consecutive row groups
 // belong to the two consumer groups in turn, each group has its own half of the ring, and producer warp `grp`
-// feeds that half with the row groups of its group.  Lane l < 16 copies row l of the row group (weights only).
+// feeds that half with the row groups of its group.  Lane l < 8 copies row l of the row group (weights only).
 // (Measured: a bulk copy costs the issuing warp 55-65 ns whatever its size, so one warp issuing the 16 copies
-// of every stage paces the whole kernel; two warps issue side by side.)
+// of every stage would pace the kernel; two warps issue side by side.)
 template <int MODE>
 __device__ __forceinline__ bool sh_produce_half(const DecodeParams &p, const SharedPlan &plan, const ShSmem &s, int grp,
                                                 RingPos &pos, uint32_t &rgc, int lane) {
@@ -104,7 +106,7 @@ __device__ __forceinline__ bool sh_produce_half(const DecodeParams &p, const Sha
             const int nrows = min(RG, r1 - g0);
             const uint8_t *src = nullptr;
             if (MODE == MODE_GATE_UP) {
-                if (lane < SH_ROWS && (lane & 7) < nrows) src = (lane < 8 ? wg : wu) + (size_t)(g0 + (lane & 7)) * row_bytes;
+                if (lane < SH_ROWS && (lane & 3) < nrows) src = (lane < 4 ? wg : wu) + (size_t)(g0 + (lane & 3)) * row_bytes;
             } else if (lane < nrows) {
                 src = (DOWN ? wd : wu) + (size_t)(g0 + lane) * row_bytes;
             }
@@ -154,9 +156,10 @@ __device__ __forceinline__ void sh_issue_vectors(const ShSmem &s, const SharedPl
     }
 }
 
-__device__ __forceinline__ void sh_mma_block(float (&acc)[4][4], int i, const uint4 &a0, const uint4 &a1, const uint4 &b) {
-    mma_bf16(acc[(2 * i) & 3], a0.x, a1.x, a0.y, a1.y, b.x, b.y);
-    mma_bf16(acc[(2 * i + 1) & 3], a0.z, a1.z, a0.w, a1.w, b.z, b.w);
+// One block: the lane's unit of its vector (A operand, rows 8..15 zero) against its unit of its weight row (B operand).
+__device__ __forceinline__ void sh_mma_block(float (&acc)[4][4], int i, const uint4 &v, const uint4 &w) {
+    mma_bf16(acc[(2 * i) & 3], v.x, 0u, v.y, 0u, w.x, w.y);
+    mma_bf16(acc[(2 * i + 1) & 3], v.z, 0u, v.w, 0u, w.z, w.w);
 }
 
 // Consumer side of one half (all 8 consumer warps).  Returns false after a give-up.
@@ -175,7 +178,6 @@ __device__ __forceinline__ bool sh_consume_half(const DecodeParams &p, const Sha
     const int g = lane >> 2, t = lane & 3;
     const int tig = tid - group * (DEC_GROUP_WARPS * 32);
     const bool has_vec = g < pl.n_vec;
-    const int row8 = 8 * pl.row_pitch / 16;  // units between rows g and g + 8 of a stage
     // this lane's unit of block 0: of its vector, and (added per stage) of row g
     const uint4 *const vec_lane = reinterpret_cast<const uint4 *>(s.vec + (size_t)(has_vec ? g : 0) * pl.vec_pitch) + t;
     const int row_lane_off = g * pl.row_pitch + t * 16;
@@ -206,84 +208,70 @@ __device__ __forceinline__ bool sh_consume_half(const DecodeParams &p, const Sha
                     const int units = min(cu, row_units - c * cu);
                     const int whole = units >> 2;          // blocks whose four units all exist
                     const int nblk = (units + 3) >> 2;     // ... and counting the cut one
-                    const uint4 *const a_lane =
+                    const uint4 *const w_lane =
                         reinterpret_cast<const uint4 *>(s.stages + (size_t)stage * pl.stage_bytes + row_lane_off);
                     const uint4 *const v_lane = vec_lane + c * cu;
                     // this warp's blocks: q, q + 4, q + 8, ...; a batch is four of them
 #pragma unroll 1
                     for (int b0 = q; b0 < nblk; b0 += DEC_GROUP_WARPS * SH_BATCH) {
-                        uint4 a0[SH_BATCH], a1[SH_BATCH], bv[SH_BATCH];
+                        uint4 wr[SH_BATCH], vr[SH_BATCH];
                         if (b0 + DEC_GROUP_WARPS * (SH_BATCH - 1) < whole) {  // warp-uniform: four whole blocks
 #pragma unroll
                             for (int i = 0; i < SH_BATCH; ++i) {
                                 const int u = 4 * (b0 + DEC_GROUP_WARPS * i);
-                                a0[i] = a_lane[u];
-                                a1[i] = a_lane[u + row8];
-                                bv[i] = has_vec ? v_lane[u] : zero;
+                                wr[i] = w_lane[u];
+                                vr[i] = has_vec ? v_lane[u] : zero;
                             }
 #pragma unroll
-                            for (int i = 0; i < SH_BATCH; ++i) sh_mma_block(acc, i, a0[i], a1[i], bv[i]);
+                            for (int i = 0; i < SH_BATCH; ++i) sh_mma_block(acc, i, vr[i], wr[i]);
                         } else {  // the chunk ends inside this batch: units past the end count as zeros
 #pragma unroll
                             for (int i = 0; i < SH_BATCH; ++i) {
                                 const int blk = b0 + DEC_GROUP_WARPS * i;
                                 const int u = 4 * blk;
                                 const bool in = u + t < units;  // (stale bytes behind a row's end could be NaN)
-                                a0[i] = in ? a_lane[u] : zero;
-                                a1[i] = in ? a_lane[u + row8] : zero;
-                                bv[i] = in && has_vec ? v_lane[u] : zero;
+                                wr[i] = in ? w_lane[u] : zero;
+                                vr[i] = in && has_vec ? v_lane[u] : zero;
                             }
 #pragma unroll
                             for (int i = 0; i < SH_BATCH; ++i)
-                                if (b0 + DEC_GROUP_WARPS * i < nblk) sh_mma_block(acc, i, a0[i], a1[i], bv[i]);  // warp-uniform
+                                if (b0 + DEC_GROUP_WARPS * i < nblk) sh_mma_block(acc, i, vr[i], wr[i]);  // warp-uniform
                         }
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&s.empty[stage]);
                 }
             }
-            // this warp's partial tile: lane (g, t) holds columns 2t, 2t+1 of rows g and g + 8
+            // this warp's partial tile: lane (g, t) holds C[vector g][rows 2t, 2t+1]
             float *const part = part_grp + parity * (DEC_GROUP_WARPS * SH_PART_FLOATS);
             {
-                float2 lo, hi;  // (a fixed order: results are reproducible)
+                float2 lo;  // (a fixed order: results are reproducible)
                 lo.x = (acc[0][0] + acc[1][0]) + (acc[2][0] + acc[3][0]);
                 lo.y = (acc[0][1] + acc[1][1]) + (acc[2][1] + acc[3][1]);
-                hi.x = (acc[0][2] + acc[1][2]) + (acc[2][2] + acc[3][2]);
-                hi.y = (acc[0][3] + acc[1][3]) + (acc[2][3] + acc[3][3]);
-                float *mine = part + q * SH_PART_FLOATS;
-                *reinterpret_cast<float2 *>(mine + g * SH_MAX_VEC + 2 * t) = lo;
-                *reinterpret_cast<float2 *>(mine + (g + 8) * SH_MAX_VEC + 2 * t) = hi;
+                *reinterpret_cast<float2 *>(part + q * SH_PART_FLOATS + g * SH_ROWS + 2 * t) = lo;
             }
             group_barrier(group);
             if (*s.abort) ok = false;
-            // thread (m, n) of the group finishes row m of the row group for vector n
-            const int m = tig >> 3, n = tig & 7;
-            if (ok && n < pl.n_vec) {
-                if (MODE == MODE_GATE_UP) {
-                    if (m < nrows) {  // (m < 8: threads 64..127 of the group have nothing to do)
-                        float a0 = 0.f, a1 = 0.f;
+            // thread (v, r) of the group's first 64 finishes row r of the row group for vector v
+            const int v = tig >> 3, r = tig & 7;
+            if (ok && tig < SH_MAX_VEC * SH_ROWS && v < pl.n_vec && r < nrows) {
+                float a0 = 0.f;
 #pragma unroll
-                        for (int w = 0; w < DEC_GROUP_WARPS; ++w) {
-                            a0 += part[w * SH_PART_FLOATS + m * SH_MAX_VEC + n];
-                            a1 += part[w * SH_PART_FLOATS + (m + 8) * SH_MAX_VEC + n];
-                        }
-                        const int j = g0 + m;
-                        if (p.seq[0].b_gate) a0 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[0].b_gate)[j]);
-                        if (p.seq[0].b_up) a1 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[0].b_up)[j]);
-                        zbits[(size_t)n * 2 * p.ldk + j] = __float2bfloat16_rn(sigma_rt(act, a0) * a1);
-                    }
-                } else if (m < nrows) {
-                    float a = 0.f;
+                for (int w = 0; w < DEC_GROUP_WARPS; ++w) a0 += part[w * SH_PART_FLOATS + v * SH_ROWS + r];
+                const int j = g0 + r;
+                if (MODE == MODE_GATE_UP) {  // (r < nrows <= 4: the gate rows; the up row of the same neuron is row r + 4)
+                    float a1 = 0.f;
 #pragma unroll
-                    for (int w = 0; w < DEC_GROUP_WARPS; ++w) a += part[w * SH_PART_FLOATS + m * SH_MAX_VEC + n];
-                    const int j = g0 + m;
-                    if (MODE == MODE_UP) {
-                        if (p.seq[0].b_up) a += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[0].b_up)[j]);
-                        zbits[(size_t)n * 2 * p.ldk + j] = __float2bfloat16_rn(sigma_rt(act, a));
-                    } else {
-                        if (p.b_down) a += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.b_down)[j]);
-                        static_cast<__nv_bfloat16 *>(p.y)[(size_t)n * p.d + j] = __float2bfloat16_rn(a);
-                    }
+                    for (int w = 0; w < DEC_GROUP_WARPS; ++w) a1 += part[w * SH_PART_FLOATS + v * SH_ROWS + r + 4];
+                    if (p.seq[0].b_gate) a0 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[0].b_gate)[j]);
+                    if (p.seq[0].b_up) a1 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[0].b_up)[j]);
+                    zbits[(size_t)v * 2 * p.ldk + j] = __float2bfloat16_rn(sigma_rt(act, a0) * a1);
+                } else if (MODE == MODE_UP) {
+                    if (p.seq[0].b_up) a0 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[0].b_up)[j]);
+                    zbits[(size_t)v * 2 * p.ldk + j] = __float2bfloat16_rn(sigma_rt(act, a0));
+                } else {
+                    if (p.b_down) a0 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.b_down)[j]);
+                    static_cast<__nv_bfloat16 *>(p.y)[(size_t)v * p.d + j] = __float2bfloat16_rn(a0);
                 }
             }
             parity ^= 1;
@@ -376,14 +364,10 @@ bool decode_shared_set(const DecodeParams &p) {
     return true;
 }
 
-#ifndef GRIFFIN_SH_CU
-#define GRIFFIN_SH_CU 128
-#endif
-#ifndef GRIFFIN_SH_STAGES
-#define GRIFFIN_SH_STAGES 6
-#endif
-
 // Chunk length and ring depth for n_vec vectors; false if even the smallest ring does not fit beside them.
+// Measured on B200 (Llama-2-7B shape): what counts is the bytes the ring keeps in flight (six stages of 32 KB:
+// 25.8 us per call, four: 28.4 us) and the size of a copy (4 KB pieces: 25.8 us, 2 KB: 29.5 us; a bulk copy
+// costs the SM 55-65 ns whatever its size); a prefetch of later rows into L2 made every case slower.
 static bool shared_plan(SharedPlan &pl, int d, int ldk, int k, int n_vec, int sms) {
     pl.n_vec = n_vec;
     pl.vec_pitch = ((max(d, ldk) * 2 + 127) & ~127) + SH_PAD;
@@ -392,21 +376,23 @@ static bool shared_plan(SharedPlan &pl, int d, int ldk, int k, int n_vec, int sm
     pl.row_units[1] = ldk / 8;
     pl.n_slices[0] = slices_for(k, sms);
     pl.n_slices[1] = slices_for(d, sms);
-    // (chunks shorter than 1 KB are only taken for a single vector: with more, two passes of half as many
-    // vectors at full speed beat one pass of short copies)
-    static const int cand[][2] = {{GRIFFIN_SH_CU, GRIFFIN_SH_STAGES}, {128, 6}, {128, 4}, {96, 6}, {96, 4}, {64, 8},
-                                  {64, 6},       {64, 4},  {48, 4},  {32, 4}};
+    // {longest chunk in units, stages}, best first: deep rings of long pieces, then shallower, then shorter
+    static const int cand[][2] = {{320, 6}, {256, 6}, {320, 4}, {256, 4}, {192, 6}, {192, 4}, {128, 6}, {128, 4}, {64, 4}, {32, 4}};
     for (const auto &c : cand) {
-        if (c[0] < 64 && n_vec > 1) continue;
-        pl.row_pitch = c[0] * 16 + SH_PAD;
+        // (chunks shorter than 2 KB are only taken for a single vector: with more, two passes of half as many
+        // vectors at full speed beat one pass of short copies)
+        if (c[0] < 128 && n_vec > 1) continue;
+        int longest = 0;
+        for (int h = 0; h < 2; ++h) {  // a row is cut into equal chunks, a multiple of 128 bytes each
+            pl.n_chunks[h] = (pl.row_units[h] + c[0] - 1) / c[0];
+            pl.cu[h] = ((pl.row_units[h] + pl.n_chunks[h] - 1) / pl.n_chunks[h] + 7) & ~7;
+            if (pl.cu[h] > c[0]) pl.cu[h] = c[0];  // (c[0] is itself a multiple of 8)
+            longest = max(longest, pl.cu[h]);
+        }
+        pl.row_pitch = longest * 16 + SH_PAD;
         pl.stage_bytes = SH_ROWS * pl.row_pitch;
         pl.n_stages = c[1];
-        if (shared_smem_bytes(pl) > 227 * 1024) continue;
-        for (int h = 0; h < 2; ++h) {
-            pl.n_chunks[h] = (pl.row_units[h] + c[0] - 1) / c[0];
-            pl.cu[h] = ((pl.row_units[h] + pl.n_chunks[h] - 1) / pl.n_chunks[h] + 7) & ~7;  // <= c[0], a multiple of 8
-        }
-        return true;
+        if (shared_smem_bytes(pl) <= 227 * 1024) return true;
     }
     return false;
 }
