@@ -395,6 +395,27 @@ class Job:
             out.append(G.compact_array([G.make_compact(wg, wu, wd, w.d_ff, w.d_ff)]))
         return out
 
+    def time_compact_neuron_major(self, reps=2):
+        """Median microseconds per (block, sequence) of the slicing step when the source of W_2_hat is the
+        neuron-major W_2^T (transposed here once per block, as at model load): the same compact sets, bit for bit,
+        from half the bytes of W_2."""
+        torch, G, st = self.torch, self.G, self.stack
+        nm = []
+        for fw in st.weights:
+            wg, wu, wd = fw._keep[0], fw._keep[1], fw._keep[2]
+            nm.append(G.make_weights_nm(wg, wu, wd.t().contiguous()))
+        us = []
+        for _ in range(reps + 1):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(self.stream)
+            for l in range(self.L):
+                for q in range(self.B):
+                    G.griffin_compact_experts_nm(st.desc, nm[l], st.idx[l, q], st.sets[l][q], st.ws)
+            e1.record(self.stream)
+            torch.cuda.synchronize()
+            us.append(e0.elapsed_time(e1) * 1e3 / (self.L * self.B))
+        return statistics.median(us[1:])
+
     def first_sequence_sets(self):
         return [self.G.compact_array(self.stack.sets[l][:1]) for l in range(self.L)]
 
@@ -420,6 +441,13 @@ def phase_report(job, ph_ms, peaks):
         rep["compact"] = {"us_per_block_and_sequence": c_us, "gbs": st.compact_bytes() / (c_us * 1e-6) / 1e9,
                           "frac_of_hbm": st.compact_bytes() / (c_us * 1e-6) / 1e9 / hbm}
     return rep
+
+
+def add_compact_nm(job, rep, peaks):
+    if rep.get("compact") is not None:
+        us = job.time_compact_neuron_major()
+        gbs = job.stack.compact_bytes() / (us * 1e-6) / 1e9
+        rep["compact"]["from_neuron_major_w_down"] = {"us_per_block_and_sequence": us, "gbs": gbs, "frac_of_hbm": gbs / peaks[0]}
 
 
 def timed_steps(job, steps, barrier):
@@ -460,6 +488,7 @@ def section_entry(w, B, keep, dev, args, peaks, with_dense):
     if job.stack.status() != job.G.OK:
         raise RuntimeError("device status word raised")
     rep = phase_report(job, median_phases(per_step), peaks)
+    add_compact_nm(job, rep, peaks)
     entry = {"workload": w.name, "B": B, "keep": keep, "k": job.k, "L": w.L, "S": w.S, "T": w.T, "steps": args.section_steps,
              "ms_per_step": total_ms / args.section_steps,
              "tokens_per_s_per_layer": B * w.T * w.L / (total_ms / args.section_steps / 1e3), "phases": rep}
@@ -589,6 +618,8 @@ def run_ours(args, w, keep):
         ms_per_step = total_ms / K
         tokens = world * B * T * L
         rep = phase_report(job, ph_ms, peaks)
+        if world == 1:
+            add_compact_nm(job, rep, peaks)
         dec = rep["decode"]
         traffic_key = f"{w.name}_B{B}_keep{keep}"
         line = {

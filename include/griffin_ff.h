@@ -226,6 +226,15 @@ griffin_status griffin_compact_experts(const griffin_ff_desc *desc, const griffi
                                        const int32_t *idx, const griffin_ff_compact *out,
                                        void *workspace /*may be NULL*/, void *stream);
 
+/* The same slicing from NEURON-MAJOR full weights (griffin_ff_weights_nm: w_down_t is the transpose of W_2,
+ * [d_ff, d]).  The result in `out` is bit for bit that of griffin_compact_experts on the row-major W_2; what
+ * differs is the traffic: the selected neurons' rows of W_2^T are contiguous, so only those k rows are read
+ * (and turned into the [d, ldk] layout of w_down_c on the way), where the row-major W_2 has to be read whole
+ * because at the usual keep ratios every 32-byte sector of it holds a selected column.  Same argument rules. */
+griffin_status griffin_compact_experts_nm(const griffin_ff_desc *desc, const griffin_ff_weights_nm *w,
+                                          const int32_t *idx, const griffin_ff_compact *out,
+                                          void *workspace /*may be NULL*/, void *stream);
+
 /* Generation phase (Eqs. 4, 5): for each of B sequences, with its own compact set,
  *   y[b] = W_2_hat (sigma(W_g_hat x[b] + b_g_hat) * (W_1_hat x[b] + b_1_hat)) + b_2
  * (without a gate: y[b] = W_2_hat sigma(W_1_hat x[b] + b_1_hat) + b_2).

@@ -35,7 +35,7 @@ EXPORTS = (
     "griffin_workspace_bytes", "griffin_workspace_init", "griffin_ff_prefill_score", "griffin_select_topk",
     "griffin_combine_scores", "griffin_compact_experts", "griffin_ff_decode", "griffin_check_device_status",
     "griffin_ff_decode_static", "griffin_ff_decode_indexed", "griffin_ff_prefill_score_chunk",
-    "griffin_kernel_launches", "griffin_ff_decode_static_status",
+    "griffin_kernel_launches", "griffin_ff_decode_static_status", "griffin_compact_experts_nm",
 )
 
 
@@ -101,6 +101,8 @@ def load(path=None):
     lib.griffin_combine_scores.argtypes = [vp, C.POINTER(i32), i32, i32, vp, vp]
     lib.griffin_compact_experts.restype = C.c_int
     lib.griffin_compact_experts.argtypes = [C.POINTER(FFDesc), C.POINTER(FFWeights), vp, C.POINTER(FFCompact), vp, vp]
+    lib.griffin_compact_experts_nm.restype = C.c_int
+    lib.griffin_compact_experts_nm.argtypes = [C.POINTER(FFDesc), C.POINTER(FFWeightsNM), vp, C.POINTER(FFCompact), vp, vp]
     lib.griffin_ff_decode.restype = C.c_int
     lib.griffin_ff_decode.argtypes = [C.POINTER(FFDesc), i32, C.POINTER(FFCompact), vp, vp, vp, vp, sz, u32, vp]
     lib.griffin_ff_decode_indexed.restype = C.c_int
@@ -236,6 +238,12 @@ def griffin_combine_scores(score, prompt_len, out, stream=None):
 def griffin_compact_experts(desc, weights, idx, out, ws=None, stream=None):
     _check(load().griffin_compact_experts(C.byref(desc), C.byref(weights), _ptr(idx), C.byref(out), _ptr(ws),
                                           _stream(stream)), "griffin_compact_experts")
+
+
+def griffin_compact_experts_nm(desc, weights_nm, idx, out, ws=None, stream=None):
+    """The same compact set from neuron-major full weights (w_down_t = W_2 transposed)."""
+    _check(load().griffin_compact_experts_nm(C.byref(desc), C.byref(weights_nm), _ptr(idx), C.byref(out), _ptr(ws),
+                                             _stream(stream)), "griffin_compact_experts_nm")
 
 
 def compact_array(sets):

@@ -207,6 +207,20 @@ griffin_status griffin_compact_experts(const griffin_ff_desc *desc, const griffi
     return launch_compact(desc, w, idx, out, workspace, static_cast<cudaStream_t>(stream));
 }
 
+griffin_status griffin_compact_experts_nm(const griffin_ff_desc *desc, const griffin_ff_weights_nm *w, const int32_t *idx,
+                                          const griffin_ff_compact *out, void *workspace, void *stream) {
+    griffin_status st = check_desc(desc);
+    if (st != GRIFFIN_OK) return st;
+    if (w == nullptr || out == nullptr || idx == nullptr) return GRIFFIN_ERR_INVALID_ARG;
+    if (w->w_up == nullptr || w->w_down_t == nullptr) return GRIFFIN_ERR_INVALID_ARG;
+    if (!gate_args_ok(desc, w->w_gate, w->b_gate)) return GRIFFIN_ERR_INVALID_ARG;
+    if (!aligned16(w->w_gate) || !aligned16(w->w_up) || !aligned16(w->w_down_t)) return GRIFFIN_ERR_ALIGNMENT;
+    st = check_compact(desc, out);
+    if (st != GRIFFIN_OK) return st;
+    if (out->ldk != griffin_compact_ldk(out->k)) return GRIFFIN_ERR_INVALID_ARG;
+    return launch_compact_nm(desc, w, idx, out, workspace, static_cast<cudaStream_t>(stream));
+}
+
 griffin_status griffin_ff_decode(const griffin_ff_desc *desc, int32_t B, const griffin_ff_compact *sets,
                                  const void *b_down, const void *x, void *y, void *workspace, size_t ws_bytes,
                                  uint32_t flags, void *stream) {

@@ -44,6 +44,9 @@ griffin_status launch_combine_scores(const float *score, const int32_t *prompt_l
 griffin_status launch_compact(const griffin_ff_desc *desc, const griffin_ff_weights *w, const int32_t *idx,
                               const griffin_ff_compact *out, void *ws, cudaStream_t stream);
 
+griffin_status launch_compact_nm(const griffin_ff_desc *desc, const griffin_ff_weights_nm *w, const int32_t *idx,
+                                 const griffin_ff_compact *out, void *ws, cudaStream_t stream);
+
 // Carve-up of the workspace behind its header for the prompt-phase path.
 struct PrefillScratch {
     size_t z_off, zf_off, rowsq_off, inv_off, colpart_off, ypart_off, total;  // byte offsets from the scratch base

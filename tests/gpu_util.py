@@ -80,6 +80,20 @@ class GpuLayer:
         G.griffin_compact_experts(self.desc, self.weights, e, cs, self.ws)
         return cs
 
+    def compact_nm(self, e):
+        """The same compact set from neuron-major weights (W_2 transposed once, as at model load)."""
+        self._neuron_major()
+        k = e.numel()
+        cs = G.alloc_compact(self.desc, k, dev(), self.tdtype, with_bias=self.t["bu"] is not None)
+        G.griffin_compact_experts_nm(self.desc, self.weights_nm, e, cs, self.ws)
+        return cs
+
+    def _neuron_major(self):
+        if not hasattr(self, "weights_nm"):
+            self.t["wd_t"] = self.t["wd"].t().contiguous()
+            self.weights_nm = G.make_weights_nm(self.t["wg"], self.t["wu"], self.t["wd_t"], self.t["bg"], self.t["bu"],
+                                                self.t["bd"])
+
     def dense_set(self):
         """The full weights viewed as a compact set with E = all neurons."""
         return G.make_compact(self.t["wg"], self.t["wu"], self.t["wd"], self.d_ff, self.d_ff, self.t["bg"], self.t["bu"])
@@ -92,10 +106,7 @@ class GpuLayer:
 
     def decode_indexed(self, idx, x, flags=0):
         """Pruned FF straight from the full weights (W_2 transposed once, as at model load)."""
-        if not hasattr(self, "weights_nm"):
-            self.t["wd_t"] = self.t["wd"].t().contiguous()
-            self.weights_nm = G.make_weights_nm(self.t["wg"], self.t["wu"], self.t["wd_t"], self.t["bg"], self.t["bu"],
-                                                self.t["bd"])
+        self._neuron_major()
         x = x.to(dev()).contiguous()
         y = torch.empty_like(x)
         G.griffin_ff_decode_indexed(self.desc, self.weights_nm, idx, x, y, self.ws, flags)

@@ -65,15 +65,22 @@ def test_combine_scores():
 
 # ------------------------------------------------------------- compaction ---
 
+@pytest.mark.parametrize("source", ["row_major", "neuron_major"])
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("d,d_ff,k", [(64, 96, 37), (256, 688, 344), (1024, 2816, 1408), (520, 1032, 1032),
-                                      (72, 200, 1)])
-def test_compact_exact(dtype, d, d_ff, k):
+                                      (72, 200, 1), (136, 30008, 15001),   # rows of W_2 too long for shared memory
+                                      (4096, 11008, 5504)])
+def test_compact_exact(dtype, d, d_ff, k, source):
+    """Slicing (Section 4.2) is indexing: raw-bit equality with W[E, :] and W[:, E], from the row-major W_2 and
+    from its transpose.  The index list is unsorted for the small shapes and starts at an address that is not a
+    multiple of 8 bytes when k is odd."""
     L, host = make_layer(d, d_ff, dtype, bias=True, seed=d + k)
     rs = np.random.default_rng(k)
-    e_np = np.sort(rs.choice(d_ff, size=k, replace=False)).astype(np.int32)
-    e = torch.from_numpy(e_np).to(dev())
-    cs = L.compact(e)
+    e_np = rs.choice(d_ff, size=k, replace=False).astype(np.int32)
+    if d_ff > 1100:
+        e_np = np.sort(e_np)
+    e = torch.from_numpy(np.concatenate([[0], e_np]).astype(np.int32)).to(dev())[1:]   # 4 bytes off an aligned address
+    cs = L.compact(e) if source == "row_major" else L.compact_nm(e)
     assert L.status() == G.OK
     g, u, dn, bg, bu = cs._keep
     ref = O.compact_experts(e_np, host["wg"].numpy() if dtype == "f32" else host["wg"].view(torch.int16).numpy(),
@@ -89,13 +96,15 @@ def test_compact_exact(dtype, d, d_ff, k):
     assert np.array_equal(bits(bg), ref["b_gate"]) and np.array_equal(bits(bu), ref["b_up"])
 
 
-def test_compact_out_of_range_index_is_reported_not_read():
-    L, host = make_layer(64, 96, "bf16")
-    e = torch.tensor([0, 5, 96, 7], dtype=torch.int32, device=dev())   # 96 is out of range
-    cs = L.compact(e)
+@pytest.mark.parametrize("source,d_ff", [("row_major", 96), ("neuron_major", 96), ("row_major", 40000)])
+def test_compact_out_of_range_index_is_reported_not_read(source, d_ff):
+    L, host = make_layer(64, d_ff, "bf16")
+    e = torch.tensor([0, 5, d_ff, 7, -1], dtype=torch.int32, device=dev())   # d_ff and -1 are out of range
+    cs = L.compact(e) if source == "row_major" else L.compact_nm(e)
     assert L.status() == G.ERR_INVALID_ARG
-    g = cs._keep[0].cpu()
-    assert torch.all(g[2] == 0) and torch.equal(g[1], host["wg"][5])
+    g, dn = cs._keep[0].cpu(), cs._keep[2].cpu()
+    assert torch.all(g[2] == 0) and torch.all(g[4] == 0) and torch.equal(g[1], host["wg"][5])
+    assert torch.all(dn[:, 2] == 0) and torch.all(dn[:, 4:] == 0) and torch.equal(dn[:, 3], host["wd"][:, 7])
     G.griffin_workspace_init(L.ws)
     assert L.status() == G.OK
 
