@@ -26,127 +26,11 @@
 // column is a neuron of its own.
 //
 // Every wait is bounded; after a give-up the CTA still frees its TMEM before it returns.
-#include "common.cuh"
-#include "launch.h"
-#include "prefill_tc.h"
-#include "tc_common.cuh"
+#include <stdlib.h>
+
+#include "prefill_tc.cuh"
 
 namespace griffin {
-
-// sigma with the fast division (2 ulp) for the epilogues: a warp there pays most of every dependent
-// latency in full, and the IEEE division is a long chain (measured: 2 us of 142 on the bench shape).
-__device__ __forceinline__ float sigma_fast_rt(int act, float t) {
-    switch (act) {
-        case GRIFFIN_ACT_SWIGLU: return __fdividef(t, 1.0f + __expf(-t));
-        case GRIFFIN_ACT_GEGLU_TANH: {
-            const float inner = 0.7978845608028654f * (t + 0.044715f * t * t * t);
-            const float th = 1.0f - __fdividef(2.0f, __expf(2.0f * inner) + 1.0f);
-            return 0.5f * t * (1.0f + th);
-        }
-        case GRIFFIN_ACT_GEGLU_ERF: return sigma<GRIFFIN_ACT_GEGLU_ERF>(t);
-        default: return fmaxf(t, 0.0f);
-    }
-}
-
-constexpr int TC_BM = 128;        // rows (tokens) per tile
-constexpr int TC_BK = 64;         // K per stage: 64 bf16 = one 128-byte swizzle row
-constexpr int TC_EPI_WARPS = 8;   // two per TMEM lane quarter
-constexpr int TC_THREADS = 64 + 32 * TC_EPI_WARPS;
-#ifndef GRIFFIN_TC_STAGES
-#define GRIFFIN_TC_STAGES 4
-#endif
-constexpr int TC_STAGES = GRIFFIN_TC_STAGES;
-
-struct TcParams {
-    int S;            // rows of the left operand and of the output
-    int n_total;      // columns of the output (d_ff for DUAL, d otherwise)
-    int K;            // reduction length (d for DUAL, d_ff otherwise), multiple of 64
-    int m_tiles, n_tiles;
-    const __nv_bfloat16 *bias0, *bias1;  // DUAL: b_gate, b_up; otherwise b_down, unused (may be null)
-    __nv_bfloat16 *out;                  // Z or Y, [S, n_total]
-    float *zf;                           // DUAL: Z in fp32, [S, n_total]
-    float *rowsq;                        // DUAL: [S, 2 n_tiles] partial sums of squares of the fp32 rows (two column halves per tile)
-    int splits;                          // K splits (1 unless the plain GEMM has too few tiles)
-    float *part;                         // splits > 1: fp32 partial outputs [splits, S, n_total]
-    int act;
-    void *ws;
-    // Tiles 256 columns wide only: tiles from tail_first on are cut along K into tail_ks parts (tail_ks = 1:
-    // none is), whose raw accumulators (fp32; gate | up in the first GEMM) go to tail_part [part][128 rows][256 columns]
-    int tail_first, tail_ks;
-    float *tail_part;
-    int gated;  // first GEMM: 1 = gate | up tiles of 128 neurons, 0 = 256 neurons of W_1 (no gate)
-};
-
-// Work item -> (row block m, column block n, K blocks [kb0, kb1), index of the cut tile's part or -1).
-// Uniform K splits (the down projection) number the items split-major; the cut tiles of the first GEMM
-// follow the whole ones.
-struct TcItem {
-    int m, n, sp, kb0, kb1, part;
-};
-__device__ __forceinline__ TcItem tc_item(const TcParams &p, int item, int kb_total) {
-    TcItem t;
-    const int tiles = p.m_tiles * p.n_tiles;
-    int tile = item, ks = p.splits;
-    t.sp = 0;
-    t.part = -1;
-    if (p.tail_ks > 1) {
-        ks = 1;
-        if (item >= p.tail_first) {
-            const int j = item - p.tail_first;
-            ks = p.tail_ks;
-            tile = p.tail_first + j / ks;
-            t.sp = j - (j / ks) * ks;
-            t.part = j;
-        }
-    } else if (ks > 1) {
-        t.sp = item / tiles;
-        tile = item - t.sp * tiles;
-    }
-    t.m = tile % p.m_tiles;  // tiles sharing weights are neighbours
-    t.n = tile / p.m_tiles;
-    t.kb0 = t.sp * kb_total / ks;
-    t.kb1 = (t.sp + 1) * kb_total / ks;
-    return t;
-}
-
-// Output staging of the epilogue warps.  A thread of an epilogue warp holds one ROW of the tile, so a
-// store straight from its registers scatters every instruction over 32 rows, 16 bytes each; those
-// requests queue behind the TMA loads on the SM's way to L2 and made the epilogue of a tile take
-// 18-23 us.  Instead the warp passes its 32 rows, 64 bytes of each at a time, through a small buffer
-// of its own in shared memory and writes them back so that an instruction covers 8 rows x 64
-// contiguous bytes.
-constexpr int TC_STG_PITCH = 80;                  // 64 data bytes + 16 of padding per staged row
-constexpr int TC_STG_BYTES = 32 * TC_STG_PITCH;   // per epilogue warp
-// v: this thread's 64 bytes of its row; g: global address of the block's first row at the wanted
-// column; rows at and beyond rows_live are not written.
-__device__ __forceinline__ void store_rows64(uint8_t *stg, const uint4 (&v)[4], void *g, size_t row_pitch_bytes,
-                                             int rows_live, int lane) {
-    uint4 *mine = reinterpret_cast<uint4 *>(stg + lane * TC_STG_PITCH);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) mine[i] = v[i];
-    __syncwarp();
-    const int piece = lane & 3, r0 = lane >> 2;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const int r = r0 + 8 * j;
-        const uint4 t = *reinterpret_cast<const uint4 *>(stg + r * TC_STG_PITCH + piece * 16);
-        if (r < rows_live) *reinterpret_cast<uint4 *>(static_cast<uint8_t *>(g) + (size_t)r * row_pitch_bytes + piece * 16) = t;
-    }
-    __syncwarp();
-}
-// 32 fp32 values of this thread's row (128 bytes) as two such passes.
-__device__ __forceinline__ void store_rows_f32x32(uint8_t *stg, const float (&a)[32], float *g, size_t row_pitch_bytes,
-                                                  int rows_live, int lane) {
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        uint4 v[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-            v[i] = make_uint4(__float_as_uint(a[16 * h + 4 * i]), __float_as_uint(a[16 * h + 4 * i + 1]),
-                              __float_as_uint(a[16 * h + 4 * i + 2]), __float_as_uint(a[16 * h + 4 * i + 3]));
-        store_rows64(stg, v, g + 16 * h, row_pitch_bytes, rows_live, lane);
-    }
-}
 
 struct TcSmem {
     uint8_t *stages;
@@ -157,7 +41,6 @@ struct TcSmem {
 };
 constexpr size_t TC_TAIL_BYTES = (2 * TC_STAGES + 4) * sizeof(uint64_t) + 16 + TC_EPI_WARPS * TC_STG_BYTES;
 
-constexpr int TC_PLAIN = 0, TC_GATED = 1, TC_WIDE = 2;
 template <int KIND, int BN>
 __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant__ CUtensorMap map_a,
                                                            const __grid_constant__ CUtensorMap map_b0,
@@ -271,7 +154,6 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
         // ---------------- epilogue (warps 2..9) ----------------
         const int wq = warp & 3;                 // the TMEM lane quarter this warp may read
         const int half = (warp - 2) >> 2;        // which half of the tile's columns this warp takes
-        const int row_in_tile = wq * 32 + lane;  // one output row per thread
         uint8_t *const stg = s.stg + (warp - 2) * TC_STG_BYTES;
         uint32_t tcount = 0;
         for (int tile = blockIdx.x; tile < n_tiles_total; tile += gridDim.x, ++tcount) {
@@ -281,111 +163,8 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
             // (256 threads wait here for most of a tile's main loop: they sleep between polls)
             if (!wait_or_abort_relaxed(&s.acc_full[acc], (tcount >> 1) & 1, s.abort, p.ws, 23)) break;
             tc_fence_after_sync();
-            const int row = m * TC_BM + row_in_tile;
-            const bool live = row < p.S;
-            const int row0 = m * TC_BM + wq * 32;  // first row of this warp's block of 32
-            const int rows_live = p.S - row0;      // rows of the block that exist (may be <= 0 or > 32)
             const uint32_t taddr = tmem_base + ((uint32_t)(wq * 32) << 16) + (uint32_t)(acc * NT);
-            if ((DUAL || BN == 256) && ti.part >= 0) {
-                // a part of a cut tile: the raw accumulators leave in fp32 (gate | up); the finishing
-                // kernel adds the parts and does what the epilogue below does
-                float *dst = p.tail_part + ((size_t)ti.part * TC_BM + wq * 32) * 256;
-#pragma unroll 1
-                for (int c = half * 128; c < half * 128 + 128; c += 32) {
-                    float a[32];
-                    tmem_ld32(taddr + c, a);
-                    store_rows_f32x32(stg, a, dst + c, 256 * sizeof(float), 32, lane);
-                }
-            } else if (KIND == TC_WIDE) {
-                // no gate: every one of the 256 accumulator columns is a neuron, Z = sigma(acc + b_1)
-                float sq = 0.f;
-#pragma unroll 1
-                for (int c = half * 128; c < half * 128 + 128; c += 32) {
-                    float u[32];
-                    tmem_ld32(taddr + c, u);
-                    const int col = n * 256 + c;
-                    uint32_t packed[16];
-#pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        float u0 = u[i], u1 = u[i + 1];
-                        if (p.bias1) { u0 += __bfloat162float(p.bias1[col + i]); u1 += __bfloat162float(p.bias1[col + i + 1]); }
-                        const float z0 = sigma_fast_rt(p.act, u0), z1 = sigma_fast_rt(p.act, u1);
-                        u[i] = z0;
-                        u[i + 1] = z1;
-                        sq = fmaf(z0, z0, sq);
-                        sq = fmaf(z1, z1, sq);
-                        const __nv_bfloat162 h = __floats2bfloat162_rn(z0, z1);
-                        packed[i >> 1] = *reinterpret_cast<const uint32_t *>(&h);
-                    }
-                    {
-                        uint4 pk[4];
-#pragma unroll
-                        for (int v = 0; v < 4; ++v)
-                            pk[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
-                        store_rows64(stg, pk, p.out + (size_t)row0 * p.n_total + col, (size_t)p.n_total * 2, rows_live, lane);
-                        store_rows_f32x32(stg, u, p.zf + (size_t)row0 * p.n_total + col, (size_t)p.n_total * 4, rows_live, lane);
-                    }
-                }
-                if (live) p.rowsq[(size_t)row * (2 * p.n_tiles) + 2 * n + half] = sq;
-            } else if (DUAL) {
-                float sq = 0.f;
-#pragma unroll 1
-                for (int c = half * 64; c < half * 64 + 64; c += 32) {
-                    float g[32], u[32];
-                    tmem_ld32x2(taddr + c, taddr + 128 + c, g, u);
-                    const int col = n * 128 + c;
-                    uint32_t packed[16];
-#pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        float g0 = g[i], g1 = g[i + 1], u0 = u[i], u1 = u[i + 1];
-                        if (p.bias0) { g0 += __bfloat162float(p.bias0[col + i]); g1 += __bfloat162float(p.bias0[col + i + 1]); }
-                        if (p.bias1) { u0 += __bfloat162float(p.bias1[col + i]); u1 += __bfloat162float(p.bias1[col + i + 1]); }
-                        const float z0 = sigma_fast_rt(p.act, g0) * u0, z1 = sigma_fast_rt(p.act, g1) * u1;
-                        g[i] = z0;
-                        g[i + 1] = z1;
-                        sq = fmaf(z0, z0, sq);
-                        sq = fmaf(z1, z1, sq);
-                        const __nv_bfloat162 h = __floats2bfloat162_rn(z0, z1);
-                        packed[i >> 1] = *reinterpret_cast<const uint32_t *>(&h);
-                    }
-                    {
-                        uint4 pk[4];
-#pragma unroll
-                        for (int v = 0; v < 4; ++v)
-                            pk[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
-                        store_rows64(stg, pk, p.out + (size_t)row0 * p.n_total + col, (size_t)p.n_total * 2, rows_live, lane);
-                        store_rows_f32x32(stg, g, p.zf + (size_t)row0 * p.n_total + col, (size_t)p.n_total * 4, rows_live, lane);
-                    }
-                }
-                if (live) p.rowsq[(size_t)row * (2 * p.n_tiles) + 2 * n + half] = sq;
-            } else {
-#pragma unroll 1
-                for (int c = half * (BN / 2); c < half * (BN / 2) + BN / 2; c += 32) {
-                    float a[32];
-                    tmem_ld32(taddr + c, a);
-                    const int col = n * BN + c;
-                    if (p.splits > 1) {  // partial sums leave in fp32; bias and rounding happen in the reduction
-                        store_rows_f32x32(stg, a, p.part + ((size_t)sp * p.S + row0) * p.n_total + col,
-                                          (size_t)p.n_total * 4, rows_live, lane);
-                        continue;
-                    }
-                    uint32_t packed[16];
-#pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        float y0 = a[i], y1 = a[i + 1];
-                        if (p.bias0) { y0 += __bfloat162float(p.bias0[col + i]); y1 += __bfloat162float(p.bias0[col + i + 1]); }
-                        const __nv_bfloat162 h = __floats2bfloat162_rn(y0, y1);
-                        packed[i >> 1] = *reinterpret_cast<const uint32_t *>(&h);
-                    }
-                    {
-                        uint4 pk[4];
-#pragma unroll
-                        for (int v = 0; v < 4; ++v)
-                            pk[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
-                        store_rows64(stg, pk, p.out + (size_t)row0 * p.n_total + col, (size_t)p.n_total * 2, rows_live, lane);
-                    }
-                }
-            }
+            tc_epilogue_item<KIND, BN>(p, m, n, sp, ti.part, taddr, stg, wq, half, lane);
             tc_fence_before_sync();  // this warp's TMEM reads are done
             __syncwarp();
             if (lane == 0) mbar_arrive(&s.acc_empty[acc]);
@@ -665,8 +444,19 @@ griffin_status launch_prefill_tc(const griffin_ff_desc *desc, const griffin_ff_w
     gemm1_tail_plan(S, d, p.n_tiles, &p.tail_first, &p.tail_ks);
     p.tail_part = ypart;  // (the down projection's partials use the same scratch, later)
     *n_col_tiles = 2 * p.n_tiles;  // partial row sums per token: one per tile and column half
-    griffin_status st = gated ? launch_tc<TC_GATED, 128>(mx, mg, mu, p, sms, stream)
-                              : launch_tc<TC_WIDE, 128>(mx, mg, mu, p, sms, stream);
+    // An even number of 128-token tiles: pairs of CTAs on tiles of 256 tokens, each staging half of the weight
+    // tile (the environment variable GRIFFIN_TC_NO_PAIRS, set to anything, keeps one CTA per tile).
+    static const bool no_pairs = getenv("GRIFFIN_TC_NO_PAIRS") != nullptr;
+    const bool pairs = !no_pairs && m_tiles % 2 == 0 && sms >= 2;
+    griffin_status st;
+    if (pairs) {
+        TcParams p2 = p;
+        p2.m_tiles = m_tiles / 2;
+        p2.tail_first = p.tail_first / 2;  // (a whole number of pairs: the plan cuts a multiple of m_tiles tiles... of an even count)
+        st = launch_tc_pairs(gated ? TC_GATED : TC_WIDE, mx, mg, mu, p2, sms, stream);
+    } else {
+        st = gated ? launch_tc<TC_GATED, 128>(mx, mg, mu, p, sms, stream) : launch_tc<TC_WIDE, 128>(mx, mg, mu, p, sms, stream);
+    }
     if (st == GRIFFIN_OK && p.tail_ks > 1) {
         dual_tail_finish_kernel<<<(p.m_tiles * p.n_tiles - p.tail_first) * (TC_BM / 4), 128, 0, stream>>>(p);
         count_launches(1);
@@ -696,8 +486,17 @@ griffin_status launch_prefill_tc(const griffin_ff_desc *desc, const griffin_ff_w
     gemm2_tail_plan(S, d, d_ff, &q.tail_first, &q.tail_ks);
     q.tail_part = ypart;
     if (q.tail_ks > 1) q.bias0 = static_cast<const __nv_bfloat16 *>(w->b_down);
-    st = bn == 256 ? launch_tc<TC_PLAIN, 256>(mz, md, md, q, sms, stream)
-                   : launch_tc<TC_PLAIN, 128>(mz, md, md, q, sms, stream);
+    if (pairs && bn == 256) {
+        CUtensorMap md2;  // the same matrix in boxes of 128 rows: each CTA of a pair stages half of a 256-wide tile
+        if (!make_map(&md2, w->w_down, d, d_ff, 128)) return GRIFFIN_ERR_CUDA;
+        TcParams q2 = q;
+        q2.m_tiles = m_tiles / 2;
+        q2.tail_first = q.tail_first / 2;
+        st = launch_tc_pairs(TC_PLAIN, mz, md2, md2, q2, sms, stream);
+    } else {
+        st = bn == 256 ? launch_tc<TC_PLAIN, 256>(mz, md, md, q, sms, stream)
+                       : launch_tc<TC_PLAIN, 128>(mz, md, md, q, sms, stream);
+    }
     if (st == GRIFFIN_OK && q.tail_ks > 1) {
         plain_tail_finish_kernel<<<(q.m_tiles * q.n_tiles - q.tail_first) * (TC_BM / 4), 128, 0, stream>>>(q);
         count_launches(1);
