@@ -247,7 +247,10 @@ griffin_status griffin_compact_experts_nm(const griffin_ff_desc *desc, const gri
  * y [B, d] out.  1 <= B <= GRIFFIN_MAX_BATCH, d <= GRIFFIN_MAX_D.  flags: GRIFFIN_DECODE_*.
  * The activations z_hat [B, ldk] pass through the workspace (4 bytes per entry).  With bf16
  * storage the call is one kernel whose CTAs (one per SM) meet half-way through a counter in
- * the workspace header: run it on a GPU whose SMs it can all occupy. */
+ * the workspace header: run it on a GPU whose SMs it can all occupy.  (The call asks the
+ * runtime whether one CTA per SM can be resident and returns GRIFFIN_ERR_UNSUPPORTED when not;
+ * SMs held by other work at the time can still make the bounded wait run out:
+ * GRIFFIN_ERR_TIMEOUT from griffin_check_device_status, y undefined.) */
 griffin_status griffin_ff_decode(const griffin_ff_desc *desc, int32_t B,
                                  const griffin_ff_compact *sets /*host*/, const void *b_down,
                                  const void *x, void *y, void *workspace, size_t ws_bytes,

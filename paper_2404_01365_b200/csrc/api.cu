@@ -52,6 +52,31 @@ cudaError_t ensure_dynamic_smem(const void *fn, size_t bytes) {
     return e;
 }
 
+bool grid_can_meet(const void *fn, int threads, size_t smem, int grid) {
+    // remembers, per (device, kernel, shared memory), how many CTAs an SM holds
+    struct Entry {
+        const void *fn;
+        int dev;
+        size_t smem;
+        int per_sm;
+    };
+    static Entry table[128];
+    static int n_entries = 0;
+    static std::mutex table_mutex;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    const int sms = device_sm_count();
+    if (sms <= 0) return false;
+    std::lock_guard<std::mutex> lock(table_mutex);
+    for (int i = 0; i < n_entries; ++i)
+        if (table[i].fn == fn && table[i].dev == dev && table[i].smem == smem)
+            return (long long)table[i].per_sm * sms >= grid;
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, threads, smem) != cudaSuccess) return false;
+    if (n_entries < 128) table[n_entries++] = Entry{fn, dev, smem, per_sm};
+    return (long long)per_sm * sms >= grid;
+}
+
 }  // namespace griffin
 
 static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }

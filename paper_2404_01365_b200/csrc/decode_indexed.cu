@@ -498,6 +498,7 @@ griffin_status launch_decode_indexed(const griffin_ff_desc *desc, int B, const g
     const size_t smem = (size_t)p.n_stages * pl.stage_bytes + idx_fixed_smem(p.d, p.n_stages);
     if (smem > 227 * 1024) return GRIFFIN_ERR_UNSUPPORTED;
     if (ensure_dynamic_smem(fn, smem) != cudaSuccess) return GRIFFIN_ERR_CUDA;
+    if (!grid_can_meet(fn, DEC_THREADS, smem, grid)) return GRIFFIN_ERR_UNSUPPORTED;
     int act = act_sigma(desc->act);
     void *args[] = {&p, &act};
     const bool overlap = (flags & GRIFFIN_DECODE_OVERLAP_WEIGHT_PREFETCH) != 0;

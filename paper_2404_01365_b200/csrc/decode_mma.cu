@@ -365,6 +365,7 @@ griffin_status decode_bf16_mma(DecodeParams &p, int act, bool gated, uint32_t fl
     if (smem > 227 * 1024) return GRIFFIN_ERR_UNSUPPORTED;
     const void *fn = gated ? (const void *)decode_fused_kernel<true> : (const void *)decode_fused_kernel<false>;
     if (ensure_dynamic_smem(fn, smem) != cudaSuccess) return GRIFFIN_ERR_CUDA;
+    if (!grid_can_meet(fn, DEC_THREADS, smem, grid)) return GRIFFIN_ERR_UNSUPPORTED;
     void *args[] = {&p, &fp, &act};
     if (launch_maybe_overlapped(fn, dim3(grid), dim3(DEC_THREADS), smem, stream, overlap, args) != cudaSuccess)
         return GRIFFIN_ERR_CUDA;

@@ -419,6 +419,7 @@ griffin_status decode_bf16_shared(DecodeParams &p, int act, bool gated, uint32_t
         ql.n_vec = q.B;
         const size_t smem = shared_smem_bytes(pl);
         if (ensure_dynamic_smem(fn, smem) != cudaSuccess) return GRIFFIN_ERR_CUDA;
+        if (!grid_can_meet(fn, SH_THREADS, smem, sms)) return GRIFFIN_ERR_UNSUPPORTED;
         void *args[] = {&q, &ql, &act};
         // every CTA of the grid must be able to run at the same time (they meet half-way): one per SM
         if (launch_maybe_overlapped(fn, dim3(sms), dim3(SH_THREADS), smem, stream, overlap, args) != cudaSuccess)

@@ -650,6 +650,7 @@ griffin_status decode_bf16_tc(DecodeParams &p, int act, uint32_t flags, cudaStre
     // every CTA of the grid must be able to run at the same time (they meet half-way): one per SM
     const void *fn = shared ? (const void *)decode_tc_kernel<true> : (const void *)decode_tc_kernel<false>;
     if (ensure_dynamic_smem(fn, smem) != cudaSuccess) return GRIFFIN_ERR_CUDA;
+    if (!grid_can_meet(fn, DTC_THREADS, smem, sms)) return GRIFFIN_ERR_UNSUPPORTED;
     void *args[] = {&p, &pl, &act};
     if (launch_maybe_overlapped(fn, dim3(sms), dim3(DTC_THREADS), smem, stream, overlap, args) != cudaSuccess)
         return GRIFFIN_ERR_CUDA;

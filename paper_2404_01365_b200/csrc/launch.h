@@ -19,6 +19,11 @@ void count_launches(int n);
 // Raises the opt-in dynamic shared memory limit of `fn` on the current device when needed.
 cudaError_t ensure_dynamic_smem(const void *fn, size_t bytes);
 
+// Whether a grid of `grid` CTAs of this kernel, with this many threads and this much dynamic shared memory, can be
+// resident on the current device all at once (what the kernels whose CTAs meet through a counter need; call it
+// after ensure_dynamic_smem).  A host-side occupancy query, remembered per kernel and shared-memory size.
+bool grid_can_meet(const void *fn, int threads, size_t smem, int grid);
+
 griffin_status launch_decode(const griffin_ff_desc *desc, int B, const griffin_ff_compact *sets, const void *b_down,
                              const void *x, void *y, float *z, void *ws, uint32_t flags, cudaStream_t stream);
 
