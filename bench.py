@@ -64,6 +64,9 @@ def parse_args():
     ap.add_argument("--no-graph", action="store_true", help="launch every decode call from the host instead of replaying a CUDA graph")
     ap.add_argument("--decode", default="compact", choices=["compact", "indexed"],
                     help="indexed: no compaction step, the decode calls read the expert rows in place from the full weights")
+    ap.add_argument("--shared-set", action="store_true",
+                    help="the batch statistic of Eq. 7 in place of per-sequence sets: every sequence of a decode call uses the "
+                         "first sequence's expert set, so the weights are streamed once per call")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-workloads", action="store_true", help="leave out the section with the other shapes")
     ap.add_argument("--section-steps", type=int, default=3, help="timed steps of each entry of the workloads section")
@@ -247,7 +250,7 @@ def run_reference(args, w, keep):
     print(json.dumps(line), flush=True)
 
 
-def workload_config(w, L, B, keep, world, indexed, graphed):
+def workload_config(w, L, B, keep, world, indexed, graphed, shared=False):
     k = max(1, min(w.d_ff, int(keep * w.d_ff + 0.5)))
     n_mats = 2 if w.act in ("relu", "gelu_tanh", "gelu_erf", "silu") else 3
     cfg = {"workload": f"{w.name} ({SHAPE_NOTE.get(w.name, w.name)})", "d": w.d, "d_ff": w.d_ff, "L": L, "S": w.S,
@@ -257,6 +260,8 @@ def workload_config(w, L, B, keep, world, indexed, graphed):
                  f"{L * B * n_mats * k * w.d * w.elem_bytes / 1e9:.1f} GB compact) are visited in turn",
            "decode": ("index-direct: no compaction step, expert rows read in place from neuron-major full weights"
                       if indexed else "compact expert sets, one per sequence")}
+    if shared:
+        cfg["decode"] = "one compact expert set for the whole batch (Eq. 7): the first sequence's"
     if graphed is not None:
         cfg["decode_launch"] = ("the T x L decode calls of a step, captured once from the public API calls, are replayed as a CUDA graph"
                                 if graphed else "one host launch per decode call")
@@ -269,7 +274,7 @@ def workload_config(w, L, B, keep, world, indexed, graphed):
 class Job:
     """One workload resident on one GPU: the stack of blocks, its inputs and outputs, and the step."""
 
-    def __init__(self, w, B, keep, L, dev, rank, indexed, use_graph):
+    def __init__(self, w, B, keep, L, dev, rank, indexed, use_graph, shared_set=False):
         import torch
         from paper_2404_01365_b200 import binding as G, synth
         from paper_2404_01365_b200.runner import FFStack
@@ -289,6 +294,13 @@ class Job:
                 self.XD[:, l, q] = synth.make_decode_inputs(w, l, seq0 + q, device=dev)
         self.Y = torch.empty_like(self.X)
         self.YD = torch.empty_like(self.XD)
+        self.shared_set = shared_set and not indexed and B > 1
+        if self.shared_set:   # one compact set named for every sequence; its bytes are read once per call
+            st = self.stack
+            st.set_arrays = [G.compact_array([st.sets[l][0]] * B) for l in range(L)]
+            per_seq = st.decode_bytes_per_call() // B
+            shared_bytes = per_seq + (B - 1) * 2 * w.d * w.elem_bytes
+            st.decode_bytes_per_call = lambda: shared_bytes
         self.stream = torch.cuda.current_stream()
         self.use_graph = use_graph
         self.graph = None
@@ -554,7 +566,7 @@ def run_ours(args, w, keep):
     L = args.layers or w.L
     B = args.batch or w.B
     indexed = args.decode == "indexed"
-    job = Job(w, B, keep, L, dev, rank, indexed, not args.no_graph)
+    job = Job(w, B, keep, L, dev, rank, indexed, not args.no_graph, shared_set=args.shared_set)
     T, S = job.T, job.S
     job.warm_up(args.warmup)
     barrier()
@@ -626,14 +638,15 @@ def run_ours(args, w, keep):
             "metric": METRIC, "value": tokens / (ms_per_step / 1e3), "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
-            "config": workload_config(w, L, B, keep, world, indexed, job.graph is not None),
+            "config": workload_config(w, L, B, keep, world, indexed, job.graph is not None, job.shared_set),
             "phases": dict(rep, note="medians over the timed steps of per-phase CUDA-event times"),
-            "roofline": {"bound": "hbm", "kernel": ("decode_indexed_kernel" if indexed else "decode_fused_kernel") +
+            "roofline": {"bound": "hbm", "kernel": ("decode_indexed_kernel" if indexed else
+                                                    "decode_shared_kernel" if job.shared_set else "decode_fused_kernel") +
                          " (one launch per decode call; the decode phase is "
                          f"{100.0 * ph_ms[3] / sum(ph_ms):.0f} % of the step)", "achieved": dec["gbs"],
                          "peak": peaks[0], "unit": "GB/s", "frac": dec["frac_of_hbm"], "peak_source": peaks[3],
                          "algorithmic_bytes_per_launch": dec["algorithmic_bytes_per_call"],
-                         "traffic": None if indexed else recorded_traffic(traffic_key)},
+                         "traffic": None if indexed or job.shared_set else recorded_traffic(traffic_key)},
             "clocks": clocks,
             "gpu_launches": job.launches_per_step * K,
             "gpu_launches_per_step": job.launches_per_step,
@@ -642,7 +655,7 @@ def run_ours(args, w, keep):
         if e2e:
             line["e2e"] = {"value": tokens / (e2e_ms / 1e3), "unit": UNIT, "h2d_bytes_per_step": e2e[1],
                            "d2h_bytes_per_step": e2e[2], "steps": e2e[3]}
-    if rank == 0 and world == 1 and not indexed and w.dtype == "bf16":
+    if rank == 0 and world == 1 and not indexed and w.dtype == "bf16" and not job.shared_set:
         # decode of the unpruned block (keep 1.0) through the same kernel, and of one pruned sequence: the
         # speed-up that pruning half of the neurons buys at batch 1 (the byte ratio is 2)
         dense_us = job.time_decode_only(job.dense_sets(), 1, 3)
@@ -658,7 +671,7 @@ def run_ours(args, w, keep):
     job = None
     release()
 
-    if rank == 0 and world == 1 and not args.no_workloads and not indexed:
+    if rank == 0 and world == 1 and not args.no_workloads and not indexed and not args.shared_set:
         sect = []
         W = synth.WORKLOADS
         for name, with_dense in (("llama2_7b", True), ("gemma_7b", True), ("llama2_13b", True)):
