@@ -16,6 +16,12 @@ int device_sm_count();
 // Adds n to the count of kernels this library has launched in this process (griffin_kernel_launches).
 void count_launches(int n);
 
+// Launches `func` (counted), optionally as a programmatic dependent launch: it may then be scheduled before the
+// previous kernel on the stream has completed, and must itself wait (griddepcontrol.wait) before it touches
+// anything that kernel writes.
+cudaError_t launch_maybe_overlapped(const void *func, dim3 grid, dim3 block, size_t smem, cudaStream_t stream, bool overlap,
+                                    void **args);
+
 // Raises the opt-in dynamic shared memory limit of `fn` on the current device when needed.
 cudaError_t ensure_dynamic_smem(const void *fn, size_t bytes);
 

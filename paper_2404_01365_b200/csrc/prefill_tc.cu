@@ -81,6 +81,7 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    pdl_launch_dependents();  // a finishing kernel behind this one may take its place on the SMs and wait there
     const uint32_t tmem_base = *s.tmem_slot;
 
     // work items: (m, n, K split), or whole tiles followed by the parts of the cut ones
@@ -184,6 +185,7 @@ __global__ void __launch_bounds__(TC_THREADS) ff_tc_kernel(const __grid_constant
 // lane.  The parts are added in order, then bias, activation and gating as in the epilogue above:
 // Z in bf16 and fp32, and the row's sum of squares over the tile's 128 columns (fixed order).
 __global__ void __launch_bounds__(128) dual_tail_finish_kernel(TcParams p) {
+    pdl_wait_prior_grids();  // (launched to start early: everything it reads comes from the GEMM kernel before it)
     const int w = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     const int tile = p.tail_first + w / TC_BM, r = w % TC_BM, c = lane * 4;
     const int m = tile % p.m_tiles, n = tile / p.m_tiles;
@@ -248,6 +250,7 @@ __global__ void __launch_bounds__(128) dual_tail_finish_kernel(TcParams p) {
 // Finishes the cut tiles of the down projection: one warp per (cut tile, row), eight outputs per lane.
 // The parts are added in order, then b_2, then rounded to bf16.
 __global__ void __launch_bounds__(128) plain_tail_finish_kernel(TcParams p) {
+    pdl_wait_prior_grids();
     const int w = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     const int tile = p.tail_first + w / TC_BM, r = w % TC_BM, c = lane * 8;
     const int m = tile % p.m_tiles, n = tile / p.m_tiles;
@@ -284,6 +287,7 @@ __global__ void __launch_bounds__(128) plain_tail_finish_kernel(TcParams p) {
 // y = bf16(sum over K splits of part + bias), four columns per thread, splits added in order.
 __global__ void splitk_reduce_kernel(const float *__restrict__ part, const __nv_bfloat16 *__restrict__ bias,
                                      __nv_bfloat16 *__restrict__ y, int splits, size_t n_elems, int n_total) {
+    pdl_wait_prior_grids();
     const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
     if (i >= n_elems) return;
     float4 acc = *reinterpret_cast<const float4 *>(part + i);
@@ -458,9 +462,10 @@ griffin_status launch_prefill_tc(const griffin_ff_desc *desc, const griffin_ff_w
         st = gated ? launch_tc<TC_GATED, 128>(mx, mg, mu, p, sms, stream) : launch_tc<TC_WIDE, 128>(mx, mg, mu, p, sms, stream);
     }
     if (st == GRIFFIN_OK && p.tail_ks > 1) {
-        dual_tail_finish_kernel<<<(p.m_tiles * p.n_tiles - p.tail_first) * (TC_BM / 4), 128, 0, stream>>>(p);
-        count_launches(1);
-        if (cudaGetLastError() != cudaSuccess) st = GRIFFIN_ERR_CUDA;
+        void *args[] = {&p};
+        if (launch_maybe_overlapped((const void *)dual_tail_finish_kernel, dim3((p.m_tiles * p.n_tiles - p.tail_first) * (TC_BM / 4)),
+                                    dim3(128), 0, stream, true, args) != cudaSuccess)
+            st = GRIFFIN_ERR_CUDA;
     }
     if (st == GRIFFIN_OK && after_ff1 != nullptr && cudaEventRecord(after_ff1, stream) != cudaSuccess) return GRIFFIN_ERR_CUDA;
     if (st != GRIFFIN_OK || y == nullptr) return st;
@@ -498,16 +503,23 @@ griffin_status launch_prefill_tc(const griffin_ff_desc *desc, const griffin_ff_w
                        : launch_tc<TC_PLAIN, 128>(mz, md, md, q, sms, stream);
     }
     if (st == GRIFFIN_OK && q.tail_ks > 1) {
-        plain_tail_finish_kernel<<<(q.m_tiles * q.n_tiles - q.tail_first) * (TC_BM / 4), 128, 0, stream>>>(q);
-        count_launches(1);
-        if (cudaGetLastError() != cudaSuccess) st = GRIFFIN_ERR_CUDA;
+        void *args[] = {&q};
+        // (not as an early, dependent launch: its waiting blocks would take the thread slots beside the GEMM's CTAs
+        // that the statistic's kernels on the side stream are meant to run in -- measured, 4.6 us lost per call)
+        if (launch_maybe_overlapped((const void *)plain_tail_finish_kernel, dim3((q.m_tiles * q.n_tiles - q.tail_first) * (TC_BM / 4)),
+                                    dim3(128), 0, stream, false, args) != cudaSuccess)
+            st = GRIFFIN_ERR_CUDA;
     }
     if (st != GRIFFIN_OK || splits == 1) return st;
     const size_t n_elems = (size_t)S * d;
-    splitk_reduce_kernel<<<(unsigned)((n_elems / 4 + 255) / 256), 256, 0, stream>>>(
-        ypart, static_cast<const __nv_bfloat16 *>(w->b_down), static_cast<__nv_bfloat16 *>(y), splits, n_elems, d);
-    count_launches(1);
-    return cudaGetLastError() == cudaSuccess ? GRIFFIN_OK : GRIFFIN_ERR_CUDA;
+    const float *part_in = ypart;
+    const __nv_bfloat16 *bias = static_cast<const __nv_bfloat16 *>(w->b_down);
+    __nv_bfloat16 *y_out = static_cast<__nv_bfloat16 *>(y);
+    size_t n_el = n_elems;
+    int n_total = d;
+    void *args[] = {&part_in, &bias, &y_out, &splits, &n_el, &n_total};
+    return launch_maybe_overlapped((const void *)splitk_reduce_kernel, dim3((unsigned)((n_elems / 4 + 255) / 256)), dim3(256), 0,
+                                   stream, false, args) == cudaSuccess ? GRIFFIN_OK : GRIFFIN_ERR_CUDA;
 }
 
 }  // namespace griffin

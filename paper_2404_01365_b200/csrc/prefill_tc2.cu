@@ -137,6 +137,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS)
     __syncthreads();
     cluster_sync_all();  // the peer's barriers are initialised before anything of this CTA reaches them
     tc_fence_after_sync();
+    pdl_launch_dependents();  // a finishing kernel behind this one may take its place on the SMs and wait there
     const uint32_t tmem_base = *s.tmem_slot;
 
     const int n_clusters = gridDim.x >> 1, cluster_id = blockIdx.x >> 1;

@@ -145,3 +145,35 @@ def test_binding_fails_loudly_without_library(tmp_path, monkeypatch):
     monkeypatch.setattr(G, "_lib", None)
     with pytest.raises(RuntimeError, match="missing"):
         G.load(str(tmp_path / "nope.so"))
+
+
+def test_slicing_from_neuron_major_weights_validates_like_the_row_major_call(lib):
+    desc = G.make_desc(256, 688, "swiglu", "bf16")
+    fake, odd = C.c_void_p(0x10000), C.c_void_p(0x10004)
+    wn = G.FFWeightsNM(fake, fake, fake, None, None, None)
+    out = G.FFCompact(fake, fake, fake, None, None, 344, 344)
+    f = lib.griffin_compact_experts_nm
+    assert f(None, C.byref(wn), fake, C.byref(out), None, None) == G.ERR_INVALID_ARG
+    assert f(C.byref(desc), None, fake, C.byref(out), None, None) == G.ERR_INVALID_ARG
+    assert f(C.byref(desc), C.byref(wn), None, C.byref(out), None, None) == G.ERR_INVALID_ARG
+    no_down = G.FFWeightsNM(fake, fake, None, None, None, None)
+    assert f(C.byref(desc), C.byref(no_down), fake, C.byref(out), None, None) == G.ERR_INVALID_ARG
+    no_gate = G.FFWeightsNM(None, fake, fake, None, None, None)          # a gated block needs W_g
+    assert f(C.byref(desc), C.byref(no_gate), fake, C.byref(out), None, None) == G.ERR_INVALID_ARG
+    misaligned = G.FFWeightsNM(fake, fake, odd, None, None, None)
+    assert f(C.byref(desc), C.byref(misaligned), fake, C.byref(out), None, None) == G.ERR_ALIGNMENT
+    bad_ldk = G.FFCompact(fake, fake, fake, None, None, 344, 352)        # ldk must be k rounded up to 8
+    assert f(C.byref(desc), C.byref(wn), fake, C.byref(bad_ldk), None, None) == G.ERR_INVALID_ARG
+    too_many = G.FFCompact(fake, fake, fake, None, None, 696, 696)       # k beyond d_ff
+    assert f(C.byref(desc), C.byref(wn), fake, C.byref(too_many), None, None) == G.ERR_INVALID_ARG
+    relu = G.make_desc(256, 688, "relu", "bf16")                         # without a gate, naming W_g is an error
+    assert f(C.byref(relu), C.byref(wn), fake, C.byref(out), None, None) == G.ERR_INVALID_ARG
+
+
+def test_launch_counter_starts_at_zero_and_refused_calls_do_not_count(lib):
+    before = G.griffin_kernel_launches()
+    desc = G.make_desc(256, 688, "swiglu", "bf16")
+    assert lib.griffin_select_topk(None, 1, 688, 344, None, None) == G.ERR_INVALID_ARG
+    assert lib.griffin_workspace_init(None, 0, None) == G.ERR_WORKSPACE
+    assert G.griffin_kernel_launches() == before
+    assert isinstance(before, int) and before >= 0
