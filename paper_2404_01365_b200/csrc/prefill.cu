@@ -11,7 +11,8 @@
 //   5. s_j = sqrt(sum over chunks of colpart[chunk, j])                 (Eq. 6)
 //
 // The row normaliser spans every column tile, so the column sums cannot finish inside
-// step 1: steps 3-5 re-read the fp32 Z (which mostly still sits in L2).  All partial sums are kept
+// step 1: steps 3-5 re-read Z (fp32 storage), or Z and the bf16 residual that step 1 wrote beside it (bf16
+// storage; both mostly still sit in L2).  All partial sums are kept
 // and added in a fixed order, so s is deterministic.
 //
 // This file holds the fp32-FMA (SIMT) matrix kernels, which serve the fp32 storage type
@@ -40,7 +41,7 @@ PrefillScratch prefill_scratch(const griffin_ff_desc *desc, int S) {
     ps.z_off = off;
     off = align_up(off + (size_t)S * desc->d_ff * esz, 256);
     ps.zf_off = off;
-    if (desc->dtype != GRIFFIN_DT_F32) off = align_up(off + (size_t)S * desc->d_ff * sizeof(float), 256);
+    if (desc->dtype != GRIFFIN_DT_F32) off = align_up(off + (size_t)S * desc->d_ff * 2, 256);  // the bf16 residual of Z
     ps.rowsq_off = off;
     off = align_up(off + (size_t)S * ps.n_col_tiles * sizeof(float), 256);
     ps.inv_off = off;
@@ -90,7 +91,7 @@ template <typename T, bool GATED>
 __global__ void __launch_bounds__(PF_THREADS) ff1_simt_kernel(const T *__restrict__ x, const T *__restrict__ w_gate,
                                                               const T *__restrict__ w_up, const T *__restrict__ b_gate,
                                                               const T *__restrict__ b_up, T *__restrict__ z,
-                                                              float *__restrict__ zf,  // fp32 copy, or null
+                                                              T *__restrict__ zlo,  // bf16 storage: z - bf16(z); else null
                                                               float *__restrict__ rowsq, int S, int d, int d_ff,
                                                               int n_col_tiles, int act) {
     __shared__ float xs[PF_BK][PF_BM + PF_PAD], gs[PF_BK][PF_BN + PF_PAD], us[PF_BK][PF_BN + PF_PAD];
@@ -131,8 +132,9 @@ __global__ void __launch_bounds__(PF_THREADS) ff1_simt_kernel(const T *__restric
                 if (GATED && b_gate) g += Elem<T>::to_float(b_gate[col]);
                 if (b_up) u += Elem<T>::to_float(b_up[col]);
                 const float zv = GATED ? sigma_rt(act, g) * u : sigma_rt(act, u);
-                z[(size_t)row * d_ff + col] = Elem<T>::from_float(zv);
-                if (zf) zf[(size_t)row * d_ff + col] = zv;
+                const T zh = Elem<T>::from_float(zv);
+                z[(size_t)row * d_ff + col] = zh;
+                if (zlo) zlo[(size_t)row * d_ff + col] = Elem<T>::from_float(zv - Elem<T>::to_float(zh));
                 sq = fmaf(zv, zv, sq);
             }
         }
@@ -197,11 +199,14 @@ __global__ void row_inv_kernel(const float *__restrict__ rowsq, int S, int n_col
     if (lane == 0) inv[row] = sq > 0.f ? 1.0f / sq : 0.f;
 }
 
-// Step 4: a CTA owns 128 neighbouring columns of the fp32 Z over one chunk of tokens; each of
-// its 8 warps takes every 8th token of the chunk (one float4 per lane, all loads of a warp in
-// flight together) and the warps' sums meet in shared memory in a fixed order.
-__global__ void __launch_bounds__(256) col_partial_kernel(const float *__restrict__ z, const float *__restrict__ inv,
-                                                          int S, int d_ff, float *__restrict__ colpart) {
+// Step 4: a CTA owns 128 neighbouring columns of Z over one chunk of tokens; each of its 8 warps takes
+// every 8th token of the chunk (four columns per lane, all loads of a warp in flight together) and
+// the warps' sums meet in shared memory in a fixed order.  Z comes in fp32 (fp32 storage: zlo null) or
+// as two bf16 numbers per entry, z = zhi + zlo (bf16 storage: the Z that the down projection reads, and
+// what its rounding lost; together 16 mantissa bits, 4e-6 relative).
+__global__ void __launch_bounds__(256) col_partial_kernel(const void *__restrict__ z, const __nv_bfloat16 *__restrict__ zlo,
+                                                          const float *__restrict__ inv, int S, int d_ff,
+                                                          float *__restrict__ colpart) {
     __shared__ float4 red[8][32];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int col = (blockIdx.x * 32 + lane) * 4;
@@ -212,7 +217,17 @@ __global__ void __launch_bounds__(256) col_partial_kernel(const float *__restric
         for (int i = 0; i < PF_ROW_CHUNK / 8; ++i) {
             const int r = r0 + warp + 8 * i;
             if (r < r1) {
-                const float4 f = *reinterpret_cast<const float4 *>(z + (size_t)r * d_ff + col);
+                float4 f;
+                if (zlo == nullptr) {
+                    f = *reinterpret_cast<const float4 *>(static_cast<const float *>(z) + (size_t)r * d_ff + col);
+                } else {
+                    const uint2 h = *reinterpret_cast<const uint2 *>(static_cast<const __nv_bfloat16 *>(z) + (size_t)r * d_ff + col);
+                    const uint2 l = *reinterpret_cast<const uint2 *>(zlo + (size_t)r * d_ff + col);
+                    f.x = __uint_as_float(h.x << 16) + __uint_as_float(l.x << 16);
+                    f.y = __uint_as_float(h.x & 0xffff0000u) + __uint_as_float(l.x & 0xffff0000u);
+                    f.z = __uint_as_float(h.y << 16) + __uint_as_float(l.y << 16);
+                    f.w = __uint_as_float(h.y & 0xffff0000u) + __uint_as_float(l.y & 0xffff0000u);
+                }
                 const float w = __ldg(inv + r);
                 acc.x = fmaf(f.x * f.x, w, acc.x);
                 acc.y = fmaf(f.y * f.y, w, acc.y);
@@ -285,7 +300,7 @@ static griffin_status prefill_typed(const griffin_ff_desc *desc, const griffin_f
     const PrefillScratch ps = prefill_scratch(desc, S);
     T *z = reinterpret_cast<T *>(scratch + ps.z_off);
     constexpr bool kBf16 = std::is_same<T, __nv_bfloat16>::value;
-    float *zf = kBf16 ? reinterpret_cast<float *>(scratch + ps.zf_off) : nullptr;
+    T *zlo = kBf16 ? reinterpret_cast<T *>(scratch + ps.zf_off) : nullptr;
     float *rowsq = reinterpret_cast<float *>(scratch + ps.rowsq_off);
     float *inv = reinterpret_cast<float *>(scratch + ps.inv_off);
     float *colpart = reinterpret_cast<float *>(scratch + ps.colpart_off);
@@ -299,7 +314,7 @@ static griffin_status prefill_typed(const griffin_ff_desc *desc, const griffin_f
     if (use_tc) {
         if constexpr (kBf16) {
             if (y != nullptr) lane = side_lane_of_current_device();  // (measured: a gain at every prompt length, 9 % at S = 512)
-            griffin_status st = launch_prefill_tc(desc, w, x, S, y, z, zf, rowsq, reinterpret_cast<float *>(scratch + ps.ypart_off),
+            griffin_status st = launch_prefill_tc(desc, w, x, S, y, z, zlo, rowsq, reinterpret_cast<float *>(scratch + ps.ypart_off),
                                                   &n_col_tiles, ws, stream, lane ? lane->fork : nullptr);
             if (st != GRIFFIN_OK) return st;
             if (lane != nullptr) {
@@ -314,12 +329,12 @@ static griffin_status prefill_typed(const griffin_ff_desc *desc, const griffin_f
         if (act_gated(desc->act)) {
             ff1_simt_kernel<T, true><<<g1, PF_THREADS, 0, stream>>>(
                 static_cast<const T *>(x), static_cast<const T *>(w->w_gate), static_cast<const T *>(w->w_up),
-                static_cast<const T *>(w->b_gate), static_cast<const T *>(w->b_up), z, zf, rowsq, S, d, d_ff,
+                static_cast<const T *>(w->b_gate), static_cast<const T *>(w->b_up), z, zlo, rowsq, S, d, d_ff,
                 n_col_tiles, desc->act);
         } else {
             ff1_simt_kernel<T, false><<<g1, PF_THREADS, 0, stream>>>(
                 static_cast<const T *>(x), nullptr, static_cast<const T *>(w->w_up), nullptr,
-                static_cast<const T *>(w->b_up), z, zf, rowsq, S, d, d_ff, n_col_tiles, act_sigma(desc->act));
+                static_cast<const T *>(w->b_up), z, zlo, rowsq, S, d, d_ff, n_col_tiles, act_sigma(desc->act));
         }
         count_launches(1);
         if (cudaGetLastError() != cudaSuccess) return GRIFFIN_ERR_CUDA;
@@ -336,10 +351,9 @@ static griffin_status prefill_typed(const griffin_ff_desc *desc, const griffin_f
     row_inv_kernel<<<(S + 7) / 8, 256, 0, stat_stream>>>(rowsq, S, n_col_tiles, inv);
     count_launches(1);
     if (cudaGetLastError() != cudaSuccess) st = GRIFFIN_ERR_CUDA;
-    const float *z32 = kBf16 ? zf : reinterpret_cast<const float *>(z);
     const dim3 g4((d_ff + 127) / 128, ps.n_row_chunks);
     if (st == GRIFFIN_OK) {
-        col_partial_kernel<<<g4, 256, 0, stat_stream>>>(z32, inv, S, d_ff, colpart);
+        col_partial_kernel<<<g4, 256, 0, stat_stream>>>(z, reinterpret_cast<const __nv_bfloat16 *>(zlo), inv, S, d_ff, colpart);
         count_launches(1);
         if (cudaGetLastError() != cudaSuccess) st = GRIFFIN_ERR_CUDA;
     }

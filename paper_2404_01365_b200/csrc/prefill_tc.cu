@@ -1,6 +1,6 @@
 // Prompt-phase FF on the 5th-generation tensor cores (Eqs. 1 and 3 of the GRIFFIN paper), bf16
 // storage, fp32 accumulation:
-//   kernel<KIND = 1> : Z = sigma(X W_g^T + b_g) * (X W_1^T + b_1), also Z in fp32 and the
+//   kernel<KIND = 1> : Z = sigma(X W_g^T + b_g) * (X W_1^T + b_1), also the bf16 residual Z - bf16(Z) and the
 //                      per-tile partial sums of squares of its rows (for the statistic)
 //   kernel<KIND = 2> : the same for a block without a gate (Eq. 2): Z = sigma(X W_1^T + b_1)
 //   kernel<KIND = 0> : Y = Z W_2^T + b_2
@@ -226,7 +226,10 @@ __global__ void __launch_bounds__(128) dual_tail_finish_kernel(TcParams p) {
             const __nv_bfloat162 h0 = __floats2bfloat162_rn(z2[0], z2[1]), h1 = __floats2bfloat162_rn(z2[2], z2[3]);
             *reinterpret_cast<uint2 *>(p.out + (size_t)row * p.n_total + col2) =
                 make_uint2(*reinterpret_cast<const uint32_t *>(&h0), *reinterpret_cast<const uint32_t *>(&h1));
-            *reinterpret_cast<float4 *>(p.zf + (size_t)row * p.n_total + col2) = make_float4(z2[0], z2[1], z2[2], z2[3]);
+            const __nv_bfloat162 l0 = __floats2bfloat162_rn(z2[0] - __low2float(h0), z2[1] - __high2float(h0));
+            const __nv_bfloat162 l1 = __floats2bfloat162_rn(z2[2] - __low2float(h1), z2[3] - __high2float(h1));
+            *reinterpret_cast<uint2 *>(p.zlo + (size_t)row * p.n_total + col2) =
+                make_uint2(*reinterpret_cast<const uint32_t *>(&l0), *reinterpret_cast<const uint32_t *>(&l1));
         }
     } else {
 #pragma unroll
@@ -241,7 +244,10 @@ __global__ void __launch_bounds__(128) dual_tail_finish_kernel(TcParams p) {
         const __nv_bfloat162 h0 = __floats2bfloat162_rn(z[0], z[1]), h1 = __floats2bfloat162_rn(z[2], z[3]);
         *reinterpret_cast<uint2 *>(p.out + (size_t)row * p.n_total + col) =
             make_uint2(*reinterpret_cast<const uint32_t *>(&h0), *reinterpret_cast<const uint32_t *>(&h1));
-        *reinterpret_cast<float4 *>(p.zf + (size_t)row * p.n_total + col) = make_float4(z[0], z[1], z[2], z[3]);
+        const __nv_bfloat162 l0 = __floats2bfloat162_rn(z[0] - __low2float(h0), z[1] - __high2float(h0));
+        const __nv_bfloat162 l1 = __floats2bfloat162_rn(z[2] - __low2float(h1), z[3] - __high2float(h1));
+        *reinterpret_cast<uint2 *>(p.zlo + (size_t)row * p.n_total + col) =
+            make_uint2(*reinterpret_cast<const uint32_t *>(&l0), *reinterpret_cast<const uint32_t *>(&l1));
     }
     sq = warp_sum(sq);
     if (lane < 2 && row < p.S) p.rowsq[(size_t)row * (2 * p.n_tiles) + 2 * n + lane] = lane == 0 ? sq : 0.f;
@@ -419,7 +425,7 @@ static griffin_status launch_tc(const CUtensorMap &ma, const CUtensorMap &mb0, c
 }
 
 griffin_status launch_prefill_tc(const griffin_ff_desc *desc, const griffin_ff_weights *w, const void *x, int S,
-                                 void *y, __nv_bfloat16 *z, float *zf, float *rowsq, float *ypart, int *n_col_tiles,
+                                 void *y, __nv_bfloat16 *z, __nv_bfloat16 *zlo, float *rowsq, float *ypart, int *n_col_tiles,
                                  void *ws, cudaStream_t stream, cudaEvent_t after_ff1) {
     const int d = desc->d, d_ff = desc->d_ff;
     const int sms = device_sm_count();
@@ -440,7 +446,7 @@ griffin_status launch_prefill_tc(const griffin_ff_desc *desc, const griffin_ff_w
     p.bias0 = static_cast<const __nv_bfloat16 *>(gated ? w->b_gate : nullptr);
     p.bias1 = static_cast<const __nv_bfloat16 *>(w->b_up);
     p.out = z;
-    p.zf = zf;
+    p.zlo = zlo;
     p.rowsq = rowsq;
     p.act = act_sigma(desc->act);
     p.ws = ws;

@@ -41,7 +41,7 @@ struct TcParams {
     int m_tiles, n_tiles;
     const __nv_bfloat16 *bias0, *bias1;  // DUAL: b_gate, b_up; otherwise b_down, unused (may be null)
     __nv_bfloat16 *out;                  // Z or Y, [S, n_total]
-    float *zf;                           // DUAL: Z in fp32, [S, n_total]
+    __nv_bfloat16 *zlo;                  // DUAL: what Z lost when it was rounded to bf16, itself in bf16: z - bf16(z), [S, n_total]
     float *rowsq;                        // DUAL: [S, 2 n_tiles] partial sums of squares of the fp32 rows (two column halves per tile)
     int splits;                          // K splits (1 unless the plain GEMM has too few tiles)
     float *part;                         // splits > 1: fp32 partial outputs [splits, S, n_total]
@@ -155,18 +155,18 @@ __device__ __forceinline__ void tc_epilogue_item(const TcParams &p, int m, int n
             float u[32];
             tmem_ld32(taddr + c, u);
             const int col = n * 256 + c;
-            uint32_t packed[16];
+            uint32_t packed[16], packed_lo[16];
 #pragma unroll
             for (int i = 0; i < 32; i += 2) {
                 float u0 = u[i], u1 = u[i + 1];
                 if (p.bias1) { u0 += __bfloat162float(p.bias1[col + i]); u1 += __bfloat162float(p.bias1[col + i + 1]); }
                 const float z0 = sigma_fast_rt(p.act, u0), z1 = sigma_fast_rt(p.act, u1);
-                u[i] = z0;
-                u[i + 1] = z1;
                 sq = fmaf(z0, z0, sq);
                 sq = fmaf(z1, z1, sq);
                 const __nv_bfloat162 h = __floats2bfloat162_rn(z0, z1);
                 packed[i >> 1] = *reinterpret_cast<const uint32_t *>(&h);
+                const __nv_bfloat162 l = __floats2bfloat162_rn(z0 - __low2float(h), z1 - __high2float(h));
+                packed_lo[i >> 1] = *reinterpret_cast<const uint32_t *>(&l);
             }
             {
                 uint4 pk[4];
@@ -174,7 +174,10 @@ __device__ __forceinline__ void tc_epilogue_item(const TcParams &p, int m, int n
                 for (int v = 0; v < 4; ++v)
                     pk[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
                 store_rows64(stg, pk, p.out + (size_t)row0 * p.n_total + col, (size_t)p.n_total * 2, rows_live, lane);
-                store_rows_f32x32(stg, u, p.zf + (size_t)row0 * p.n_total + col, (size_t)p.n_total * 4, rows_live, lane);
+#pragma unroll
+                for (int v = 0; v < 4; ++v)
+                    pk[v] = make_uint4(packed_lo[4 * v], packed_lo[4 * v + 1], packed_lo[4 * v + 2], packed_lo[4 * v + 3]);
+                store_rows64(stg, pk, p.zlo + (size_t)row0 * p.n_total + col, (size_t)p.n_total * 2, rows_live, lane);
             }
         }
         if (live) p.rowsq[(size_t)row * (2 * p.n_tiles) + 2 * n + half] = sq;
@@ -185,19 +188,19 @@ __device__ __forceinline__ void tc_epilogue_item(const TcParams &p, int m, int n
             float g[32], u[32];
             tmem_ld32x2(taddr + c, taddr + 128 + c, g, u);
             const int col = n * 128 + c;
-            uint32_t packed[16];
+            uint32_t packed[16], packed_lo[16];
 #pragma unroll
             for (int i = 0; i < 32; i += 2) {
                 float g0 = g[i], g1 = g[i + 1], u0 = u[i], u1 = u[i + 1];
                 if (p.bias0) { g0 += __bfloat162float(p.bias0[col + i]); g1 += __bfloat162float(p.bias0[col + i + 1]); }
                 if (p.bias1) { u0 += __bfloat162float(p.bias1[col + i]); u1 += __bfloat162float(p.bias1[col + i + 1]); }
                 const float z0 = sigma_fast_rt(p.act, g0) * u0, z1 = sigma_fast_rt(p.act, g1) * u1;
-                g[i] = z0;
-                g[i + 1] = z1;
                 sq = fmaf(z0, z0, sq);
                 sq = fmaf(z1, z1, sq);
                 const __nv_bfloat162 h = __floats2bfloat162_rn(z0, z1);
                 packed[i >> 1] = *reinterpret_cast<const uint32_t *>(&h);
+                const __nv_bfloat162 l = __floats2bfloat162_rn(z0 - __low2float(h), z1 - __high2float(h));
+                packed_lo[i >> 1] = *reinterpret_cast<const uint32_t *>(&l);
             }
             {
                 uint4 pk[4];
@@ -205,7 +208,10 @@ __device__ __forceinline__ void tc_epilogue_item(const TcParams &p, int m, int n
                 for (int v = 0; v < 4; ++v)
                     pk[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
                 store_rows64(stg, pk, p.out + (size_t)row0 * p.n_total + col, (size_t)p.n_total * 2, rows_live, lane);
-                store_rows_f32x32(stg, g, p.zf + (size_t)row0 * p.n_total + col, (size_t)p.n_total * 4, rows_live, lane);
+#pragma unroll
+                for (int v = 0; v < 4; ++v)
+                    pk[v] = make_uint4(packed_lo[4 * v], packed_lo[4 * v + 1], packed_lo[4 * v + 2], packed_lo[4 * v + 3]);
+                store_rows64(stg, pk, p.zlo + (size_t)row0 * p.n_total + col, (size_t)p.n_total * 2, rows_live, lane);
             }
         }
         if (live) p.rowsq[(size_t)row * (2 * p.n_tiles) + 2 * n + half] = sq;

@@ -33,11 +33,11 @@ size_t gemm2_tail_bytes(int S, int d, int d_ff);
 // Whether the tensor-core kernels take this shape (bf16, d and d_ff multiples of 64, ...).
 bool prefill_tc_supported(const griffin_ff_desc *desc, int S);
 
-// Steps 1 and 2 of the prompt phase: writes Z (bf16), its fp32 copy zf and the per-tile partial
+// Steps 1 and 2 of the prompt phase: writes Z (bf16), the bf16 residual zlo = z - bf16(z) and the per-tile partial
 // row sums of squares rowsq [S, *n_col_tiles]; writes Y unless y is NULL.  after_ff1 (may be
 // NULL) is recorded on the stream between the two GEMMs: what only needs Z may start there.
 griffin_status launch_prefill_tc(const griffin_ff_desc *desc, const griffin_ff_weights *w, const void *x, int S,
-                                 void *y, __nv_bfloat16 *z, float *zf, float *rowsq, float *ypart, int *n_col_tiles, void *ws,
+                                 void *y, __nv_bfloat16 *z, __nv_bfloat16 *zlo, float *rowsq, float *ypart, int *n_col_tiles, void *ws,
                                  cudaStream_t stream, cudaEvent_t after_ff1);
 
 }  // namespace griffin
