@@ -200,6 +200,9 @@ SHARED_SET_SHAPES = [
     (64, 96, 37, 2, "reglu", True),            # fewer neurons than CTAs: most work items are empty
     (2048, 8192, 4000, 6, "relu", True),       # a block without a gate (Eq. 2)
     (1024, 4096, 2048, 8, "gelu_tanh", False),  # ... and another
+    (5120, 13824, 6912, 8, "swiglu", False),   # Llama-2-13B shape: rows of 10 KB and 13.5 KB in three and four chunks
+    (3072, 24576, 12288, 8, "geglu_tanh", False),  # Gemma shape: eight vectors of 24 KB do not fit, two passes of four
+    (4096, 14336, 3584, 4, "swiglu", False),   # Mistral shape at keep 0.25
 ]
 
 
