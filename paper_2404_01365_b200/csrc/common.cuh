@@ -25,6 +25,7 @@ struct WsHeader {
     unsigned int meet_warp;  // meeting-point counter of the warp-level fused decode kernel (see grid_meet)
     unsigned int meet_tc;    // ... and of the tcgen05 one (the two have different numbers of parties)
     unsigned int meet_idx;   // ... and of the index-direct one
+    unsigned int meet_stream;  // ... and of the register-streaming one
 };
 
 __device__ __forceinline__ void raise_status(void *ws, int status, int detail) {

@@ -17,6 +17,7 @@
 //     kernel (x, z, y) is touched only after griddepcontrol.wait.
 // Results are deterministic: every sum has a fixed order.
 #include <atomic>
+#include <cstdlib>
 
 #include "decode_common.cuh"
 
@@ -417,6 +418,11 @@ griffin_status launch_decode(const griffin_ff_desc *desc, int B, const griffin_f
     // one expert set for several sequences (Eq. 7): streamed once for up to 8 of them at a time
     if (decode_shared_set(p) && !(want_tc && decode_tc_shared(p))) {
         const griffin_status st = decode_bf16_shared(p, act, gated, flags, stream);
+        if (st != GRIFFIN_ERR_UNSUPPORTED) return st;
+    }
+    static const bool use_stream = getenv("GRIFFIN_DECODE_STREAM") != nullptr;
+    if (use_stream && !want_tc) {
+        const griffin_status st = decode_bf16_stream(p, act, gated, flags, stream);
         if (st != GRIFFIN_ERR_UNSUPPORTED) return st;
     }
     if (!gated) return decode_bf16_mma(p, act, false, flags, stream);

@@ -121,6 +121,9 @@ int slices_for(int rows, int grid);
 // act: the code of sigma (0..3); gated: whether the block has a gate (Eq. 3) or not (Eq. 2).
 griffin_status decode_bf16_mma(DecodeParams &p, int act, bool gated, uint32_t flags, cudaStream_t stream);
 
+// bf16 decode streamed through registers, without a shared-memory ring (decode_stream.cu).
+griffin_status decode_bf16_stream(DecodeParams &p, int act, bool gated, uint32_t flags, cudaStream_t stream);
+
 // bf16 decode of a batch that shares one expert set (decode_shared.cu): the weights are streamed once per
 // pass of up to 8 vectors, which are the columns of the warp-level MMA.
 bool decode_shared_set(const DecodeParams &p);  // 2 or more sequences that all name the same buffers

@@ -1,0 +1,344 @@
+// Generation-phase pruned FF (Eqs. 4 and 5 of the GRIFFIN paper) for bf16 storage, streamed
+// through registers: ONE kernel per call, one persistent CTA of 16 warps per SM, no shared-memory
+// ring, no producer, no barriers on the way.
+//   first half   z_hat = sigma(W_g_hat x + b_g_hat) * (W_1_hat x + b_1_hat)
+//   meeting      every CTA has written its z entries; all CTAs wait for each other (bounded)
+//   second half  y_hat = W_2_hat z_hat + b_2
+//
+// Both halves are matrix-vector products whose cost is the single pass over the compact weights,
+// and a read-only stream of HBM runs fastest (measured on B200: 6.8-7.2 TB/s against 6.5 TB/s for
+// a copy) when every warp keeps 8 KB of plain 16-byte loads in flight and does nothing else that
+// could hold them up.  So every warp streams weight rows straight from global memory into
+// registers, two steps deep (a step is 2 KB of each of the two rows of a "pair"), and hands them
+// to the warp-level tensor-core instruction mma.sync.m16n8k16, which takes the place of unpacking
+// and multiplying element by element (the diagonal of the 16 x 8 tile is the dot product, see
+// diagonal_sum).  The vector (x, then z) sits in shared memory, read conflict-free by the same
+// lane that holds the matching weights.
+//
+// Work split.  A pair is (gate row j, up row j) in the first half of a gated block, two
+// consecutive rows of W_1_hat (no gate) or of W_2_hat otherwise.  The B * P pairs of a half are
+// dealt to the CTAs as contiguous ranges (a range spans at most two sequences, whose vectors are
+// both staged), and a CTA's range, counted in steps, to its 16 warps as contiguous ranges again.
+// A pair that is cut between warps leaves partial sums in shared memory, which are added, in warp
+// order, once the CTA's warps have met at the end of the half: the split is even to one step and
+// every sum has a fixed order.
+#include "decode_mma.cuh"
+
+namespace griffin {
+
+constexpr int ST_WARPS = 16;
+constexpr int ST_THREADS = ST_WARPS * 32;
+constexpr int ST_H = 4;                    // 16-byte units of each row of a pair, per lane and step
+constexpr int ST_STEP_UNITS = 32 * ST_H;   // units of a row that one step covers (2 KB)
+constexpr int ST_GATE_UP = 0, ST_DOWN = 1, ST_UP = 2;
+
+struct StreamPartial {  // what a warp has summed of a pair that it shares with its neighbours
+    int f;              // pair (index among the B * P of the half), -1: none
+    float a0, a1;
+    int pad;
+};
+
+struct StreamGeom {
+    int rows;       // rows per sequence: k, or d
+    int P;          // pairs per sequence
+    int row_units;  // 16-byte units per row
+    int S;          // steps per row
+};
+template <int MODE> __device__ __forceinline__ StreamGeom stream_geom(const DecodeParams &p) {
+    StreamGeom g;
+    g.rows = MODE == ST_DOWN ? p.d : p.k;
+    g.P = MODE == ST_GATE_UP ? g.rows : (g.rows + 1) / 2;
+    g.row_units = (MODE == ST_DOWN ? p.ldk : p.d) / 8;
+    g.S = (g.row_units + ST_STEP_UNITS - 1) / ST_STEP_UNITS;
+    return g;
+}
+
+__device__ __forceinline__ uint4 ldg_stream(const uint4 *p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+// What a finished pair turns into: one entry of z (gated), or two of z or of y.
+template <int MODE>
+__device__ __forceinline__ void finish_pair(const DecodeParams &p, const StreamGeom &g, int act, int f, float a0, float a1) {
+    const int b = f / g.P, j = f - b * g.P;
+    __nv_bfloat16 *zb = reinterpret_cast<__nv_bfloat16 *>(p.z) + (size_t)b * 2 * p.ldk;  // z of sequence b, bf16
+    if (MODE == ST_GATE_UP) {
+        if (p.seq[b].b_gate) a0 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[b].b_gate)[j]);
+        if (p.seq[b].b_up) a1 += __bfloat162float(static_cast<const __nv_bfloat16 *>(p.seq[b].b_up)[j]);
+        zb[j] = __float2bfloat16_rn(sigma_rt(act, a0) * a1);
+    } else if (MODE == ST_UP) {
+        const __nv_bfloat16 *bias = static_cast<const __nv_bfloat16 *>(p.seq[b].b_up);
+        const int r = 2 * j;
+        zb[r] = __float2bfloat16_rn(sigma_rt(act, a0 + (bias ? __bfloat162float(bias[r]) : 0.f)));
+        if (r + 1 < g.rows) zb[r + 1] = __float2bfloat16_rn(sigma_rt(act, a1 + (bias ? __bfloat162float(bias[r + 1]) : 0.f)));
+    } else {
+        const __nv_bfloat16 *bias = static_cast<const __nv_bfloat16 *>(p.b_down);
+        __nv_bfloat16 *y = static_cast<__nv_bfloat16 *>(p.y) + (size_t)b * p.d;
+        const int r = 2 * j;
+        y[r] = __float2bfloat16_rn(a0 + (bias ? __bfloat162float(bias[r]) : 0.f));
+        if (r + 1 < g.rows) y[r + 1] = __float2bfloat16_rn(a1 + (bias ? __bfloat162float(bias[r + 1]) : 0.f));
+    }
+}
+
+// One warp's part of one half.  Usage: init, prologue (weights only: may run before anything the
+// half depends on is ready), then run.
+template <int MODE>
+struct StreamHalf {
+    StreamGeom g;
+    int lo, hi;          // the CTA's pairs [lo, hi) of the half's B * P
+    int b0;              // sequence of pair lo (its vector is slot 0, the next sequence's slot 1)
+    int f_slot1;         // first pair of sequence b0 + 1
+    int full_steps;      // steps of a row with every lane inside the row
+    int n_issue, n_comp; // steps of this warp not yet loaded / not yet multiplied
+    bool mid;            // the pair being summed began in another warp
+    // load cursor: pair, step within it, this lane's unit 0 of the pair's rows
+    int lf, lsp;
+    const uint4 *r0, *r1;
+    bool two;
+    // the steps held in registers A and B
+    int af, asp, bf, bsp;
+    int lane, warp;
+
+    __device__ __forceinline__ void set_pair(const DecodeParams &p, int f) {
+        const int b = f / g.P, j = f - b * g.P;
+        if (MODE == ST_GATE_UP) {
+            r0 = static_cast<const uint4 *>(p.seq[b].w_gate) + (size_t)j * g.row_units + lane;
+            r1 = static_cast<const uint4 *>(p.seq[b].w_up) + (size_t)j * g.row_units + lane;
+            two = true;
+        } else {
+            const void *m = MODE == ST_DOWN ? p.seq[b].w_down : p.seq[b].w_up;
+            r0 = static_cast<const uint4 *>(m) + (size_t)(2 * j) * g.row_units + lane;
+            r1 = r0 + g.row_units;
+            two = 2 * j + 1 < g.rows;
+        }
+    }
+
+    __device__ __forceinline__ void init(const DecodeParams &p, int warp_, int lane_) {
+        warp = warp_;
+        lane = lane_;
+        g = stream_geom<MODE>(p);
+        const long long T = (long long)p.B * g.P;
+        lo = (int)(T * blockIdx.x / gridDim.x);
+        hi = (int)(T * (blockIdx.x + 1) / gridDim.x);
+        b0 = lo / g.P;
+        f_slot1 = (b0 + 1) * g.P;
+        full_steps = g.row_units / ST_STEP_UNITS;
+        const int n = (hi - lo) * g.S;  // the CTA's steps
+        const int s0 = (int)((long long)n * warp / ST_WARPS), s1 = (int)((long long)n * (warp + 1) / ST_WARPS);
+        n_issue = n_comp = s1 - s0;
+        const int pr = s0 / g.S;
+        lf = lo + pr;
+        lsp = s0 - pr * g.S;
+        mid = lsp != 0;
+        af = asp = bf = bsp = 0;
+        r0 = r1 = nullptr;
+        two = false;
+        if (n_issue > 0) set_pair(p, lf);
+    }
+
+    // Loads the next step into r and moves the cursor on.
+    __device__ __forceinline__ void issue(const DecodeParams &p, uint4 (&r)[2 * ST_H], int &mf, int &msp) {
+        mf = lf;
+        msp = lsp;
+        const int u0 = lsp * ST_STEP_UNITS;
+        if (lsp < full_steps && two) {  // (warp-uniform) the common case: nothing to guard
+#pragma unroll
+            for (int i = 0; i < ST_H; ++i) {
+                r[i] = ldg_stream(r0 + u0 + i * 32);
+                r[ST_H + i] = ldg_stream(r1 + u0 + i * 32);
+            }
+        } else {  // the end of a row, or a pair of one row: what is not there counts as zero
+            const uint4 zero = make_uint4(0, 0, 0, 0);
+#pragma unroll
+            for (int i = 0; i < ST_H; ++i) {
+                const bool in = u0 + i * 32 + lane < g.row_units;
+                r[i] = in ? ldg_stream(r0 + u0 + i * 32) : zero;
+                r[ST_H + i] = (in && two) ? ldg_stream(r1 + u0 + i * 32) : zero;
+            }
+        }
+        --n_issue;
+        if (++lsp == g.S) {
+            lsp = 0;
+            ++lf;
+            if (n_issue > 0) set_pair(p, lf);
+        }
+    }
+
+    // The warp's first two steps: what is in flight while the CTA waits for others.
+    __device__ __forceinline__ void prologue(const DecodeParams &p, uint4 (&A)[2 * ST_H], uint4 (&Bq)[2 * ST_H]) {
+        if (n_issue > 0) issue(p, A, af, asp);
+        if (n_issue > 0) issue(p, Bq, bf, bsp);
+    }
+
+    // Multiplies the step held in r and, at the end of a pair or of the warp's range, hands the sums on.
+    __device__ __forceinline__ void compute(const DecodeParams &p, const uint4 (&r)[2 * ST_H], int mf, int msp,
+                                            float (&acc)[4][4], const uint4 *vec, int vec_units, StreamPartial *part,
+                                            int act) {
+        const uint4 *v = vec + (mf >= f_slot1 ? vec_units : 0) + msp * ST_STEP_UNITS + lane;
+#pragma unroll
+        for (int i = 0; i < ST_H; ++i) {
+            const uint4 vv = v[i * 32];
+            mma_bf16(acc[(2 * i) & 3], r[i].x, r[ST_H + i].x, r[i].y, r[ST_H + i].y, vv.x, vv.y);
+            mma_bf16(acc[(2 * i + 1) & 3], r[i].z, r[ST_H + i].z, r[i].w, r[ST_H + i].w, vv.z, vv.w);
+        }
+        --n_comp;
+        const bool complete = msp == g.S - 1;
+        if (complete || n_comp == 0) {
+            float sum[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                sum[e] = (acc[0][e] + acc[1][e]) + (acc[2][e] + acc[3][e]);
+                acc[0][e] = acc[1][e] = acc[2][e] = acc[3][e] = 0.f;
+            }
+            const float a0 = diagonal_sum(sum, lane);          // lane 0: first row, lane 4: second row
+            const float a1 = __shfl_sync(0xffffffffu, a0, 4);
+            if (lane == 0) {
+                if (complete && !mid) {
+                    finish_pair<MODE>(p, g, act, mf, a0, a1);
+                } else {
+                    StreamPartial *s = part + 2 * warp + (mid ? 0 : 1);
+                    s->f = mf;
+                    s->a0 = a0;
+                    s->a1 = a1;
+                }
+            }
+            mid = false;
+        }
+    }
+
+    // A and Bq hold the first two steps (prologue); every step multiplied makes room for the load of the one after next.
+    __device__ __forceinline__ void run(const DecodeParams &p, uint4 (&A)[2 * ST_H], uint4 (&Bq)[2 * ST_H], const uint4 *vec,
+                                        int vec_units, StreamPartial *part, int act) {
+        float acc[4][4] = {};
+        while (n_comp > 0) {
+            compute(p, A, af, asp, acc, vec, vec_units, part, act);
+            if (n_comp == 0) break;
+            if (n_issue > 0) issue(p, A, af, asp);
+            compute(p, Bq, bf, bsp, acc, vec, vec_units, part, act);
+            if (n_issue > 0) issue(p, Bq, bf, bsp);
+        }
+    }
+};
+
+// The pairs that were cut between warps: entry e = 2 * warp + (0: the warp's first pair, begun
+// elsewhere; 1: its last, ended elsewhere) is in step order, so the pieces of one pair follow each
+// other among the entries in use; the thread of a pair's first piece adds the rest to it.
+template <int MODE>
+__device__ __forceinline__ void combine_partials(const DecodeParams &p, const StreamPartial *part, int act, int tid) {
+    if (tid >= 2 * ST_WARPS) return;
+    const StreamPartial me = part[tid];
+    if (me.f < 0) return;
+    int pe = tid - 1;
+    while (pe >= 0 && part[pe].f < 0) --pe;
+    if (pe >= 0 && part[pe].f == me.f) return;
+    float a0 = me.a0, a1 = me.a1;
+    for (int e = tid + 1; e < 2 * ST_WARPS; ++e) {
+        const StreamPartial o = part[e];
+        if (o.f < 0) continue;
+        if (o.f != me.f) break;
+        a0 += o.a0;
+        a1 += o.a1;
+    }
+    const StreamGeom g = stream_geom<MODE>(p);
+    finish_pair<MODE>(p, g, act, me.f, a0, a1);
+}
+
+// bf16 words of a 16-byte unit whose elements from `keep` on are cleared (keep in 1..7)
+__device__ __forceinline__ uint4 keep_elems(uint4 v, int keep) {
+    uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if (2 * i >= keep) w[i] = 0;
+        else if (2 * i + 1 >= keep) w[i] &= 0xffffu;
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+template <bool GATED>
+__global__ void __launch_bounds__(ST_THREADS, 1) decode_stream_kernel(const __grid_constant__ DecodeParams p, int act,
+                                                                    int vec_units) {
+    constexpr int FIRST = GATED ? ST_GATE_UP : ST_UP;
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    uint4 *vec = reinterpret_cast<uint4 *>(smem_raw);                       // two vectors of vec_units units
+    StreamPartial *part = reinterpret_cast<StreamPartial *>(vec + 2 * vec_units);
+    volatile int *abort = reinterpret_cast<volatile int *>(part + 2 * ST_WARPS);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    uint4 A[2 * ST_H], Bq[2 * ST_H];
+
+    // ---- first half: the first weights are on their way before anything else happens
+    StreamHalf<FIRST> h1;
+    h1.init(p, warp, lane);
+    h1.prologue(p, A, Bq);
+    pdl_launch_dependents();
+    if (tid == 0) *abort = 0;
+    if (tid < 2 * ST_WARPS) part[tid].f = -1;
+    pdl_wait_prior_grids();  // x, the z scratch and the outputs belong to earlier work on the stream
+    {
+        const int row_units = p.d / 8;
+        const uint4 *x = static_cast<const uint4 *>(p.x);
+        const uint4 zero = make_uint4(0, 0, 0, 0);
+        for (int u = tid; u < 2 * vec_units; u += ST_THREADS) {
+            const int slot = u >= vec_units ? 1 : 0, uu = u - slot * vec_units, b = h1.b0 + slot;
+            vec[u] = (uu < row_units && b < p.B) ? __ldcg(x + (size_t)b * row_units + uu) : zero;
+        }
+    }
+    __syncthreads();
+    h1.run(p, A, Bq, vec, vec_units, part, act);
+    __syncthreads();  // the partial sums are in place, nobody reads x any more
+    combine_partials<FIRST>(p, part, act, tid);
+
+    // ---- meeting point, with the first weights of the second half on their way
+    StreamHalf<ST_DOWN> h2;
+    h2.init(p, warp, lane);
+    h2.prologue(p, A, Bq);
+    __syncthreads();  // every z entry of this CTA is written (thread 0's fence makes them visible device-wide)
+    if (tid == 0) grid_meet(&static_cast<WsHeader *>(p.ws)->meet_stream, gridDim.x, abort, p.ws);
+    if (tid < 2 * ST_WARPS) part[tid].f = -1;
+    __syncthreads();
+    if (*abort) return;  // the wait gave up (status raised): nothing of this CTA is in flight but loads into registers
+    {
+        // z of the two sequences, read through L2 (other CTAs wrote it), entries from k on cleared
+        const int row_units = p.ldk / 8;
+        const uint4 zero = make_uint4(0, 0, 0, 0);
+        for (int u = tid; u < 2 * vec_units; u += ST_THREADS) {
+            const int slot = u >= vec_units ? 1 : 0, uu = u - slot * vec_units, b = h2.b0 + slot;
+            uint4 v = zero;
+            if (uu < row_units && 8 * uu < p.k && b < p.B) {
+                v = __ldcg(reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(p.z) + (size_t)b * 2 * p.ldk) + uu);
+                if (8 * uu + 8 > p.k) v = keep_elems(v, p.k - 8 * uu);
+            }
+            vec[u] = v;
+        }
+    }
+    __syncthreads();
+    h2.run(p, A, Bq, vec, vec_units, part, act);
+    __syncthreads();
+    combine_partials<ST_DOWN>(p, part, act, tid);
+}
+
+griffin_status decode_bf16_stream(DecodeParams &p, int act, bool gated, uint32_t flags, cudaStream_t stream) {
+    const int sms = device_sm_count();
+    if (sms <= 0) return GRIFFIN_ERR_CUDA;
+    if (p.ws == nullptr) return GRIFFIN_ERR_WORKSPACE;  // the meeting point's counter lives in the header
+    const int grid = sms;
+    if (p.B > grid) return GRIFFIN_ERR_UNSUPPORTED;  // a CTA's range must not span more than two sequences
+    const bool overlap = (flags & GRIFFIN_DECODE_OVERLAP_WEIGHT_PREFETCH) != 0;
+    const int units = max(p.d, p.ldk) / 8;
+    int vec_units = (units + ST_STEP_UNITS - 1) / ST_STEP_UNITS * ST_STEP_UNITS;
+    const size_t smem = (size_t)2 * vec_units * 16 + 2 * ST_WARPS * sizeof(StreamPartial) + 16;
+    if (smem > 227 * 1024) return GRIFFIN_ERR_UNSUPPORTED;
+    const void *fn = gated ? (const void *)decode_stream_kernel<true> : (const void *)decode_stream_kernel<false>;
+    if (ensure_dynamic_smem(fn, smem) != cudaSuccess) return GRIFFIN_ERR_CUDA;
+    // every CTA of the grid must be able to run at the same time (they meet half-way): one per SM
+    if (!grid_can_meet(fn, ST_THREADS, smem, grid)) return GRIFFIN_ERR_UNSUPPORTED;
+    void *args[] = {&p, &act, &vec_units};
+    if (launch_maybe_overlapped(fn, dim3(grid), dim3(ST_THREADS), smem, stream, overlap, args) != cudaSuccess)
+        return GRIFFIN_ERR_CUDA;
+    return GRIFFIN_OK;
+}
+
+}  // namespace griffin
