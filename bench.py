@@ -83,6 +83,15 @@ def measured_peaks():
         return FALLBACK_HBM_GBS, 1590.0, 1400.0, "fallback (6.65 TB/s, 1.59 / 1.40 PFLOP/s: earlier measurements on this pool)"
 
 
+def decode_kernel_name(w, B, k):
+    """Which of the two warp-level kernels griffin_ff_decode picks for sequences with their own sets (bf16): the
+    register stream from about 200 MB of compact weights per call, the shared-memory ring below (the rule stated
+    with GRIFFIN_DECODE_RING / GRIFFIN_DECODE_STREAM in include/griffin_ff.h)."""
+    if w.dtype != "bf16":
+        return "decode_gate_up_kernel + decode_down_kernel"
+    return "decode_stream_kernel" if B * 3 * k * w.d * 2 >= 200e6 else "decode_fused_kernel"
+
+
 def recorded_traffic(key):
     """DRAM bytes per launch of the dominant kernel from the committed ncu summary of this workload, if the
     kernel's sources are unchanged since that capture; otherwise None."""
@@ -641,7 +650,8 @@ def run_ours(args, w, keep):
             "config": workload_config(w, L, B, keep, world, indexed, job.graph is not None, job.shared_set),
             "phases": dict(rep, note="medians over the timed steps of per-phase CUDA-event times"),
             "roofline": {"bound": "hbm", "kernel": ("decode_indexed_kernel" if indexed else
-                                                    "decode_shared_kernel" if job.shared_set else "decode_fused_kernel") +
+                                                    "decode_shared_kernel" if job.shared_set else
+                                                    decode_kernel_name(w, B, job.k)) +
                          " (one launch per decode call; the decode phase is "
                          f"{100.0 * ph_ms[3] / sum(ph_ms):.0f} % of the step)", "achieved": dec["gbs"],
                          "peak": peaks[0], "unit": "GB/s", "frac": dec["frac_of_hbm"], "peak_source": peaks[3],

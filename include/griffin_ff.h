@@ -136,7 +136,7 @@ typedef struct {
 /* Flags of griffin_ff_decode. */
 #define GRIFFIN_DECODE_DEFAULT 0u
 /* Launch the decode kernels with programmatic dependent launch: each kernel may begin
- * streaming its (read-only) weights into shared memory while the previous kernel on the
+ * streaming its (read-only) weights into shared memory or registers while the previous kernel on the
  * stream is still finishing; it reads x and writes y / the workspace only after that
  * kernel has completed.  The caller promises that no earlier work still running on the
  * stream WRITES the compact weights this call reads (do not set it on the first decode
@@ -149,6 +149,18 @@ typedef struct {
  * measured workloads the warp-level kernels are the faster ones, which is why they are the
  * default. */
 #define GRIFFIN_DECODE_TCGEN05 2u
+/* bf16, sequences with their own expert sets: which of the two warp-level kernels runs.  Both make
+ * one pass over the compact weights and hand them to mma.sync; they differ in how the weights
+ * travel.  RING: bulk copies (TMA) by a producer warp into a ring of shared-memory stages that two
+ * groups of consumer warps read.  STREAM: every one of 16 warps loads its own rows straight into
+ * registers with plain 16-byte loads, two steps deep.  Without either flag the call picks by size:
+ * the register stream is the faster one once every warp has enough to do (about 200 MB of weights
+ * per call on a B200: 6.7 TB/s against 6.0-6.3 on the Llama-2-13B shape with 8 sets), the ring
+ * when the call is so short that filling and draining 2368 separate pipelines shows (Llama-2-7B
+ * shape, one sequence: 24.8 against 26.4 us).  Giving both is an error.  Results of the two agree
+ * within the documented tolerance (the sums are taken in different orders). */
+#define GRIFFIN_DECODE_RING 4u
+#define GRIFFIN_DECODE_STREAM 8u
 
 /* Status text for a code (static string, never NULL). */
 const char *griffin_status_string(griffin_status st);

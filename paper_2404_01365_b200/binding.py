@@ -18,7 +18,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ER
 ACT_SWIGLU, ACT_GEGLU_TANH, ACT_REGLU, ACT_GEGLU_ERF = 0, 1, 2, 3
 ACT_RELU, ACT_GELU_TANH, ACT_GELU_ERF, ACT_SILU = 4, 5, 6, 7   # blocks without a gate (Eq. 2): w_gate is None
 DT_F32, DT_BF16 = 0, 1
-DECODE_DEFAULT, DECODE_OVERLAP_WEIGHT_PREFETCH, DECODE_TCGEN05 = 0, 1, 2
+DECODE_DEFAULT, DECODE_OVERLAP_WEIGHT_PREFETCH, DECODE_TCGEN05, DECODE_RING, DECODE_STREAM = 0, 1, 2, 4, 8
 MAX_BATCH = 32
 
 ACT_BY_NAME = {"swiglu": ACT_SWIGLU, "geglu_tanh": ACT_GEGLU_TANH, "reglu": ACT_REGLU, "geglu_erf": ACT_GEGLU_ERF,

@@ -254,7 +254,9 @@ griffin_status griffin_ff_decode(const griffin_ff_desc *desc, int32_t B, const g
     if (sets == nullptr || x == nullptr || y == nullptr) return GRIFFIN_ERR_INVALID_ARG;
     if (B < 1) return GRIFFIN_ERR_INVALID_ARG;
     if (B > GRIFFIN_MAX_BATCH || desc->d > GRIFFIN_MAX_D) return GRIFFIN_ERR_UNSUPPORTED;
-    if (flags & ~(GRIFFIN_DECODE_OVERLAP_WEIGHT_PREFETCH | GRIFFIN_DECODE_TCGEN05)) return GRIFFIN_ERR_INVALID_ARG;
+    if (flags & ~(GRIFFIN_DECODE_OVERLAP_WEIGHT_PREFETCH | GRIFFIN_DECODE_TCGEN05 | GRIFFIN_DECODE_RING | GRIFFIN_DECODE_STREAM))
+        return GRIFFIN_ERR_INVALID_ARG;
+    if ((flags & GRIFFIN_DECODE_RING) && (flags & GRIFFIN_DECODE_STREAM)) return GRIFFIN_ERR_INVALID_ARG;
     for (int b = 0; b < B; ++b) {
         st = check_compact(desc, &sets[b]);
         if (st != GRIFFIN_OK) return st;
@@ -296,7 +298,9 @@ griffin_status griffin_ff_decode_static(const griffin_ff_desc *desc, int32_t B, 
     if (sets == nullptr || x == nullptr || y == nullptr) return GRIFFIN_ERR_INVALID_ARG;
     if (B < 1) return GRIFFIN_ERR_INVALID_ARG;
     if (B > GRIFFIN_MAX_BATCH || desc->d > GRIFFIN_MAX_D) return GRIFFIN_ERR_UNSUPPORTED;
-    if (flags & ~(GRIFFIN_DECODE_OVERLAP_WEIGHT_PREFETCH | GRIFFIN_DECODE_TCGEN05)) return GRIFFIN_ERR_INVALID_ARG;
+    if (flags & ~(GRIFFIN_DECODE_OVERLAP_WEIGHT_PREFETCH | GRIFFIN_DECODE_TCGEN05 | GRIFFIN_DECODE_RING | GRIFFIN_DECODE_STREAM))
+        return GRIFFIN_ERR_INVALID_ARG;
+    if ((flags & GRIFFIN_DECODE_RING) && (flags & GRIFFIN_DECODE_STREAM)) return GRIFFIN_ERR_INVALID_ARG;
     for (int b = 0; b < B; ++b) {
         st = check_compact(desc, &sets[b]);
         if (st != GRIFFIN_OK) return st;

@@ -17,7 +17,6 @@
 //     kernel (x, z, y) is touched only after griddepcontrol.wait.
 // Results are deterministic: every sum has a fixed order.
 #include <atomic>
-#include <cstdlib>
 
 #include "decode_common.cuh"
 
@@ -392,6 +391,10 @@ static griffin_status decode_simt(DecodeParams &p, int act, bool gated, uint32_t
     return GRIFFIN_OK;
 }
 
+// Weight bytes of a call from which the register-streaming kernel is the default.
+#ifndef GRIFFIN_STREAM_MIN_MB
+#define GRIFFIN_STREAM_MIN_MB 200
+#endif
 griffin_status launch_decode(const griffin_ff_desc *desc, int B, const griffin_ff_compact *sets, const void *b_down,
                              const void *x, void *y, float *z, void *ws, uint32_t flags, cudaStream_t stream) {
     DecodeParams p = {};
@@ -420,8 +423,12 @@ griffin_status launch_decode(const griffin_ff_desc *desc, int B, const griffin_f
         const griffin_status st = decode_bf16_shared(p, act, gated, flags, stream);
         if (st != GRIFFIN_ERR_UNSUPPORTED) return st;
     }
-    static const bool use_stream = getenv("GRIFFIN_DECODE_STREAM") != nullptr;
-    if (use_stream && !want_tc) {
+    // sequences with their own sets: the register stream once every warp has enough to do, else the ring
+    // (a shape that the stream kernel cannot place goes to the ring kernel after all)
+    bool use_stream = (flags & GRIFFIN_DECODE_STREAM) != 0;
+    if (!use_stream && !(flags & GRIFFIN_DECODE_RING) && !want_tc)
+        use_stream = (size_t)B * 3 * p.k * p.d * 2 >= (size_t)GRIFFIN_STREAM_MIN_MB * 1000 * 1000;
+    if (use_stream) {
         const griffin_status st = decode_bf16_stream(p, act, gated, flags, stream);
         if (st != GRIFFIN_ERR_UNSUPPORTED) return st;
     }

@@ -1,19 +1,21 @@
 // Generation-phase pruned FF (Eqs. 4 and 5 of the GRIFFIN paper) for bf16 storage, streamed
 // through registers: ONE kernel per call, one persistent CTA of 16 warps per SM, no shared-memory
-// ring, no producer, no barriers on the way.
+// ring, no producer warp, no barriers on the way.
 //   first half   z_hat = sigma(W_g_hat x + b_g_hat) * (W_1_hat x + b_1_hat)
 //   meeting      every CTA has written its z entries; all CTAs wait for each other (bounded)
 //   second half  y_hat = W_2_hat z_hat + b_2
 //
 // Both halves are matrix-vector products whose cost is the single pass over the compact weights,
-// and a read-only stream of HBM runs fastest (measured on B200: 6.8-7.2 TB/s against 6.5 TB/s for
+// and a read-only stream of HBM runs fastest (measured on B200: 6.8-7.2 TB/s, against 6.5 TB/s for
 // a copy) when every warp keeps 8 KB of plain 16-byte loads in flight and does nothing else that
 // could hold them up.  So every warp streams weight rows straight from global memory into
 // registers, two steps deep (a step is 2 KB of each of the two rows of a "pair"), and hands them
 // to the warp-level tensor-core instruction mma.sync.m16n8k16, which takes the place of unpacking
 // and multiplying element by element (the diagonal of the 16 x 8 tile is the dot product, see
 // diagonal_sum).  The vector (x, then z) sits in shared memory, read conflict-free by the same
-// lane that holds the matching weights.
+// lane that holds the matching weights.  Where the CTA has to wait for others (for the previous
+// kernel on the stream, at the meeting point) each warp has, besides its two steps in registers,
+// one more on its way into shared memory by bulk copies (TMA), so that HBM stays busy meanwhile.
 //
 // Work split.  A pair is (gate row j, up row j) in the first half of a gated block, two
 // consecutive rows of W_1_hat (no gate) or of W_2_hat otherwise.  The B * P pairs of a half are
@@ -30,6 +32,10 @@ constexpr int ST_WARPS = 16;
 constexpr int ST_THREADS = ST_WARPS * 32;
 constexpr int ST_H = 4;                    // 16-byte units of each row of a pair, per lane and step
 constexpr int ST_STEP_UNITS = 32 * ST_H;   // units of a row that one step covers (2 KB)
+#ifndef GRIFFIN_ST_ACCS
+#define GRIFFIN_ST_ACCS 2
+#endif
+constexpr int ST_ACCS = GRIFFIN_ST_ACCS;            // independent accumulators of a warp (2 or 4)
 constexpr int ST_GATE_UP = 0, ST_DOWN = 1, ST_UP = 2;
 
 struct StreamPartial {  // what a warp has summed of a pair that it shares with its neighbours
@@ -44,13 +50,32 @@ struct StreamGeom {
     int row_units;  // 16-byte units per row
     int S;          // steps per row
 };
-template <int MODE> __device__ __forceinline__ StreamGeom stream_geom(const DecodeParams &p) {
+__device__ __forceinline__ StreamGeom stream_geom(const DecodeParams &p, int mode) {
     StreamGeom g;
-    g.rows = MODE == ST_DOWN ? p.d : p.k;
-    g.P = MODE == ST_GATE_UP ? g.rows : (g.rows + 1) / 2;
-    g.row_units = (MODE == ST_DOWN ? p.ldk : p.d) / 8;
+    g.rows = mode == ST_DOWN ? p.d : p.k;
+    g.P = mode == ST_GATE_UP ? g.rows : (g.rows + 1) / 2;
+    g.row_units = (mode == ST_DOWN ? p.ldk : p.d) / 8;
     g.S = (g.row_units + ST_STEP_UNITS - 1) / ST_STEP_UNITS;
     return g;
+}
+
+// This warp's share of a half: `first` is the CTA-wide... the pair that holds its first step, sp0 the
+// step within that pair, n the number of steps; b0 the sequence of the CTA's first pair.
+struct StreamRange {
+    int f0, sp0, n, b0;
+};
+__device__ __forceinline__ StreamRange stream_range(const DecodeParams &p, const StreamGeom &g, int warp) {
+    const long long T = (long long)p.B * g.P;
+    const int lo = (int)(T * blockIdx.x / gridDim.x), hi = (int)(T * (blockIdx.x + 1) / gridDim.x);
+    const int n = (hi - lo) * g.S;  // the CTA's steps
+    const int s0 = (int)((long long)n * warp / ST_WARPS), s1 = (int)((long long)n * (warp + 1) / ST_WARPS);
+    const int pr = s0 / g.S;
+    StreamRange r;
+    r.f0 = lo + pr;
+    r.sp0 = s0 - pr * g.S;
+    r.n = s1 - s0;
+    r.b0 = lo / g.P;
+    return r;
 }
 
 __device__ __forceinline__ uint4 ldg_stream(const uint4 *p) {
@@ -84,68 +109,73 @@ __device__ __forceinline__ void finish_pair(const DecodeParams &p, const StreamG
     }
 }
 
-// One warp's part of one half.  Usage: init, prologue (weights only: may run before anything the
-// half depends on is ready), then run.
+// One warp's part of one half.  The steps are loaded and multiplied in order; two register
+// buffers A and B hold the next two of them and are used in turn.
+//
+// What keeps HBM busy while the CTA waits for others (the previous kernel on the stream, the
+// meeting point) is loaded ahead, weights only:
+//   * the warp's first two steps of a half go into A and B;
+//   * up to `ahead` further steps go into the warp's own piece of shared memory by bulk copies
+//     (TMA) counted on the warp's own barrier, and are multiplied from there after the first two.
 template <int MODE>
 struct StreamHalf {
     StreamGeom g;
-    int lo, hi;          // the CTA's pairs [lo, hi) of the half's B * P
-    int b0;              // sequence of pair lo (its vector is slot 0, the next sequence's slot 1)
+    int b0;              // sequence of the CTA's first pair (its vector is slot 0, the next sequence's slot 1)
     int f_slot1;         // first pair of sequence b0 + 1
-    int full_steps;      // steps of a row with every lane inside the row
     int n_issue, n_comp; // steps of this warp not yet loaded / not yet multiplied
+    int n_staged;        // steps of this warp staged in shared memory
     bool mid;            // the pair being summed began in another warp
-    // load cursor: pair, step within it, this lane's unit 0 of the pair's rows
+    // load cursor: pair, step within it, unit 0 of the pair's rows
     int lf, lsp;
     const uint4 *r0, *r1;
     bool two;
-    // the steps held in registers A and B
-    int af, asp, bf, bsp;
+    // compute cursor
+    int cf, csp;
     int lane, warp;
 
     __device__ __forceinline__ void set_pair(const DecodeParams &p, int f) {
         const int b = f / g.P, j = f - b * g.P;
         if (MODE == ST_GATE_UP) {
-            r0 = static_cast<const uint4 *>(p.seq[b].w_gate) + (size_t)j * g.row_units + lane;
-            r1 = static_cast<const uint4 *>(p.seq[b].w_up) + (size_t)j * g.row_units + lane;
+            r0 = static_cast<const uint4 *>(p.seq[b].w_gate) + (size_t)j * g.row_units;
+            r1 = static_cast<const uint4 *>(p.seq[b].w_up) + (size_t)j * g.row_units;
             two = true;
         } else {
             const void *m = MODE == ST_DOWN ? p.seq[b].w_down : p.seq[b].w_up;
-            r0 = static_cast<const uint4 *>(m) + (size_t)(2 * j) * g.row_units + lane;
+            r0 = static_cast<const uint4 *>(m) + (size_t)(2 * j) * g.row_units;
             r1 = r0 + g.row_units;
             two = 2 * j + 1 < g.rows;
+        }
+    }
+    __device__ __forceinline__ void advance_load(const DecodeParams &p) {
+        --n_issue;
+        if (++lsp == g.S) {
+            lsp = 0;
+            ++lf;
+            if (n_issue > 0) set_pair(p, lf);
         }
     }
 
     __device__ __forceinline__ void init(const DecodeParams &p, int warp_, int lane_) {
         warp = warp_;
         lane = lane_;
-        g = stream_geom<MODE>(p);
-        const long long T = (long long)p.B * g.P;
-        lo = (int)(T * blockIdx.x / gridDim.x);
-        hi = (int)(T * (blockIdx.x + 1) / gridDim.x);
-        b0 = lo / g.P;
+        g = stream_geom(p, MODE);
+        const StreamRange r = stream_range(p, g, warp);
+        b0 = r.b0;
         f_slot1 = (b0 + 1) * g.P;
-        full_steps = g.row_units / ST_STEP_UNITS;
-        const int n = (hi - lo) * g.S;  // the CTA's steps
-        const int s0 = (int)((long long)n * warp / ST_WARPS), s1 = (int)((long long)n * (warp + 1) / ST_WARPS);
-        n_issue = n_comp = s1 - s0;
-        const int pr = s0 / g.S;
-        lf = lo + pr;
-        lsp = s0 - pr * g.S;
+        n_issue = n_comp = r.n;
+        n_staged = 0;
+        cf = lf = r.f0;
+        csp = lsp = r.sp0;
         mid = lsp != 0;
-        af = asp = bf = bsp = 0;
         r0 = r1 = nullptr;
         two = false;
         if (n_issue > 0) set_pair(p, lf);
     }
 
-    // Loads the next step into r and moves the cursor on.
-    __device__ __forceinline__ void issue(const DecodeParams &p, uint4 (&r)[2 * ST_H], int &mf, int &msp) {
-        mf = lf;
-        msp = lsp;
-        const int u0 = lsp * ST_STEP_UNITS;
-        if (lsp < full_steps && two) {  // (warp-uniform) the common case: nothing to guard
+    // Loads the next step into r and moves the load cursor on.
+    __device__ __forceinline__ void issue(const DecodeParams &p, uint4 (&r)[2 * ST_H]) {
+        const int u0 = lsp * ST_STEP_UNITS + lane;
+        if ((lsp + 1) * ST_STEP_UNITS <= g.row_units && two) {  // (warp-uniform) the common case: nothing to guard
 #pragma unroll
             for (int i = 0; i < ST_H; ++i) {
                 r[i] = ldg_stream(r0 + u0 + i * 32);
@@ -155,72 +185,125 @@ struct StreamHalf {
             const uint4 zero = make_uint4(0, 0, 0, 0);
 #pragma unroll
             for (int i = 0; i < ST_H; ++i) {
-                const bool in = u0 + i * 32 + lane < g.row_units;
+                const bool in = u0 + i * 32 < g.row_units;
                 r[i] = in ? ldg_stream(r0 + u0 + i * 32) : zero;
                 r[ST_H + i] = (in && two) ? ldg_stream(r1 + u0 + i * 32) : zero;
             }
         }
-        --n_issue;
-        if (++lsp == g.S) {
-            lsp = 0;
-            ++lf;
-            if (n_issue > 0) set_pair(p, lf);
-        }
+        advance_load(p);
     }
 
-    // The warp's first two steps: what is in flight while the CTA waits for others.
-    __device__ __forceinline__ void prologue(const DecodeParams &p, uint4 (&A)[2 * ST_H], uint4 (&Bq)[2 * ST_H]) {
-        if (n_issue > 0) issue(p, A, af, asp);
-        if (n_issue > 0) issue(p, Bq, bf, bsp);
+    // stage: the warp's 2 * ST_STEP_UNITS * ahead units of shared memory; bar: its barrier for this half.
+    __device__ __forceinline__ void prologue(const DecodeParams &p, uint4 (&A)[2 * ST_H], uint4 (&Bq)[2 * ST_H], uint4 *stage,
+                                             uint64_t *bar, int ahead) {
+        if (n_issue > 0) issue(p, A);
+        if (n_issue > 0) issue(p, Bq);
+        uint32_t bytes = 0;
+        for (int s = 0; s < ahead && n_issue > 0; ++s, ++n_staged) {
+            const int u0 = lsp * ST_STEP_UNITS;
+            const uint32_t nb = (uint32_t)min(ST_STEP_UNITS, g.row_units - u0) * 16;
+            if (lane == 0) bulk_g2s(stage + s * 2 * ST_STEP_UNITS, r0 + u0, nb, bar);
+            if (lane == 1 && two) bulk_g2s(stage + (s * 2 + 1) * ST_STEP_UNITS, r1 + u0, nb, bar);
+            bytes += two ? 2 * nb : nb;
+            advance_load(p);
+        }
+        if (n_staged > 0 && lane == 0) mbar_arrive_expect_tx(bar, bytes);
     }
 
-    // Multiplies the step held in r and, at the end of a pair or of the warp's range, hands the sums on.
-    __device__ __forceinline__ void compute(const DecodeParams &p, const uint4 (&r)[2 * ST_H], int mf, int msp,
-                                            float (&acc)[4][4], const uint4 *vec, int vec_units, StreamPartial *part,
-                                            int act) {
-        const uint4 *v = vec + (mf >= f_slot1 ? vec_units : 0) + msp * ST_STEP_UNITS + lane;
-#pragma unroll
-        for (int i = 0; i < ST_H; ++i) {
-            const uint4 vv = v[i * 32];
-            mma_bf16(acc[(2 * i) & 3], r[i].x, r[ST_H + i].x, r[i].y, r[ST_H + i].y, vv.x, vv.y);
-            mma_bf16(acc[(2 * i + 1) & 3], r[i].z, r[ST_H + i].z, r[i].w, r[ST_H + i].w, vv.z, vv.w);
-        }
+    // The sums of a pair, or of this warp's piece of it, are complete: hand them on.
+    __device__ __forceinline__ void step_done(const DecodeParams &p, float (&acc)[ST_ACCS][4], StreamPartial *part, int act) {
         --n_comp;
-        const bool complete = msp == g.S - 1;
+        const bool complete = csp == g.S - 1;
         if (complete || n_comp == 0) {
             float sum[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                sum[e] = (acc[0][e] + acc[1][e]) + (acc[2][e] + acc[3][e]);
-                acc[0][e] = acc[1][e] = acc[2][e] = acc[3][e] = 0.f;
+                float t = 0.f;
+#pragma unroll
+                for (int a = 0; a < ST_ACCS; a += 2) t += acc[a][e] + acc[a + 1][e];
+                sum[e] = t;
+#pragma unroll
+                for (int a = 0; a < ST_ACCS; ++a) acc[a][e] = 0.f;
             }
             const float a0 = diagonal_sum(sum, lane);          // lane 0: first row, lane 4: second row
             const float a1 = __shfl_sync(0xffffffffu, a0, 4);
             if (lane == 0) {
                 if (complete && !mid) {
-                    finish_pair<MODE>(p, g, act, mf, a0, a1);
+                    finish_pair<MODE>(p, g, act, cf, a0, a1);
                 } else {
                     StreamPartial *s = part + 2 * warp + (mid ? 0 : 1);
-                    s->f = mf;
+                    s->f = cf;
                     s->a0 = a0;
                     s->a1 = a1;
                 }
             }
             mid = false;
         }
+        if (++csp == g.S) {
+            csp = 0;
+            ++cf;
+        }
     }
 
-    // A and Bq hold the first two steps (prologue); every step multiplied makes room for the load of the one after next.
-    __device__ __forceinline__ void run(const DecodeParams &p, uint4 (&A)[2 * ST_H], uint4 (&Bq)[2 * ST_H], const uint4 *vec,
-                                        int vec_units, StreamPartial *part, int act) {
-        float acc[4][4] = {};
-        while (n_comp > 0) {
-            compute(p, A, af, asp, acc, vec, vec_units, part, act);
-            if (n_comp == 0) break;
-            if (n_issue > 0) issue(p, A, af, asp);
-            compute(p, Bq, bf, bsp, acc, vec, vec_units, part, act);
-            if (n_issue > 0) issue(p, Bq, bf, bsp);
+    // Multiplies the step held in r.
+    __device__ __forceinline__ void compute(const DecodeParams &p, const uint4 (&r)[2 * ST_H], float (&acc)[ST_ACCS][4],
+                                            const uint4 *vec, int vec_units, StreamPartial *part, int act) {
+        const uint4 *v = vec + (cf >= f_slot1 ? vec_units : 0) + csp * ST_STEP_UNITS + lane;
+#pragma unroll
+        for (int i = 0; i < ST_H; ++i) {
+            const uint4 vv = v[i * 32];
+            mma_bf16(acc[(2 * i) & (ST_ACCS - 1)], r[i].x, r[ST_H + i].x, r[i].y, r[ST_H + i].y, vv.x, vv.y);
+            mma_bf16(acc[(2 * i + 1) & (ST_ACCS - 1)], r[i].z, r[ST_H + i].z, r[i].w, r[ST_H + i].w, vv.z, vv.w);
         }
+        step_done(p, acc, part, act);
+    }
+
+    // Multiplies staged step s (the copies have landed).  A staged step may be the cut end of a row or half a pair.
+    __device__ __forceinline__ void compute_staged(const DecodeParams &p, const uint4 *stage, int s, float (&acc)[ST_ACCS][4],
+                                                   const uint4 *vec, int vec_units, StreamPartial *part, int act) {
+        const uint4 *v = vec + (cf >= f_slot1 ? vec_units : 0) + csp * ST_STEP_UNITS + lane;
+        const uint4 *w = stage + s * 2 * ST_STEP_UNITS + lane;
+        const int u0 = csp * ST_STEP_UNITS + lane;
+        const bool second = MODE == ST_GATE_UP || 2 * (cf - (cf / g.P) * g.P) + 1 < g.rows;
+        const uint4 zero = make_uint4(0, 0, 0, 0);
+#pragma unroll
+        for (int i = 0; i < ST_H; ++i) {
+            const bool in = u0 + i * 32 < g.row_units;
+            const uint4 a = in ? w[i * 32] : zero;
+            const uint4 b = (in && second) ? w[ST_STEP_UNITS + i * 32] : zero;
+            const uint4 vv = v[i * 32];
+            mma_bf16(acc[(2 * i) & (ST_ACCS - 1)], a.x, b.x, a.y, b.y, vv.x, vv.y);
+            mma_bf16(acc[(2 * i + 1) & (ST_ACCS - 1)], a.z, b.z, a.w, b.w, vv.z, vv.w);
+        }
+        step_done(p, acc, part, act);
+    }
+
+    // All of this warp's steps of the half; A and Bq hold steps 0 and 1, the staged steps follow them.
+    // Returns false when the wait for the staged steps gave up.
+    __device__ __forceinline__ bool run(const DecodeParams &p, uint4 (&A)[2 * ST_H], uint4 (&Bq)[2 * ST_H], const uint4 *stage,
+                                        uint64_t *bar, const uint4 *vec, int vec_units, StreamPartial *part,
+                                        volatile int *abort, int act) {
+        float acc[ST_ACCS][4] = {};
+        if (n_comp > 0) {
+            compute(p, A, acc, vec, vec_units, part, act);
+            if (n_issue > 0) issue(p, A);
+        }
+        if (n_comp > 0) {
+            compute(p, Bq, acc, vec, vec_units, part, act);
+            if (n_issue > 0) issue(p, Bq);
+        }
+        if (n_staged > 0) {
+            if (!wait_or_abort(bar, 0, abort, p.ws, MODE == ST_DOWN ? 11 : 10)) return false;
+            for (int s = 0; s < n_staged; ++s) compute_staged(p, stage, s, acc, vec, vec_units, part, act);
+        }
+        while (n_comp > 0) {
+            compute(p, A, acc, vec, vec_units, part, act);
+            if (n_issue > 0) issue(p, A);
+            if (n_comp == 0) break;
+            compute(p, Bq, acc, vec, vec_units, part, act);
+            if (n_issue > 0) issue(p, Bq);
+        }
+        return true;
     }
 };
 
@@ -243,7 +326,7 @@ __device__ __forceinline__ void combine_partials(const DecodeParams &p, const St
         a0 += o.a0;
         a1 += o.a1;
     }
-    const StreamGeom g = stream_geom<MODE>(p);
+    const StreamGeom g = stream_geom(p, MODE);
     finish_pair<MODE>(p, g, act, me.f, a0, a1);
 }
 
@@ -258,21 +341,41 @@ __device__ __forceinline__ uint4 keep_elems(uint4 v, int keep) {
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
+// After a give-up: the copies this warp started may still be on their way into its shared memory,
+// which must not be handed back under them.  One more bounded wait (normally over at once).
+__device__ __forceinline__ void drain_staged(uint64_t *bar, int n_staged) {
+    if (n_staged == 0 || mbar_try_wait(bar, 0)) return;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, 0))
+        if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
+}
+
 template <bool GATED>
 __global__ void __launch_bounds__(ST_THREADS, 1) decode_stream_kernel(const __grid_constant__ DecodeParams p, int act,
-                                                                    int vec_units) {
+                                                                    int vec_units, int ahead) {
     constexpr int FIRST = GATED ? ST_GATE_UP : ST_UP;
     extern __shared__ __align__(128) uint8_t smem_raw[];
     uint4 *vec = reinterpret_cast<uint4 *>(smem_raw);                       // two vectors of vec_units units
     StreamPartial *part = reinterpret_cast<StreamPartial *>(vec + 2 * vec_units);
     volatile int *abort = reinterpret_cast<volatile int *>(part + 2 * ST_WARPS);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(const_cast<int *>(abort) + 4);  // [2 halves][ST_WARPS]
+    uint4 *stages = reinterpret_cast<uint4 *>(bars + 2 * ST_WARPS);                 // [ST_WARPS][ahead] steps
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    uint4 A[2 * ST_H], Bq[2 * ST_H];
+    uint4 *stage = stages + (size_t)warp * ahead * 2 * ST_STEP_UNITS;
+    uint64_t *bar1 = bars + warp, *bar2 = bars + ST_WARPS + warp;
+
+    if (lane == 0) {
+        mbar_init(bar1, 1);
+        mbar_init(bar2, 1);
+        mbar_fence_init();
+    }
+    __syncwarp();
 
     // ---- first half: the first weights are on their way before anything else happens
+    uint4 A[2 * ST_H], Bq[2 * ST_H];
     StreamHalf<FIRST> h1;
     h1.init(p, warp, lane);
-    h1.prologue(p, A, Bq);
+    h1.prologue(p, A, Bq, stage, bar1, ahead);
     pdl_launch_dependents();
     if (tid == 0) *abort = 0;
     if (tid < 2 * ST_WARPS) part[tid].f = -1;
@@ -287,19 +390,28 @@ __global__ void __launch_bounds__(ST_THREADS, 1) decode_stream_kernel(const __gr
         }
     }
     __syncthreads();
-    h1.run(p, A, Bq, vec, vec_units, part, act);
+    h1.run(p, A, Bq, stage, bar1, vec, vec_units, part, abort, act);
     __syncthreads();  // the partial sums are in place, nobody reads x any more
+    if (*abort) {  // the meeting still gets this CTA's arrival: the others are not held up and the counter stays in phase
+        if (tid == 0) grid_arrive_only(&static_cast<WsHeader *>(p.ws)->meet_stream, gridDim.x);
+        drain_staged(bar1, h1.n_staged);
+        return;
+    }
     combine_partials<FIRST>(p, part, act, tid);
 
     // ---- meeting point, with the first weights of the second half on their way
     StreamHalf<ST_DOWN> h2;
     h2.init(p, warp, lane);
-    h2.prologue(p, A, Bq);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the staged steps of the first half have been read
+    h2.prologue(p, A, Bq, stage, bar2, ahead);
     __syncthreads();  // every z entry of this CTA is written (thread 0's fence makes them visible device-wide)
     if (tid == 0) grid_meet(&static_cast<WsHeader *>(p.ws)->meet_stream, gridDim.x, abort, p.ws);
     if (tid < 2 * ST_WARPS) part[tid].f = -1;
     __syncthreads();
-    if (*abort) return;  // the wait gave up (status raised): nothing of this CTA is in flight but loads into registers
+    if (*abort) {  // the wait gave up (status raised)
+        drain_staged(bar2, h2.n_staged);
+        return;
+    }
     {
         // z of the two sequences, read through L2 (other CTAs wrote it), entries from k on cleared
         const int row_units = p.ldk / 8;
@@ -315,11 +427,19 @@ __global__ void __launch_bounds__(ST_THREADS, 1) decode_stream_kernel(const __gr
         }
     }
     __syncthreads();
-    h2.run(p, A, Bq, vec, vec_units, part, act);
+    h2.run(p, A, Bq, stage, bar2, vec, vec_units, part, abort, act);
     __syncthreads();
+    if (*abort) {
+        drain_staged(bar2, h2.n_staged);
+        return;
+    }
     combine_partials<ST_DOWN>(p, part, act, tid);
 }
 
+#ifndef GRIFFIN_ST_AHEAD
+#define GRIFFIN_ST_AHEAD 1
+#endif
+constexpr size_t ST_SMEM_BUDGET = 128 * 1024;  // shared memory that vectors and staged steps may take together
 griffin_status decode_bf16_stream(DecodeParams &p, int act, bool gated, uint32_t flags, cudaStream_t stream) {
     const int sms = device_sm_count();
     if (sms <= 0) return GRIFFIN_ERR_CUDA;
@@ -329,13 +449,21 @@ griffin_status decode_bf16_stream(DecodeParams &p, int act, bool gated, uint32_t
     const bool overlap = (flags & GRIFFIN_DECODE_OVERLAP_WEIGHT_PREFETCH) != 0;
     const int units = max(p.d, p.ldk) / 8;
     int vec_units = (units + ST_STEP_UNITS - 1) / ST_STEP_UNITS * ST_STEP_UNITS;
-    const size_t smem = (size_t)2 * vec_units * 16 + 2 * ST_WARPS * sizeof(StreamPartial) + 16;
-    if (smem > 227 * 1024) return GRIFFIN_ERR_UNSUPPORTED;
+    const size_t fixed = (size_t)2 * vec_units * 16 + 2 * ST_WARPS * sizeof(StreamPartial) + 16 + 2 * ST_WARPS * sizeof(uint64_t);
+    if (fixed > 227 * 1024) return GRIFFIN_ERR_UNSUPPORTED;
+    // Steps per warp staged in shared memory across the waits.  Shared memory is taken from the
+    // same 256 KB as the L1 cache, which the loads in flight pass through: measured on B200, with
+    // 221 KB of shared memory (three staged steps) the stream drops from 6.7 to 5.9 TB/s, with up
+    // to 157 KB (two) it is unharmed.  One step (64 KB) covers the waits as well as two do.
+    const size_t per_step = (size_t)ST_WARPS * 2 * ST_STEP_UNITS * 16;
+    int ahead = fixed < ST_SMEM_BUDGET ? (int)((ST_SMEM_BUDGET - fixed) / per_step) : 0;
+    if (ahead > GRIFFIN_ST_AHEAD) ahead = GRIFFIN_ST_AHEAD;
+    const size_t smem = fixed + ahead * per_step;
     const void *fn = gated ? (const void *)decode_stream_kernel<true> : (const void *)decode_stream_kernel<false>;
     if (ensure_dynamic_smem(fn, smem) != cudaSuccess) return GRIFFIN_ERR_CUDA;
     // every CTA of the grid must be able to run at the same time (they meet half-way): one per SM
     if (!grid_can_meet(fn, ST_THREADS, smem, grid)) return GRIFFIN_ERR_UNSUPPORTED;
-    void *args[] = {&p, &act, &vec_units};
+    void *args[] = {&p, &act, &vec_units, &ahead};
     if (launch_maybe_overlapped(fn, dim3(grid), dim3(ST_THREADS), smem, stream, overlap, args) != cudaSuccess)
         return GRIFFIN_ERR_CUDA;
     return GRIFFIN_OK;

@@ -106,7 +106,8 @@ def test_host_validation_rejects_before_any_launch(lib):
     sets = (G.FFCompact * 2)(out, out)
     assert dcd(C.byref(desc), 0, sets, None, fake, fake, fake, 1 << 30, 0, None) == G.ERR_INVALID_ARG
     assert dcd(C.byref(desc), 33, sets, None, fake, fake, fake, 1 << 30, 0, None) == G.ERR_UNSUPPORTED
-    assert dcd(C.byref(desc), 2, sets, None, fake, fake, fake, 1 << 30, 8, None) == G.ERR_INVALID_ARG
+    assert dcd(C.byref(desc), 2, sets, None, fake, fake, fake, 1 << 30, 16, None) == G.ERR_INVALID_ARG   # an unknown flag
+    assert dcd(C.byref(desc), 2, sets, None, fake, fake, fake, 1 << 30, G.DECODE_RING | G.DECODE_STREAM, None) == G.ERR_INVALID_ARG
     assert dcd(C.byref(desc), 2, sets, None, fake, fake, fake, 100, 0, None) == G.ERR_WORKSPACE
     assert dcd(C.byref(desc), 2, sets, None, odd, fake, fake, 1 << 30, 0, None) == G.ERR_ALIGNMENT
     mixed = (G.FFCompact * 2)(out, G.FFCompact(fake, fake, fake, None, None, 336, 336))

@@ -123,12 +123,17 @@ DECODE_SHAPES = [
     (8192, 1024, 512, 1),    # largest supported d
     (512, 9008, 9008, 1),    # rows of W_2_hat longer than one stage chunk (two chunks)
     (256, 20000, 16400, 2),  # three chunks per row, two sequences
+    (5120, 13824, 6912, 3),  # Llama-2-13B shape; with 3 sequences the CTAs' ranges of the register stream straddle them
 ]
 
+# The two warp-level kernels for sequences with their own sets (bf16), and the choice by size.
+DECODE_KERNELS = {"by_size": 0, "ring": G.DECODE_RING, "stream": G.DECODE_STREAM}
 
-@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+
+@pytest.mark.parametrize("dtype,kernel", [("f32", "by_size"), ("bf16", "by_size"), ("bf16", "ring"), ("bf16", "stream")])
 @pytest.mark.parametrize("d,d_ff,k,B", DECODE_SHAPES)
-def test_decode_matches_oracle(dtype, d, d_ff, k, B):
+def test_decode_matches_oracle(dtype, kernel, d, d_ff, k, B):
+    kf = DECODE_KERNELS[kernel]
     act = {3072: "geglu_tanh", 2048: "geglu_erf", 1000: "reglu"}.get(d, "swiglu")
     L, host = make_layer(d, d_ff, dtype, act=act, bias=(d_ff < 2000), seed=d + k, n_seq=B)
     rs = np.random.default_rng(d + k)
@@ -139,13 +144,39 @@ def test_decode_matches_oracle(dtype, d, d_ff, k, B):
         sets.append(L.compact(torch.from_numpy(e_np).to(dev())))
         c = O.compact_experts(e_np, h64(host, "wg"), h64(host, "wu"), h64(host, "wd"), h64(host, "bg"), h64(host, "bu"))
         refs.append(O.ff_pruned(np64(x[b]), c, act, h64(host, "bd")))
-    y = L.decode(sets, x)
-    y2 = L.decode(sets, x, G.DECODE_OVERLAP_WEIGHT_PREFETCH)
-    y3 = L.decode(sets, x, G.DECODE_OVERLAP_WEIGHT_PREFETCH)
+    y = L.decode(sets, x, kf)
+    y2 = L.decode(sets, x, kf | G.DECODE_OVERLAP_WEIGHT_PREFETCH)
+    y3 = L.decode(sets, x, kf | G.DECODE_OVERLAP_WEIGHT_PREFETCH)
     assert L.status() == G.OK
     for b in range(B):
         assert_output(np64(y[b]), refs[b], dtype, b)
     assert torch.equal(y, y2) and torch.equal(y, y3)   # deterministic, launch mode does not matter
+
+
+def test_decode_kernels_take_turns_on_one_workspace():
+    """The ring kernel and the register-streaming kernel keep separate meeting-point counters in the
+    workspace header, so calls of the two may alternate in any order."""
+    d, d_ff, k, B = 1024, 2816, 1408, 3
+    L, host = make_layer(d, d_ff, "bf16", seed=21, n_seq=B)
+    rs = np.random.default_rng(21)
+    sets = [L.compact(torch.from_numpy(np.sort(rs.choice(d_ff, size=k, replace=False)).astype(np.int32)).to(dev()))
+            for _ in range(B)]
+    x = rand((B, d), torch.bfloat16, 22)
+    first = {}
+    for kernel in ["ring", "stream", "stream", "ring", "stream", "ring", "ring", "stream"]:
+        y = L.decode(sets, x, DECODE_KERNELS[kernel] | G.DECODE_OVERLAP_WEIGHT_PREFETCH)
+        assert torch.equal(first.setdefault(kernel, y), y)
+    assert L.status() == G.OK
+    # the two sum in different orders: close, not equal
+    assert_output(np64(first["stream"]), np64(first["ring"]), "bf16")
+
+
+def test_decode_rejects_both_kernel_flags_at_once():
+    L, host = make_layer(256, 688, "bf16")
+    cs = L.compact(torch.arange(0, 688, 2, dtype=torch.int32, device=dev()))
+    with pytest.raises(G.GriffinError) as err:
+        L.decode([cs], rand((1, 256), torch.bfloat16, 1), G.DECODE_RING | G.DECODE_STREAM)
+    assert err.value.status == G.ERR_INVALID_ARG
 
 
 # Shapes that the opt-in tcgen05 kernel takes (d and ldk multiples of 128) and two that it hands
@@ -311,7 +342,8 @@ def test_decode_with_all_neurons_is_the_dense_ff(dtype):
     assert torch.equal(L.decode([cs, cs], x), y)
 
 
-def test_decode_many_steps_back_to_back_with_overlap():
+@pytest.mark.parametrize("kernel", ["ring", "stream"])
+def test_decode_many_steps_back_to_back_with_overlap(kernel):
     d, d_ff, k = 1024, 2816, 1408
     L, host = make_layer(d, d_ff, "bf16")
     e_np = np.arange(0, d_ff, 2, dtype=np.int32)
@@ -321,14 +353,16 @@ def test_decode_many_steps_back_to_back_with_overlap():
     arr = G.compact_array([cs])
     torch.cuda.synchronize()
     for t in range(16):
-        G.griffin_ff_decode(L.desc, arr, None, xs[t:t + 1], ys[t:t + 1], L.ws, G.DECODE_OVERLAP_WEIGHT_PREFETCH)
+        G.griffin_ff_decode(L.desc, arr, None, xs[t:t + 1], ys[t:t + 1], L.ws,
+                            G.DECODE_OVERLAP_WEIGHT_PREFETCH | DECODE_KERNELS[kernel])
     assert L.status() == G.OK
     c = O.compact_experts(e_np, h64(host, "wg"), h64(host, "wu"), h64(host, "wd"))
     ref = O.ff_pruned(np64(xs), c, "swiglu")
     assert_output(np64(ys), ref, "bf16")
 
 
-def test_decode_calls_replayed_from_a_cuda_graph_give_the_same_bits():
+@pytest.mark.parametrize("kernel", ["ring", "stream"])
+def test_decode_calls_replayed_from_a_cuda_graph_give_the_same_bits(kernel):
     """bench.py captures the decode calls of a step once and replays them: same kernels, same
     launch attributes (the overlapped-launch edges included), so the same bits."""
     d, d_ff, k, n = 1024, 2816, 1408, 6
@@ -341,7 +375,7 @@ def test_decode_calls_replayed_from_a_cuda_graph_give_the_same_bits():
     def calls(out):
         for t in range(n):
             G.griffin_ff_decode(L.desc, arr, None, xs[t:t + 1], out[t:t + 1], L.ws,
-                                G.DECODE_OVERLAP_WEIGHT_PREFETCH if t > 0 else G.DECODE_DEFAULT)
+                                (G.DECODE_OVERLAP_WEIGHT_PREFETCH if t > 0 else G.DECODE_DEFAULT) | DECODE_KERNELS[kernel])
 
     calls(y_direct)
     torch.cuda.synchronize()

@@ -108,9 +108,9 @@ DECODE_SHAPES = [
 ]
 
 
-@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("dtype,kernel", [("f32", 0), ("bf16", G.DECODE_RING), ("bf16", G.DECODE_STREAM)])
 @pytest.mark.parametrize("d,d_ff,k,B", DECODE_SHAPES)
-def test_decode_without_a_gate_matches_oracle(dtype, d, d_ff, k, B):
+def test_decode_without_a_gate_matches_oracle(dtype, kernel, d, d_ff, k, B):
     act = ACTS[(d // 8 + k) % 4]
     L, host = make_layer(d, d_ff, dtype, act=act, bias=(d_ff < 6000), seed=d + k, n_seq=B)
     rs = np.random.default_rng(d + k)
@@ -121,9 +121,9 @@ def test_decode_without_a_gate_matches_oracle(dtype, d, d_ff, k, B):
         sets.append(L.compact(torch.from_numpy(e_np).to(dev())))
         c = O.compact_experts(e_np, None, h64(host, "wu"), h64(host, "wd"), None, h64(host, "bu"))
         refs.append(O.ff_pruned(np64(x[b]), c, act, h64(host, "bd")))
-    y = L.decode(sets, x)
-    y2 = L.decode(sets, x, G.DECODE_OVERLAP_WEIGHT_PREFETCH)
-    y3 = L.decode(sets, x, G.DECODE_OVERLAP_WEIGHT_PREFETCH | G.DECODE_TCGEN05)   # (the flag falls back here)
+    y = L.decode(sets, x, kernel)
+    y2 = L.decode(sets, x, kernel | G.DECODE_OVERLAP_WEIGHT_PREFETCH)
+    y3 = L.decode(sets, x, kernel | G.DECODE_OVERLAP_WEIGHT_PREFETCH | G.DECODE_TCGEN05)   # (the flag falls back here)
     assert L.status() == G.OK
     for b in range(B):
         assert_output(np64(y[b]), refs[b], dtype, b)

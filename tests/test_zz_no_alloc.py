@@ -91,6 +91,14 @@ def test_static_scratch_decode_through_the_tcgen05_kernel_and_with_overlapped_la
     _two_calls_in_a_row(desc, sets, ws, xs, refs, torch.bfloat16, flags=G.DECODE_TCGEN05 | G.DECODE_OVERLAP_WEIGHT_PREFETCH)
 
 
+@pytest.mark.parametrize("kernel", [G.DECODE_RING, G.DECODE_STREAM])
+def test_static_scratch_decode_through_either_warp_level_kernel(kernel):
+    # both keep their meeting-point counter in the header in front of the static array
+    desc, sets, ws, xs, refs = _layer(1024, 2816, 1401, 3, torch.bfloat16, seed=41)
+    _two_calls_in_a_row(desc, sets, ws, xs, refs, torch.bfloat16, flags=kernel)
+    _two_calls_in_a_row(desc, sets, ws, xs, refs, torch.bfloat16, flags=kernel | G.DECODE_OVERLAP_WEIGHT_PREFETCH)
+
+
 def test_static_scratch_decode_of_a_block_without_a_gate():
     desc, sets, ws, xs, refs = _layer(512, 2048, 1000, 2, torch.bfloat16, seed=31, act="relu")
     _two_calls_in_a_row(desc, sets, ws, xs, refs, torch.bfloat16)
