@@ -101,6 +101,26 @@ __device__ __forceinline__ bool grid_meet(unsigned int *counter, unsigned int n,
     }
 }
 
+// The same in two steps, for a party that has other work to start between reporting in and waiting:
+// grid_arrive returns which half of the counter's round this call's arrivals fall into.
+__device__ __forceinline__ bool grid_arrive(unsigned int *counter, unsigned int n) {
+    __threadfence();
+    return atomicInc(counter, 2 * n - 1) >= n;
+}
+__device__ __forceinline__ bool grid_wait(const unsigned int *counter, unsigned int n, bool upper, volatile int *abort, void *ws) {
+    const long long t0 = clock64();
+    for (;;) {
+        const unsigned int v = ld_acquire_u32(counter);
+        if (upper ? v < n : v >= n) return true;
+        if (*abort) return false;
+        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+            *abort = 1;
+            raise_status(ws, DEV_STATUS_TIMEOUT, 9);
+            return false;
+        }
+    }
+}
+
 // The arrival alone, for a party that has given up on its work: the other parties of this launch are not
 // held up by it and the counter stays in phase for the next launch.
 __device__ __forceinline__ void grid_arrive_only(unsigned int *counter, unsigned int n) {

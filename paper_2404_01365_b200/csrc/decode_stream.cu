@@ -112,11 +112,16 @@ __device__ __forceinline__ void finish_pair(const DecodeParams &p, const StreamG
 // One warp's part of one half.  The steps are loaded and multiplied in order; two register
 // buffers A and B hold the next two of them and are used in turn.
 //
-// What keeps HBM busy while the CTA waits for others (the previous kernel on the stream, the
-// meeting point) is loaded ahead, weights only:
-//   * the warp's first two steps of a half go into A and B;
+// Every answer from the memory system reaches an SM in the order it was asked for, at the SM's share
+// of the bandwidth: whatever a CTA asks for while it waits for others (for the previous kernel on the
+// stream before it may read x, for the meeting point before it may read z) is not lost time as long
+// as something is still on its way when the wait ends and the vector has been read.  So, weights only:
+//   * the warp's first two steps of a half go into A and B as early as possible: at the start of
+//     the kernel, and for the second half as soon as the warp has multiplied its last step of the first;
 //   * up to `ahead` further steps go into the warp's own piece of shared memory by bulk copies
-//     (TMA) counted on the warp's own barrier, and are multiplied from there after the first two.
+//     (TMA) counted on the warp's own barrier, asked for right AFTER the loads of the vector, so that
+//     they are still arriving when the vector is there and the first multiplications free A and B
+//     for new loads.  They are multiplied from shared memory after the first two.
 template <int MODE>
 struct StreamHalf {
     StreamGeom g;
@@ -193,11 +198,14 @@ struct StreamHalf {
         advance_load(p);
     }
 
-    // stage: the warp's 2 * ST_STEP_UNITS * ahead units of shared memory; bar: its barrier for this half.
-    __device__ __forceinline__ void prologue(const DecodeParams &p, uint4 (&A)[2 * ST_H], uint4 (&Bq)[2 * ST_H], uint4 *stage,
-                                             uint64_t *bar, int ahead) {
+    // The warp's first two steps, into the register buffers.
+    __device__ __forceinline__ void prologue_regs(const DecodeParams &p, uint4 (&A)[2 * ST_H], uint4 (&Bq)[2 * ST_H]) {
         if (n_issue > 0) issue(p, A);
         if (n_issue > 0) issue(p, Bq);
+    }
+    // Up to `ahead` further steps, into stage (the warp's 2 * ST_STEP_UNITS * ahead units of shared memory)
+    // by bulk copies counted on bar, the warp's barrier for this half.
+    __device__ __forceinline__ void prologue_staged(const DecodeParams &p, uint4 *stage, uint64_t *bar, int ahead) {
         uint32_t bytes = 0;
         for (int s = 0; s < ahead && n_issue > 0; ++s, ++n_staged) {
             const int u0 = lsp * ST_STEP_UNITS;
@@ -307,27 +315,43 @@ struct StreamHalf {
     }
 };
 
-// The pairs that were cut between warps: entry e = 2 * warp + (0: the warp's first pair, begun
-// elsewhere; 1: its last, ended elsewhere) is in step order, so the pieces of one pair follow each
-// other among the entries in use; the thread of a pair's first piece adds the rest to it.
+// The pairs that were cut between warps, added up by the first warp: entry e = 2 * warp + (0: the
+// warp's first pair, begun elsewhere; 1: its last, ended elsewhere) is in step order, so the pieces of
+// one pair follow each other among the entries in use.  Lane e holds entry e; the lane of a pair's
+// first piece collects the rest through shuffles, in entry order (a fixed order), and finishes the
+// pair.  (A loop over shared memory instead took 1.4 us at the end of each half.)
 template <int MODE>
-__device__ __forceinline__ void combine_partials(const DecodeParams &p, const StreamPartial *part, int act, int tid) {
-    if (tid >= 2 * ST_WARPS) return;
-    const StreamPartial me = part[tid];
-    if (me.f < 0) return;
-    int pe = tid - 1;
-    while (pe >= 0 && part[pe].f < 0) --pe;
-    if (pe >= 0 && part[pe].f == me.f) return;
+__device__ __forceinline__ void combine_partials(const DecodeParams &p, const StreamPartial *part, int act, int lane) {
+    static_assert(2 * ST_WARPS == 32, "one lane per entry");
+    const StreamPartial me = part[lane];
+    const bool valid = me.f >= 0;
+    const unsigned int mask = __ballot_sync(0xffffffffu, valid);
+    if (mask == 0) return;  // (warp-uniform) nothing was cut
+    const unsigned int below = mask & ((1u << lane) - 1u);
+    const int prev = below ? 31 - __clz(below) : lane;
+    const int f_prev = __shfl_sync(0xffffffffu, me.f, prev);
+    const bool head = valid && (below == 0 || f_prev != me.f);
     float a0 = me.a0, a1 = me.a1;
-    for (int e = tid + 1; e < 2 * ST_WARPS; ++e) {
-        const StreamPartial o = part[e];
-        if (o.f < 0) continue;
-        if (o.f != me.f) break;
-        a0 += o.a0;
-        a1 += o.a1;
+    bool open = head;  // still collecting
+    for (int j = 1; j < 32; ++j) {
+        const int f_j = __shfl_down_sync(0xffffffffu, me.f, j);
+        const float a0_j = __shfl_down_sync(0xffffffffu, me.a0, j);
+        const float a1_j = __shfl_down_sync(0xffffffffu, me.a1, j);
+        if (lane + j >= 32) open = false;
+        if (open && f_j >= 0) {
+            if (f_j == me.f) {
+                a0 += a0_j;
+                a1 += a1_j;
+            } else {
+                open = false;
+            }
+        }
+        if (!__any_sync(0xffffffffu, open)) break;
     }
-    const StreamGeom g = stream_geom(p, MODE);
-    finish_pair<MODE>(p, g, act, me.f, a0, a1);
+    if (head) {
+        const StreamGeom g = stream_geom(p, MODE);
+        finish_pair<MODE>(p, g, act, me.f, a0, a1);
+    }
 }
 
 // bf16 words of a 16-byte unit whose elements from `keep` on are cleared (keep in 1..7)
@@ -350,6 +374,52 @@ __device__ __forceinline__ void drain_staged(uint64_t *bar, int n_staged) {
         if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
 }
 
+__device__ __forceinline__ uint4 ld_cg_now(const uint4 *p) {  // through L2; volatile: stays where it is written
+    uint4 v;
+    asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+    return v;
+}
+
+// Stages the vectors of sequences b0 and b0 + 1 (x: row_units units each; z: the same with the entries
+// from k on cleared) as two rows of vec_units units, zero-filled.  The loads of the first
+// ST_VEC_EARLY units per thread are issued before `between` runs and stored after it: what `between`
+// asks the memory system for arrives behind the vector.
+constexpr int ST_VEC_EARLY = 4;
+template <bool IS_Z, class F>
+__device__ __forceinline__ void stage_vectors(const DecodeParams &p, uint4 *vec, int vec_units, int b0, int tid, F between) {
+    const int row_units = (IS_Z ? p.ldk : p.d) / 8;
+    const int limit = IS_Z ? p.k : p.d;  // elements that exist
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+    auto src_of = [&](int u, bool &in) -> const uint4 * {
+        const int slot = u >= vec_units ? 1 : 0, uu = u - slot * vec_units, b = b0 + slot;
+        in = u < 2 * vec_units && uu < row_units && 8 * uu < limit && b < p.B;
+        if (IS_Z) return reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(p.z) + (size_t)b * 2 * p.ldk) + uu;
+        return static_cast<const uint4 *>(p.x) + (size_t)b * row_units + uu;
+    };
+    auto fix = [&](uint4 v, int u) -> uint4 {
+        const int slot = u >= vec_units ? 1 : 0, uu = u - slot * vec_units;
+        return (IS_Z && 8 * uu + 8 > limit) ? keep_elems(v, limit - 8 * uu) : v;
+    };
+    uint4 early[ST_VEC_EARLY];
+#pragma unroll
+    for (int i = 0; i < ST_VEC_EARLY; ++i) {
+        bool in;
+        const uint4 *src = src_of(tid + i * ST_THREADS, in);
+        early[i] = in ? ld_cg_now(src) : zero;
+    }
+    between();
+#pragma unroll
+    for (int i = 0; i < ST_VEC_EARLY; ++i) {
+        const int u = tid + i * ST_THREADS;
+        if (u < 2 * vec_units) vec[u] = fix(early[i], u);
+    }
+    for (int u = tid + ST_VEC_EARLY * ST_THREADS; u < 2 * vec_units; u += ST_THREADS) {
+        bool in;
+        const uint4 *src = src_of(u, in);
+        vec[u] = in ? fix(__ldcg(src), u) : zero;
+    }
+}
+
 template <bool GATED>
 __global__ void __launch_bounds__(ST_THREADS, 1) decode_stream_kernel(const __grid_constant__ DecodeParams p, int act,
                                                                     int vec_units, int ahead) {
@@ -363,6 +433,7 @@ __global__ void __launch_bounds__(ST_THREADS, 1) decode_stream_kernel(const __gr
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     uint4 *stage = stages + (size_t)warp * ahead * 2 * ST_STEP_UNITS;
     uint64_t *bar1 = bars + warp, *bar2 = bars + ST_WARPS + warp;
+    unsigned int *const meet = &static_cast<WsHeader *>(p.ws)->meet_stream;
 
     if (lane == 0) {
         mbar_init(bar1, 1);
@@ -371,61 +442,57 @@ __global__ void __launch_bounds__(ST_THREADS, 1) decode_stream_kernel(const __gr
     }
     __syncwarp();
 
+    // Which half of its round the meeting-point counter is in.  Every CTA of the call before has passed its
+    // meeting (this CTA runs on an SM that one of them has left), and fewer than gridDim.x CTAs of this call
+    // can have reported in: the value read here and every arrival of this call fall into the same half.
+    // (Asked for before the weights, so that the answer does not queue behind them; needed at the meeting.)
+    unsigned int meet_at_start = 0;
+    if (tid == 0) meet_at_start = *reinterpret_cast<volatile unsigned int *>(meet);
+
     // ---- first half: the first weights are on their way before anything else happens
     uint4 A[2 * ST_H], Bq[2 * ST_H];
     StreamHalf<FIRST> h1;
     h1.init(p, warp, lane);
-    h1.prologue(p, A, Bq, stage, bar1, ahead);
+    h1.prologue_regs(p, A, Bq);
     pdl_launch_dependents();
     if (tid == 0) *abort = 0;
     if (tid < 2 * ST_WARPS) part[tid].f = -1;
     pdl_wait_prior_grids();  // x, the z scratch and the outputs belong to earlier work on the stream
-    {
-        const int row_units = p.d / 8;
-        const uint4 *x = static_cast<const uint4 *>(p.x);
-        const uint4 zero = make_uint4(0, 0, 0, 0);
-        for (int u = tid; u < 2 * vec_units; u += ST_THREADS) {
-            const int slot = u >= vec_units ? 1 : 0, uu = u - slot * vec_units, b = h1.b0 + slot;
-            vec[u] = (uu < row_units && b < p.B) ? __ldcg(x + (size_t)b * row_units + uu) : zero;
-        }
-    }
+    stage_vectors<false>(p, vec, vec_units, h1.b0, tid, [&]() { h1.prologue_staged(p, stage, bar1, ahead); });
     __syncthreads();
     h1.run(p, A, Bq, stage, bar1, vec, vec_units, part, abort, act);
+    // the first weights of the second half, as soon as this warp has room for them
+    StreamHalf<ST_DOWN> h2;
+    h2.init(p, warp, lane);
+    h2.prologue_regs(p, A, Bq);
     __syncthreads();  // the partial sums are in place, nobody reads x any more
     if (*abort) {  // the meeting still gets this CTA's arrival: the others are not held up and the counter stays in phase
-        if (tid == 0) grid_arrive_only(&static_cast<WsHeader *>(p.ws)->meet_stream, gridDim.x);
+        if (tid == 0) grid_arrive_only(meet, gridDim.x);
         drain_staged(bar1, h1.n_staged);
         return;
     }
-    combine_partials<FIRST>(p, part, act, tid);
-
-    // ---- meeting point, with the first weights of the second half on their way
-    StreamHalf<ST_DOWN> h2;
-    h2.init(p, warp, lane);
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the staged steps of the first half have been read
-    h2.prologue(p, A, Bq, stage, bar2, ahead);
-    __syncthreads();  // every z entry of this CTA is written (thread 0's fence makes them visible device-wide)
-    if (tid == 0) grid_meet(&static_cast<WsHeader *>(p.ws)->meet_stream, gridDim.x, abort, p.ws);
-    if (tid < 2 * ST_WARPS) part[tid].f = -1;
+    // ---- meeting point.  The first warp adds the cut pairs and reports this CTA in (thread 0's fence makes
+    //      every z entry of the CTA visible device-wide: the other warps wrote theirs before the barrier
+    //      above, the lanes of this warp before the __syncwarp).
+    if (warp == 0) {
+        combine_partials<FIRST>(p, part, act, lane);
+        part[lane].f = -1;
+        __syncwarp();
+        if (lane == 0) {
+            grid_arrive_only(meet, gridDim.x);  // (nothing waits for the answer: it would queue behind the weights)
+            grid_wait(meet, gridDim.x, meet_at_start >= gridDim.x, abort, p.ws);
+        }
+    }
     __syncthreads();
     if (*abort) {  // the wait gave up (status raised)
         drain_staged(bar2, h2.n_staged);
         return;
     }
-    {
-        // z of the two sequences, read through L2 (other CTAs wrote it), entries from k on cleared
-        const int row_units = p.ldk / 8;
-        const uint4 zero = make_uint4(0, 0, 0, 0);
-        for (int u = tid; u < 2 * vec_units; u += ST_THREADS) {
-            const int slot = u >= vec_units ? 1 : 0, uu = u - slot * vec_units, b = h2.b0 + slot;
-            uint4 v = zero;
-            if (uu < row_units && 8 * uu < p.k && b < p.B) {
-                v = __ldcg(reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(p.z) + (size_t)b * 2 * p.ldk) + uu);
-                if (8 * uu + 8 > p.k) v = keep_elems(v, p.k - 8 * uu);
-            }
-            vec[u] = v;
-        }
-    }
+    // z of the two sequences, read through L2 (other CTAs wrote it); the staged step is asked for behind it
+    stage_vectors<true>(p, vec, vec_units, h2.b0, tid, [&]() {
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the staged steps of the first half have been read
+        h2.prologue_staged(p, stage, bar2, ahead);
+    });
     __syncthreads();
     h2.run(p, A, Bq, stage, bar2, vec, vec_units, part, abort, act);
     __syncthreads();
@@ -433,7 +500,7 @@ __global__ void __launch_bounds__(ST_THREADS, 1) decode_stream_kernel(const __gr
         drain_staged(bar2, h2.n_staged);
         return;
     }
-    combine_partials<ST_DOWN>(p, part, act, tid);
+    if (warp == 0) combine_partials<ST_DOWN>(p, part, act, lane);
 }
 
 #ifndef GRIFFIN_ST_AHEAD

@@ -124,6 +124,9 @@ DECODE_SHAPES = [
     (512, 9008, 9008, 1),    # rows of W_2_hat longer than one stage chunk (two chunks)
     (256, 20000, 16400, 2),  # three chunks per row, two sequences
     (5120, 13824, 6912, 3),  # Llama-2-13B shape; with 3 sequences the CTAs' ranges of the register stream straddle them
+    (256, 688, 344, 32),     # the largest batch
+    (128, 64, 1, 2),         # one expert: most CTAs have nothing to do in the first half
+    (136, 200, 9, 5),        # rows shorter than one step, odd k, more sequences than pairs per CTA
 ]
 
 # The two warp-level kernels for sequences with their own sets (bf16), and the choice by size.
