@@ -85,11 +85,11 @@ def measured_peaks():
 
 def decode_kernel_name(w, B, k):
     """Which of the two warp-level kernels griffin_ff_decode picks for sequences with their own sets (bf16): the
-    register stream from about 200 MB of compact weights per call, the shared-memory ring below (the rule stated
+    register stream from about 150 MB of compact weights per call, the shared-memory ring below (the rule stated
     with GRIFFIN_DECODE_RING / GRIFFIN_DECODE_STREAM in include/griffin_ff.h)."""
     if w.dtype != "bf16":
         return "decode_gate_up_kernel + decode_down_kernel"
-    return "decode_stream_kernel" if B * 3 * k * w.d * 2 >= 200e6 else "decode_fused_kernel"
+    return "decode_stream_kernel" if B * 3 * k * w.d * 2 >= 150e6 else "decode_fused_kernel"
 
 
 def recorded_traffic(key):

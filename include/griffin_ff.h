@@ -154,10 +154,10 @@ typedef struct {
  * travel.  RING: bulk copies (TMA) by a producer warp into a ring of shared-memory stages that two
  * groups of consumer warps read.  STREAM: every one of 16 warps loads its own rows straight into
  * registers with plain 16-byte loads, two steps deep.  Without either flag the call picks by size:
- * the register stream is the faster one once every warp has enough to do (about 200 MB of weights
+ * the register stream is the faster one once every warp has enough to do (about 150 MB of weights
  * per call on a B200: 6.7 TB/s against 6.0-6.3 on the Llama-2-13B shape with 8 sets), the ring
  * when the call is so short that filling and draining 2368 separate pipelines shows (Llama-2-7B
- * shape, one sequence: 24.8 against 26.4 us).  Giving both is an error.  Results of the two agree
+ * shape, one sequence: 24.8 against 24.9-25.2 us).  Giving both is an error.  Results of the two agree
  * within the documented tolerance (the sums are taken in different orders). */
 #define GRIFFIN_DECODE_RING 4u
 #define GRIFFIN_DECODE_STREAM 8u

@@ -393,7 +393,7 @@ static griffin_status decode_simt(DecodeParams &p, int act, bool gated, uint32_t
 
 // Weight bytes of a call from which the register-streaming kernel is the default.
 #ifndef GRIFFIN_STREAM_MIN_MB
-#define GRIFFIN_STREAM_MIN_MB 200
+#define GRIFFIN_STREAM_MIN_MB 150
 #endif
 griffin_status launch_decode(const griffin_ff_desc *desc, int B, const griffin_ff_compact *sets, const void *b_down,
                              const void *x, void *y, float *z, void *ws, uint32_t flags, cudaStream_t stream) {
