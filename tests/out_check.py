@@ -12,7 +12,7 @@ import os
 
 import numpy as np
 
-NORTH_STAR_L2 = {"f32": 1e-4, "bf16": 2e-2}      # the stated bounds on the relative L2 error
+STATED_L2 = {"f32": 1e-4, "bf16": 2e-2}      # the stated bounds on the relative L2 error
 # bf16 storage: y is rounded to bf16 (half an ulp = 2^-9 of the element, elements reach 4-5 rms) and the
 # activations between the two products are rounded to bf16 (2^-9 each, averaging out over k terms);
 # measured worst case over the suite (1123 outputs): relative L2 3.0e-3, largest element error 0.019 rms.
@@ -42,7 +42,7 @@ def assert_output(y, ref, dtype, what=None, scale=1.0):
     l2, mx = output_error(y, ref)
     s = _stats.setdefault(dtype, [0.0, 0.0, 0])
     s[0], s[1], s[2] = max(s[0], l2 / scale), max(s[1], mx / scale), s[2] + 1
-    assert l2 <= NORTH_STAR_L2[dtype], ("relative L2 beyond the stated bound", what, l2)
+    assert l2 <= STATED_L2[dtype], ("relative L2 beyond the stated bound", what, l2)
     if os.environ.get("GRIFFIN_TEST_STATS") == "loose":     # collecting the worst case: only the stated bound applies
         return l2, mx
     assert l2 <= scale * TEST_L2[dtype], ("relative L2", what, l2)

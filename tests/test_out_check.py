@@ -6,7 +6,7 @@ import pytest
 import torch
 
 from oracle import griffin_oracle as O
-from out_check import NORTH_STAR_L2, assert_output, output_error
+from out_check import STATED_L2, assert_output, output_error
 
 
 def _decode_output(d=4096, k=512, seed=3):
@@ -35,7 +35,7 @@ def test_one_wrong_element_of_a_wide_vector_is_caught_although_the_l2_error_is_i
     i = int(np.argmin(np.abs(y)))            # the least conspicuous place: an element near zero ...
     bad[i] = np.sqrt(np.mean(y ** 2))        # ... that comes out as a typical element's size
     l2, mx = output_error(bad, y)
-    assert l2 < NORTH_STAR_L2["bf16"]        # 1/64: the stated metric alone would pass it
+    assert l2 < STATED_L2["bf16"]        # 1/64: the stated metric alone would pass it
     with pytest.raises(AssertionError):
         assert_output(bad, y, "bf16")
 
@@ -46,7 +46,7 @@ def test_a_wrong_32_column_segment_of_a_prompt_output_is_caught():
     bad = _as_bf16(y)
     bad[100, 64:96] = 0.0                    # a dropped store of one 64-byte piece
     l2, _ = output_error(bad, y)
-    assert l2 < NORTH_STAR_L2["bf16"]
+    assert l2 < STATED_L2["bf16"]
     with pytest.raises(AssertionError):
         assert_output(bad, y, "bf16")
 
