@@ -64,6 +64,9 @@ def parse_args():
     ap.add_argument("--no-graph", action="store_true", help="launch every decode call from the host instead of replaying a CUDA graph")
     ap.add_argument("--decode", default="compact", choices=["compact", "indexed"],
                     help="indexed: no compaction step, the decode calls read the expert rows in place from the full weights")
+    ap.add_argument("--decode-kernel", default="auto", choices=["auto", "ring", "stream"],
+                    help="bf16, sequences with their own sets: force one of the two warp-level decode kernels "
+                         "(auto: the library picks by the size of the call)")
     ap.add_argument("--shared-set", action="store_true",
                     help="the batch statistic of Eq. 7 in place of per-sequence sets: every sequence of a decode call uses the "
                          "first sequence's expert set, so the weights are streamed once per call")
@@ -83,25 +86,27 @@ def measured_peaks():
         return FALLBACK_HBM_GBS, 1590.0, 1400.0, "fallback (6.65 TB/s, 1.59 / 1.40 PFLOP/s: earlier measurements on this pool)"
 
 
-def decode_kernel_name(w, B, k):
+def decode_kernel_name(w, B, k, forced="auto"):
     """Which of the two warp-level kernels griffin_ff_decode picks for sequences with their own sets (bf16): the
     register stream from about 150 MB of compact weights per call, the shared-memory ring below (the rule stated
     with GRIFFIN_DECODE_RING / GRIFFIN_DECODE_STREAM in include/griffin_ff.h)."""
     if w.dtype != "bf16":
         return "decode_gate_up_kernel + decode_down_kernel"
+    if forced != "auto":
+        return {"ring": "decode_fused_kernel", "stream": "decode_stream_kernel"}[forced]
     return "decode_stream_kernel" if B * 3 * k * w.d * 2 >= 150e6 else "decode_fused_kernel"
 
 
-def recorded_traffic(key):
-    """DRAM bytes per launch of the dominant kernel from the committed ncu summary of this workload, if the
-    kernel's sources are unchanged since that capture; otherwise None."""
+def recorded_traffic(key, kernel):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary of this workload, if it is the
+    kernel that ran and its sources are unchanged since that capture; otherwise None."""
     p = os.path.join(ROOT, "profiles", "decode_traffic.json")
     try:
         rec = json.load(open(p))[key]
         h = hashlib.sha1()
         for name in rec["sources"]:
             h.update(open(os.path.join(ROOT, name), "rb").read())
-        if h.hexdigest() == rec["sha1"]:
+        if h.hexdigest() == rec["sha1"] and rec.get("kernel") == kernel:
             return rec["dram_bytes_per_decode_call"]
     except Exception:
         pass
@@ -576,6 +581,7 @@ def run_ours(args, w, keep):
     B = args.batch or w.B
     indexed = args.decode == "indexed"
     job = Job(w, B, keep, L, dev, rank, indexed, not args.no_graph, shared_set=args.shared_set)
+    job.stack.decode_flags = {"auto": 0, "ring": 4, "stream": 8}[args.decode_kernel]   # GRIFFIN_DECODE_RING / _STREAM
     T, S = job.T, job.S
     job.warm_up(args.warmup)
     barrier()
@@ -651,12 +657,13 @@ def run_ours(args, w, keep):
             "phases": dict(rep, note="medians over the timed steps of per-phase CUDA-event times"),
             "roofline": {"bound": "hbm", "kernel": ("decode_indexed_kernel" if indexed else
                                                     "decode_shared_kernel" if job.shared_set else
-                                                    decode_kernel_name(w, B, job.k)) +
+                                                    decode_kernel_name(w, B, job.k, args.decode_kernel)) +
                          " (one launch per decode call; the decode phase is "
                          f"{100.0 * ph_ms[3] / sum(ph_ms):.0f} % of the step)", "achieved": dec["gbs"],
                          "peak": peaks[0], "unit": "GB/s", "frac": dec["frac_of_hbm"], "peak_source": peaks[3],
                          "algorithmic_bytes_per_launch": dec["algorithmic_bytes_per_call"],
-                         "traffic": None if indexed or job.shared_set else recorded_traffic(traffic_key)},
+                         "traffic": None if indexed or job.shared_set else
+                         recorded_traffic(traffic_key, decode_kernel_name(w, B, job.k, args.decode_kernel))},
             "clocks": clocks,
             "gpu_launches": job.launches_per_step * K,
             "gpu_launches_per_step": job.launches_per_step,

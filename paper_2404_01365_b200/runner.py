@@ -29,6 +29,7 @@ class FFStack:
         self.ldk = G.griffin_compact_ldk(k)
         self.ws = G.alloc_workspace(self.desc, S_max, n_seq, device)
         self.indexed = indexed
+        self.decode_flags = 0  # GRIFFIN_DECODE_RING / _STREAM / _TCGEN05 to add to every decode call (0: the library's own choice)
         self.weights = []      # per block: binding.FFWeights
         self.weights_nm = []   # per block (indexed only): binding.FFWeightsNM
         self.score = torch.empty((L, n_seq, d_ff), device=device, dtype=torch.float32)
@@ -62,7 +63,7 @@ class FFStack:
     def decode(self, layer, x, y, overlap):
         """Pruned FF for one token of each of the n_seq sequences: x, y are [n_seq, d]."""
         G.griffin_ff_decode(self.desc, self.set_arrays[layer], None, x, y, self.ws,
-                            G.DECODE_OVERLAP_WEIGHT_PREFETCH if overlap else G.DECODE_DEFAULT)
+                            (G.DECODE_OVERLAP_WEIGHT_PREFETCH if overlap else G.DECODE_DEFAULT) | self.decode_flags)
 
     def decode_indexed(self, layer, x, y, overlap):
         """The same without compact sets: the rows idx[layer] are read from the full weights."""
