@@ -26,6 +26,7 @@ struct WsHeader {
     unsigned int meet_tc;    // ... and of the tcgen05 one (the two have different numbers of parties)
     unsigned int meet_idx;   // ... and of the index-direct one
     unsigned int meet_stream;  // ... and of the register-streaming one
+    unsigned int pool_stream;  // that kernel's count of claims on its pool of pairs (runs round once per call)
 };
 
 __device__ __forceinline__ void raise_status(void *ws, int status, int detail) {

@@ -64,8 +64,8 @@ __device__ __forceinline__ StreamGeom stream_geom(const DecodeParams &p, int mod
 struct StreamRange {
     int f0, sp0, n, b0;
 };
-__device__ __forceinline__ StreamRange stream_range(const DecodeParams &p, const StreamGeom &g, int warp) {
-    const long long T = (long long)p.B * g.P;
+// T: the pairs dealt out this way (all B * P of the half, or what the pool below leaves)
+__device__ __forceinline__ StreamRange stream_range(const StreamGeom &g, long long T, int warp) {
     const int lo = (int)(T * blockIdx.x / gridDim.x), hi = (int)(T * (blockIdx.x + 1) / gridDim.x);
     const int n = (hi - lo) * g.S;  // the CTA's steps
     const int s0 = (int)((long long)n * warp / ST_WARPS), s1 = (int)((long long)n * (warp + 1) / ST_WARPS);
@@ -160,11 +160,12 @@ struct StreamHalf {
         }
     }
 
-    __device__ __forceinline__ void init(const DecodeParams &p, int warp_, int lane_) {
+    // pool_pairs: pairs at the end of the half that are not dealt out here (see the pool in the kernel)
+    __device__ __forceinline__ void init(const DecodeParams &p, int warp_, int lane_, int pool_pairs = 0) {
         warp = warp_;
         lane = lane_;
         g = stream_geom(p, MODE);
-        const StreamRange r = stream_range(p, g, warp);
+        const StreamRange r = stream_range(g, (long long)p.B * g.P - pool_pairs, warp);
         b0 = r.b0;
         f_slot1 = (b0 + 1) * g.P;
         n_issue = n_comp = r.n;
@@ -175,6 +176,21 @@ struct StreamHalf {
         r0 = r1 = nullptr;
         two = false;
         if (n_issue > 0) set_pair(p, lf);
+    }
+
+    // This warp takes the whole of pair f and nothing else; its vector is slot 0 of the `vec` given to run().
+    __device__ __forceinline__ void init_single(const DecodeParams &p, int warp_, int lane_, int f) {
+        warp = warp_;
+        lane = lane_;
+        g = stream_geom(p, MODE);
+        b0 = f / g.P;
+        f_slot1 = 0x7fffffff;
+        n_issue = n_comp = g.S;
+        n_staged = 0;
+        cf = lf = f;
+        csp = lsp = 0;
+        mid = false;
+        set_pair(p, lf);
     }
 
     // Loads the next step into r and moves the load cursor on.
@@ -381,23 +397,26 @@ __device__ __forceinline__ uint4 ld_cg_now(const uint4 *p) {  // through L2; vol
 }
 
 // Stages the vectors of sequences b0 and b0 + 1 (x: row_units units each; z: the same with the entries
-// from k on cleared) as two rows of vec_units units, zero-filled.  The loads of the first
+// from k on cleared) as rows of vec_units units, zero-filled.  The loads of the first
 // ST_VEC_EARLY units per thread are issued before `between` runs and stored after it: what `between`
 // asks the memory system for arrives behind the vector.
 constexpr int ST_VEC_EARLY = 4;
+// n_slots = 3: a third row holds the vector of the last sequence (for the pool of the first half).
 template <bool IS_Z, class F>
-__device__ __forceinline__ void stage_vectors(const DecodeParams &p, uint4 *vec, int vec_units, int b0, int tid, F between) {
+__device__ __forceinline__ void stage_vectors(const DecodeParams &p, uint4 *vec, int vec_units, int n_slots, int b0, int tid,
+                                              F between) {
     const int row_units = (IS_Z ? p.ldk : p.d) / 8;
     const int limit = IS_Z ? p.k : p.d;  // elements that exist
     const uint4 zero = make_uint4(0, 0, 0, 0);
     auto src_of = [&](int u, bool &in) -> const uint4 * {
-        const int slot = u >= vec_units ? 1 : 0, uu = u - slot * vec_units, b = b0 + slot;
-        in = u < 2 * vec_units && uu < row_units && 8 * uu < limit && b < p.B;
+        const int slot = u >= 2 * vec_units ? 2 : (u >= vec_units ? 1 : 0), uu = u - slot * vec_units;
+        const int b = slot == 2 ? p.B - 1 : b0 + slot;
+        in = u < n_slots * vec_units && uu < row_units && 8 * uu < limit && b < p.B;
         if (IS_Z) return reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(p.z) + (size_t)b * 2 * p.ldk) + uu;
         return static_cast<const uint4 *>(p.x) + (size_t)b * row_units + uu;
     };
     auto fix = [&](uint4 v, int u) -> uint4 {
-        const int slot = u >= vec_units ? 1 : 0, uu = u - slot * vec_units;
+        const int slot = u >= 2 * vec_units ? 2 : (u >= vec_units ? 1 : 0), uu = u - slot * vec_units;
         return (IS_Z && 8 * uu + 8 > limit) ? keep_elems(v, limit - 8 * uu) : v;
     };
     uint4 early[ST_VEC_EARLY];
@@ -411,9 +430,9 @@ __device__ __forceinline__ void stage_vectors(const DecodeParams &p, uint4 *vec,
 #pragma unroll
     for (int i = 0; i < ST_VEC_EARLY; ++i) {
         const int u = tid + i * ST_THREADS;
-        if (u < 2 * vec_units) vec[u] = fix(early[i], u);
+        if (u < n_slots * vec_units) vec[u] = fix(early[i], u);
     }
-    for (int u = tid + ST_VEC_EARLY * ST_THREADS; u < 2 * vec_units; u += ST_THREADS) {
+    for (int u = tid + ST_VEC_EARLY * ST_THREADS; u < n_slots * vec_units; u += ST_THREADS) {
         bool in;
         const uint4 *src = src_of(u, in);
         vec[u] = in ? fix(__ldcg(src), u) : zero;
@@ -422,12 +441,14 @@ __device__ __forceinline__ void stage_vectors(const DecodeParams &p, uint4 *vec,
 
 template <bool GATED>
 __global__ void __launch_bounds__(ST_THREADS, 1) decode_stream_kernel(const __grid_constant__ DecodeParams p, int act,
-                                                                    int vec_units, int ahead) {
+                                                                    int vec_units, int ahead, int pool_chunks) {
     constexpr int FIRST = GATED ? ST_GATE_UP : ST_UP;
     extern __shared__ __align__(128) uint8_t smem_raw[];
-    uint4 *vec = reinterpret_cast<uint4 *>(smem_raw);                       // two vectors of vec_units units
-    StreamPartial *part = reinterpret_cast<StreamPartial *>(vec + 2 * vec_units);
-    volatile int *abort = reinterpret_cast<volatile int *>(part + 2 * ST_WARPS);
+    const int n_slots = pool_chunks > 0 ? 3 : 2;
+    uint4 *vec = reinterpret_cast<uint4 *>(smem_raw);                       // n_slots vectors of vec_units units
+    StreamPartial *part = reinterpret_cast<StreamPartial *>(vec + n_slots * vec_units);
+    volatile int *abort = reinterpret_cast<volatile int *>(part + 2 * ST_WARPS);  // [0]: abort flag; [2], [3]: claims of the pool
+    volatile int *claim = abort + 2;
     uint64_t *bars = reinterpret_cast<uint64_t *>(const_cast<int *>(abort) + 4);  // [2 halves][ST_WARPS]
     uint4 *stages = reinterpret_cast<uint4 *>(bars + 2 * ST_WARPS);                 // [ST_WARPS][ahead] steps
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -452,15 +473,40 @@ __global__ void __launch_bounds__(ST_THREADS, 1) decode_stream_kernel(const __gr
     // ---- first half: the first weights are on their way before anything else happens
     uint4 A[2 * ST_H], Bq[2 * ST_H];
     StreamHalf<FIRST> h1;
-    h1.init(p, warp, lane);
+    h1.init(p, warp, lane, pool_chunks * ST_WARPS);
     h1.prologue_regs(p, A, Bq);
+    // the first claim on the pool (asked for now, needed when this CTA's own share is done)
+    unsigned int *const pool = &static_cast<WsHeader *>(p.ws)->pool_stream;
+    int my_claim = 0;
+    if (pool_chunks > 0 && tid == 0) my_claim = (int)atomicInc(pool, (unsigned int)pool_chunks + gridDim.x - 1);
     pdl_launch_dependents();
     if (tid == 0) *abort = 0;
     if (tid < 2 * ST_WARPS) part[tid].f = -1;
     pdl_wait_prior_grids();  // x, the z scratch and the outputs belong to earlier work on the stream
-    stage_vectors<false>(p, vec, vec_units, h1.b0, tid, [&]() { h1.prologue_staged(p, stage, bar1, ahead); });
+    stage_vectors<false>(p, vec, vec_units, n_slots, h1.b0, tid, [&]() { h1.prologue_staged(p, stage, bar1, ahead); });
     __syncthreads();
     h1.run(p, A, Bq, stage, bar1, vec, vec_units, part, abort, act);
+    // ---- the pool: the last pool_chunks * 16 pairs of the half (all of the last sequence) are not dealt out
+    //      beforehand but handed out at run time, 16 whole pairs (one per warp) at a time, to the CTAs that are done
+    //      with their own share: at saturation some groups of SMs get 8 % less out of the memory system than the
+    //      others, and the meeting point below waits for the slowest.  Whole pairs, each summed by one warp in the
+    //      order of its steps: the result does not depend on who takes what.  Every CTA claims until it is told that
+    //      nothing is left, exactly once: pool_chunks + gridDim.x claims per call take the counter round to where
+    //      it was.
+    if (pool_chunks > 0) {
+        const int pool_base = p.B * h1.g.P - pool_chunks * ST_WARPS;
+        for (int it = 0;; ++it) {
+            if (tid == 0) claim[it & 1] = my_claim;
+            __syncthreads();  // (also: every warp is done with its share, or with the chunk before)
+            const int chunk = claim[it & 1];
+            if (chunk >= pool_chunks || *abort) break;
+            StreamHalf<FIRST> hp;
+            hp.init_single(p, warp, lane, pool_base + chunk * ST_WARPS + warp);
+            hp.prologue_regs(p, A, Bq);
+            if (tid == 0) my_claim = (int)atomicInc(pool, (unsigned int)pool_chunks + gridDim.x - 1);  // (needed next time round)
+            hp.run(p, A, Bq, stage, bar1, vec + 2 * vec_units, vec_units, part, abort, act);
+        }
+    }
     // the first weights of the second half, as soon as this warp has room for them
     StreamHalf<ST_DOWN> h2;
     h2.init(p, warp, lane);
@@ -489,7 +535,7 @@ __global__ void __launch_bounds__(ST_THREADS, 1) decode_stream_kernel(const __gr
         return;
     }
     // z of the two sequences, read through L2 (other CTAs wrote it); the staged step is asked for behind it
-    stage_vectors<true>(p, vec, vec_units, h2.b0, tid, [&]() {
+    stage_vectors<true>(p, vec, vec_units, 2, h2.b0, tid, [&]() {
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the staged steps of the first half have been read
         h2.prologue_staged(p, stage, bar2, ahead);
     });
@@ -503,6 +549,12 @@ __global__ void __launch_bounds__(ST_THREADS, 1) decode_stream_kernel(const __gr
     if (warp == 0) combine_partials<ST_DOWN>(p, part, act, lane);
 }
 
+#ifndef GRIFFIN_ST_POOL_PCT
+#define GRIFFIN_ST_POOL_PCT 8
+#endif
+#ifndef GRIFFIN_ST_POOL_MIN
+#define GRIFFIN_ST_POOL_MIN 16
+#endif
 #ifndef GRIFFIN_ST_AHEAD
 #define GRIFFIN_ST_AHEAD 1
 #endif
@@ -516,7 +568,20 @@ griffin_status decode_bf16_stream(DecodeParams &p, int act, bool gated, uint32_t
     const bool overlap = (flags & GRIFFIN_DECODE_OVERLAP_WEIGHT_PREFETCH) != 0;
     const int units = max(p.d, p.ldk) / 8;
     int vec_units = (units + ST_STEP_UNITS - 1) / ST_STEP_UNITS * ST_STEP_UNITS;
-    const size_t fixed = (size_t)2 * vec_units * 16 + 2 * ST_WARPS * sizeof(StreamPartial) + 16 + 2 * ST_WARPS * sizeof(uint64_t);
+    // The pool of the first half: GRIFFIN_ST_POOL_PCT per cent of its pairs, in chunks of 16, all within the last
+    // sequence; only when every warp has at least GRIFFIN_ST_POOL_MIN pairs of its own (the chunks cost a barrier each
+    // and restart the pipelines).  Measured on B200: Llama-2-13B shape, 8 sets (23 pairs per warp): 252.6 us per call
+    // without, 251.4 / 245.7 / 245.2 with 5 / 8 / 12 per cent; Mistral shape, 4 sets (12 pairs per warp): 107.2 without,
+    // 107.9 - 108.8 with, hence the threshold.
+    const long long pairs1 = (long long)p.B * (gated ? p.k : (p.k + 1) / 2), per_seq1 = gated ? p.k : (p.k + 1) / 2;
+    int pool_chunks = 0;
+    if (GRIFFIN_ST_POOL_PCT > 0 && pairs1 / ((long long)grid * ST_WARPS) >= GRIFFIN_ST_POOL_MIN) {
+        long long pool_pairs = pairs1 * GRIFFIN_ST_POOL_PCT / 100;
+        if (pool_pairs > per_seq1) pool_pairs = per_seq1;
+        pool_chunks = (int)(pool_pairs / ST_WARPS);
+    }
+    const size_t fixed = (size_t)(pool_chunks > 0 ? 3 : 2) * vec_units * 16 + 2 * ST_WARPS * sizeof(StreamPartial) + 16 +
+                         2 * ST_WARPS * sizeof(uint64_t);
     if (fixed > 227 * 1024) return GRIFFIN_ERR_UNSUPPORTED;
     // Steps per warp staged in shared memory across the waits.  Shared memory is taken from the
     // same 256 KB as the L1 cache, which the loads in flight pass through: measured on B200, with
@@ -530,7 +595,7 @@ griffin_status decode_bf16_stream(DecodeParams &p, int act, bool gated, uint32_t
     if (ensure_dynamic_smem(fn, smem) != cudaSuccess) return GRIFFIN_ERR_CUDA;
     // every CTA of the grid must be able to run at the same time (they meet half-way): one per SM
     if (!grid_can_meet(fn, ST_THREADS, smem, grid)) return GRIFFIN_ERR_UNSUPPORTED;
-    void *args[] = {&p, &act, &vec_units, &ahead};
+    void *args[] = {&p, &act, &vec_units, &ahead, &pool_chunks};
     if (launch_maybe_overlapped(fn, dim3(grid), dim3(ST_THREADS), smem, stream, overlap, args) != cudaSuccess)
         return GRIFFIN_ERR_CUDA;
     return GRIFFIN_OK;

@@ -77,6 +77,41 @@ def test_every_step_is_taken_once_and_ranges_span_two_sequences_at_most(d, k, ld
         assert not full_step or u < row_units
 
 
+def pool_chunks(B, k, gated, grid, pct=8, min_pairs_per_warp=16):
+    """The launcher's rule for the pool of the first half (pairs handed out at run time, 16 at a time)."""
+    per_seq = k if gated else (k + 1) // 2
+    pairs = B * per_seq
+    if pairs // (grid * ST_WARPS) < min_pairs_per_warp:
+        return 0
+    return min(per_seq, pairs * pct // 100) // ST_WARPS
+
+
+@pytest.mark.parametrize("B,k,gated", [(8, 6912, True), (8, 6912, False), (32, 5504, True), (4, 7168, True), (16, 24576, True)])
+def test_the_pool_lies_in_the_last_sequence_and_the_rest_is_dealt_out_as_before(B, k, gated):
+    grid = 148
+    per_seq = k if gated else (k + 1) // 2
+    T = B * per_seq
+    n = pool_chunks(B, k, gated, grid)
+    if T // (grid * ST_WARPS) < 16:                      # e.g. the Mistral shape with 4 sets: 12 pairs per warp
+        assert n == 0
+        return
+    assert n > 0
+    pool_base = T - n * ST_WARPS
+    assert pool_base // per_seq == B - 1 and (T - 1) // per_seq == B - 1      # one vector (the third slot) serves the pool
+    covered = 0
+    for cta in range(grid):
+        lo, hi = (T - n * ST_WARPS) * cta // grid, (T - n * ST_WARPS) * (cta + 1) // grid
+        covered += hi - lo
+        if hi > lo:
+            assert (hi - 1) // per_seq - lo // per_seq <= 1
+    assert covered == pool_base and covered + n * ST_WARPS == T
+    # the claims of one call take the counter round: n successful ones and one failing per CTA
+    counter, limit = 0, n + grid - 1
+    for _ in range(n + grid):
+        counter = 0 if counter >= limit else counter + 1
+    assert counter == 0
+
+
 def test_the_size_rule_of_the_bench_names_the_kernel_the_library_picks():
     import bench
     from paper_2404_01365_b200 import synth
