@@ -397,26 +397,23 @@ __device__ __forceinline__ uint4 ld_cg_now(const uint4 *p) {  // through L2; vol
 }
 
 // Stages the vectors of sequences b0 and b0 + 1 (x: row_units units each; z: the same with the entries
-// from k on cleared) as rows of vec_units units, zero-filled.  The loads of the first
+// from k on cleared) as two rows of vec_units units, zero-filled.  The loads of the first
 // ST_VEC_EARLY units per thread are issued before `between` runs and stored after it: what `between`
 // asks the memory system for arrives behind the vector.
 constexpr int ST_VEC_EARLY = 4;
-// n_slots = 3: a third row holds the vector of the last sequence (for the pool of the first half).
 template <bool IS_Z, class F>
-__device__ __forceinline__ void stage_vectors(const DecodeParams &p, uint4 *vec, int vec_units, int n_slots, int b0, int tid,
-                                              F between) {
+__device__ __forceinline__ void stage_vectors(const DecodeParams &p, uint4 *vec, int vec_units, int b0, int tid, F between) {
     const int row_units = (IS_Z ? p.ldk : p.d) / 8;
     const int limit = IS_Z ? p.k : p.d;  // elements that exist
     const uint4 zero = make_uint4(0, 0, 0, 0);
     auto src_of = [&](int u, bool &in) -> const uint4 * {
-        const int slot = u >= 2 * vec_units ? 2 : (u >= vec_units ? 1 : 0), uu = u - slot * vec_units;
-        const int b = slot == 2 ? p.B - 1 : b0 + slot;
-        in = u < n_slots * vec_units && uu < row_units && 8 * uu < limit && b < p.B;
+        const int slot = u >= vec_units ? 1 : 0, uu = u - slot * vec_units, b = b0 + slot;
+        in = u < 2 * vec_units && uu < row_units && 8 * uu < limit && b < p.B;
         if (IS_Z) return reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(p.z) + (size_t)b * 2 * p.ldk) + uu;
         return static_cast<const uint4 *>(p.x) + (size_t)b * row_units + uu;
     };
     auto fix = [&](uint4 v, int u) -> uint4 {
-        const int slot = u >= 2 * vec_units ? 2 : (u >= vec_units ? 1 : 0), uu = u - slot * vec_units;
+        const int slot = u >= vec_units ? 1 : 0, uu = u - slot * vec_units;
         return (IS_Z && 8 * uu + 8 > limit) ? keep_elems(v, limit - 8 * uu) : v;
     };
     uint4 early[ST_VEC_EARLY];
@@ -430,9 +427,9 @@ __device__ __forceinline__ void stage_vectors(const DecodeParams &p, uint4 *vec,
 #pragma unroll
     for (int i = 0; i < ST_VEC_EARLY; ++i) {
         const int u = tid + i * ST_THREADS;
-        if (u < n_slots * vec_units) vec[u] = fix(early[i], u);
+        if (u < 2 * vec_units) vec[u] = fix(early[i], u);
     }
-    for (int u = tid + ST_VEC_EARLY * ST_THREADS; u < n_slots * vec_units; u += ST_THREADS) {
+    for (int u = tid + ST_VEC_EARLY * ST_THREADS; u < 2 * vec_units; u += ST_THREADS) {
         bool in;
         const uint4 *src = src_of(u, in);
         vec[u] = in ? fix(__ldcg(src), u) : zero;
@@ -444,9 +441,11 @@ __global__ void __launch_bounds__(ST_THREADS, 1) decode_stream_kernel(const __gr
                                                                     int vec_units, int ahead, int pool_chunks) {
     constexpr int FIRST = GATED ? ST_GATE_UP : ST_UP;
     extern __shared__ __align__(128) uint8_t smem_raw[];
-    const int n_slots = pool_chunks > 0 ? 3 : 2;
-    uint4 *vec = reinterpret_cast<uint4 *>(smem_raw);                       // n_slots vectors of vec_units units
-    StreamPartial *part = reinterpret_cast<StreamPartial *>(vec + n_slots * vec_units);
+    // two vectors of vec_units units and, for the pool of the first half, x of the last sequence (x_units units)
+    const int x_units = pool_chunks > 0 ? (p.d / 8 + ST_STEP_UNITS - 1) / ST_STEP_UNITS * ST_STEP_UNITS : 0;
+    uint4 *vec = reinterpret_cast<uint4 *>(smem_raw);
+    uint4 *vec_pool = vec + 2 * vec_units;
+    StreamPartial *part = reinterpret_cast<StreamPartial *>(vec_pool + x_units);
     volatile int *abort = reinterpret_cast<volatile int *>(part + 2 * ST_WARPS);  // [0]: abort flag; [2], [3]: claims of the pool
     volatile int *claim = abort + 2;
     uint64_t *bars = reinterpret_cast<uint64_t *>(const_cast<int *>(abort) + 4);  // [2 halves][ST_WARPS]
@@ -483,7 +482,9 @@ __global__ void __launch_bounds__(ST_THREADS, 1) decode_stream_kernel(const __gr
     if (tid == 0) *abort = 0;
     if (tid < 2 * ST_WARPS) part[tid].f = -1;
     pdl_wait_prior_grids();  // x, the z scratch and the outputs belong to earlier work on the stream
-    stage_vectors<false>(p, vec, vec_units, n_slots, h1.b0, tid, [&]() { h1.prologue_staged(p, stage, bar1, ahead); });
+    stage_vectors<false>(p, vec, vec_units, h1.b0, tid, [&]() { h1.prologue_staged(p, stage, bar1, ahead); });
+    for (int u = tid; u < x_units; u += ST_THREADS)
+        vec_pool[u] = u < p.d / 8 ? __ldcg(static_cast<const uint4 *>(p.x) + (size_t)(p.B - 1) * (p.d / 8) + u) : make_uint4(0, 0, 0, 0);
     __syncthreads();
     h1.run(p, A, Bq, stage, bar1, vec, vec_units, part, abort, act);
     // ---- the pool: the last pool_chunks * 16 pairs of the half (all of the last sequence) are not dealt out
@@ -504,7 +505,7 @@ __global__ void __launch_bounds__(ST_THREADS, 1) decode_stream_kernel(const __gr
             hp.init_single(p, warp, lane, pool_base + chunk * ST_WARPS + warp);
             hp.prologue_regs(p, A, Bq);
             if (tid == 0) my_claim = (int)atomicInc(pool, (unsigned int)pool_chunks + gridDim.x - 1);  // (needed next time round)
-            hp.run(p, A, Bq, stage, bar1, vec + 2 * vec_units, vec_units, part, abort, act);
+            hp.run(p, A, Bq, stage, bar1, vec_pool, vec_units, part, abort, act);
         }
     }
     // the first weights of the second half, as soon as this warp has room for them
@@ -535,7 +536,7 @@ __global__ void __launch_bounds__(ST_THREADS, 1) decode_stream_kernel(const __gr
         return;
     }
     // z of the two sequences, read through L2 (other CTAs wrote it); the staged step is asked for behind it
-    stage_vectors<true>(p, vec, vec_units, 2, h2.b0, tid, [&]() {
+    stage_vectors<true>(p, vec, vec_units, h2.b0, tid, [&]() {
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the staged steps of the first half have been read
         h2.prologue_staged(p, stage, bar2, ahead);
     });
@@ -558,7 +559,7 @@ __global__ void __launch_bounds__(ST_THREADS, 1) decode_stream_kernel(const __gr
 #ifndef GRIFFIN_ST_AHEAD
 #define GRIFFIN_ST_AHEAD 1
 #endif
-constexpr size_t ST_SMEM_BUDGET = 128 * 1024;  // shared memory that vectors and staged steps may take together
+constexpr size_t ST_SMEM_BUDGET = 144 * 1024;  // shared memory that vectors and staged steps may take together
 griffin_status decode_bf16_stream(DecodeParams &p, int act, bool gated, uint32_t flags, cudaStream_t stream) {
     const int sms = device_sm_count();
     if (sms <= 0) return GRIFFIN_ERR_CUDA;
@@ -569,18 +570,21 @@ griffin_status decode_bf16_stream(DecodeParams &p, int act, bool gated, uint32_t
     const int units = max(p.d, p.ldk) / 8;
     int vec_units = (units + ST_STEP_UNITS - 1) / ST_STEP_UNITS * ST_STEP_UNITS;
     // The pool of the first half: GRIFFIN_ST_POOL_PCT per cent of its pairs, in chunks of 16, all within the last
-    // sequence; only when every warp has at least GRIFFIN_ST_POOL_MIN pairs of its own (the chunks cost a barrier each
-    // and restart the pipelines).  Measured on B200: Llama-2-13B shape, 8 sets (23 pairs per warp): 252.6 us per call
-    // without, 251.4 / 245.7 / 245.2 with 5 / 8 / 12 per cent; Mistral shape, 4 sets (12 pairs per warp): 107.2 without,
-    // 107.9 - 108.8 with, hence the threshold.
+    // sequence; only when every warp has at least GRIFFIN_ST_POOL_MIN pairs of its own and a pair has four steps or
+    // more (the chunks cost a barrier each and restart the pipelines, with one pair per warp to fill them).  Measured
+    // on B200, us per call without / with: Llama-2-13B shape, 8 sets (23 pairs per warp) 250.8 / 243.2 (5 per cent:
+    // no gain, 12: as 8); Llama-2-7B shape, 8 sets 163.1 / 158.6; Mistral shape, 4 sets, keep 0.75 158.0 / 152.8, keep 1.0
+    // 205.5 / 207.9, keep 0.5 (12 pairs per warp) 107.2 / 107.9 - 108.8; Gemma shape, 4 sets (pairs of three steps)
+    // 133.8 / 136.8.
     const long long pairs1 = (long long)p.B * (gated ? p.k : (p.k + 1) / 2), per_seq1 = gated ? p.k : (p.k + 1) / 2;
     int pool_chunks = 0;
-    if (GRIFFIN_ST_POOL_PCT > 0 && pairs1 / ((long long)grid * ST_WARPS) >= GRIFFIN_ST_POOL_MIN) {
+    if (GRIFFIN_ST_POOL_PCT > 0 && pairs1 / ((long long)grid * ST_WARPS) >= GRIFFIN_ST_POOL_MIN && p.d / 8 > 3 * ST_STEP_UNITS) {
         long long pool_pairs = pairs1 * GRIFFIN_ST_POOL_PCT / 100;
         if (pool_pairs > per_seq1) pool_pairs = per_seq1;
         pool_chunks = (int)(pool_pairs / ST_WARPS);
     }
-    const size_t fixed = (size_t)(pool_chunks > 0 ? 3 : 2) * vec_units * 16 + 2 * ST_WARPS * sizeof(StreamPartial) + 16 +
+    const int x_units = pool_chunks > 0 ? (p.d / 8 + ST_STEP_UNITS - 1) / ST_STEP_UNITS * ST_STEP_UNITS : 0;
+    const size_t fixed = (size_t)(2 * vec_units + x_units) * 16 + 2 * ST_WARPS * sizeof(StreamPartial) + 16 +
                          2 * ST_WARPS * sizeof(uint64_t);
     if (fixed > 227 * 1024) return GRIFFIN_ERR_UNSUPPORTED;
     // Steps per warp staged in shared memory across the waits.  Shared memory is taken from the

@@ -77,11 +77,11 @@ def test_every_step_is_taken_once_and_ranges_span_two_sequences_at_most(d, k, ld
         assert not full_step or u < row_units
 
 
-def pool_chunks(B, k, gated, grid, pct=8, min_pairs_per_warp=16):
+def pool_chunks(B, k, gated, grid, d=4096, pct=8, min_pairs_per_warp=16):
     """The launcher's rule for the pool of the first half (pairs handed out at run time, 16 at a time)."""
     per_seq = k if gated else (k + 1) // 2
     pairs = B * per_seq
-    if pairs // (grid * ST_WARPS) < min_pairs_per_warp:
+    if pairs // (grid * ST_WARPS) < min_pairs_per_warp or d // 8 <= 3 * STEP_UNITS:
         return 0
     return min(per_seq, pairs * pct // 100) // ST_WARPS
 
