@@ -127,6 +127,7 @@ DECODE_SHAPES = [
     (256, 688, 344, 32),     # the largest batch
     (128, 64, 1, 2),         # one expert: most CTAs have nothing to do in the first half
     (136, 200, 9, 5),        # rows shorter than one step, odd k, more sequences than pairs per CTA
+    (3136, 4800, 4736, 8),   # 16 pairs per warp in the first half: the register stream hands the last 8 % out at run time
 ]
 
 # The two warp-level kernels for sequences with their own sets (bf16), and the choice by size.

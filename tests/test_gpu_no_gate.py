@@ -105,6 +105,7 @@ DECODE_SHAPES = [
     (5120, 2048, 1024, 8),
     (8192, 1024, 512, 1),
     (512, 9008, 9008, 1),    # k = d_ff, rows of W_2_hat of two chunks
+    (3136, 9504, 9473, 8),   # 16 pairs of rows per warp: the run-time pool of the register stream, ending in a pair of one row
 ]
 
 
